@@ -1,0 +1,18 @@
+"""B200-native physics loss for data-free generative PDE solvers.
+
+``inputs``  -- seeded synthetic workloads (numpy only, no method arithmetic).
+``binding`` -- thin ctypes binding of the C-ABI CUDA library (``libdn.so``):
+               ``dn_kl_field``, ``dn_energy``, ``dn_energy_grad``, ``dn_apply_bc``.
+
+The binding is imported on first attribute access so that the input generators
+can be used without the CUDA library being built.
+"""
+import importlib
+
+__all__ = ["inputs", "binding"]
+
+
+def __getattr__(name):
+    if name in ("binding", "inputs", "build"):
+        return importlib.import_module(f"{__name__}.{name}")
+    raise AttributeError(name)
