@@ -1,0 +1,145 @@
+/*
+ * dn -- physics loss of a data-free generative PDE solver, as CUDA kernels for sm_100a.
+ *
+ * The paper trains a generator of full solution fields without data: the loss scores
+ * a batch of generated fields against the PDE  A_nu(u) = f,  B(u) = b  on the unit
+ * domain ("Mathematical preliminaries", Eq. (pde)), as an expectation over sampled
+ * coefficients nu and boundary data b ("DiffNets", Eq. (pde_loss)), and the gradient
+ * of that loss with respect to the field is what enters back-propagation
+ * (Algorithm 1, local back-propagation step).  This library evaluates that loss for
+ * the diffusion equation
+ *
+ *        -div( nu grad u ) = f   on [0,1]^d, d = 2 or 3,
+ *        u = bc_x0 on x = 0,  u = bc_x1 on x = 1,  zero flux on the other faces,
+ *
+ * in its variational (Ritz/Galerkin) form on a uniform mesh of bilinear / trilinear
+ * (Q1) elements with 2-point-per-axis Gauss quadrature:
+ *
+ *        J(u)  = sum_e sum_q W_q ( 1/2 nu_q |grad u_q|^2 - f_q u_q )          (energy)
+ *        r     = dJ/du = K(nu) u - F,  set to 0 at the Dirichlet nodes         (residual)
+ *
+ * Conventions shared by all entry points
+ *  - Fields are C-ordered [batch][nz][ny][nx] float32 (x fastest; nz = 1 in 2D).  Node
+ *    (ix,iy,iz) sits at (ix*hx, iy*hy, iz*hz), h_a = 1/(n_a - 1).  Dirichlet nodes are
+ *    those with ix == 0 or ix == nx-1.
+ *  - Every pointer is a DEVICE pointer unless its name ends in _host; structs are read
+ *    on the host.  The caller owns every buffer.  The library allocates no memory,
+ *    keeps no state between calls and never synchronises (the *_host entry point
+ *    excepted, which returns after its last copy has finished).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
+ *    enqueued on it in order; outputs are valid once that work has finished.
+ *  - Return value: DN_OK or an error code; nothing is thrown, nothing aborts.  When
+ *    validation fails nothing has been enqueued and no output is touched.
+ *  - Results are deterministic: no atomics, fixed reduction order.
+ */
+#ifndef DN_H_
+#define DN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DN_OK = 0,
+    DN_ERR_NULL = 1,       /* a required pointer is NULL                                   */
+    DN_ERR_DIM = 2,        /* dim is not 2 or 3                                            */
+    DN_ERR_SIZE = 3,       /* a grid extent < 2, batch < 1, or an extent beyond the limits */
+    DN_ERR_MODE = 4,       /* unknown nu_mode / bc mode, kl_modes outside 1..DN_MAX_KL_MODES */
+    DN_ERR_WORKSPACE = 5,  /* workspace NULL, misaligned (256 B) or smaller than required  */
+    DN_ERR_CUDA = 6,       /* a CUDA runtime call or kernel launch failed                  */
+    DN_ERR_ALIAS = 7       /* r overlaps u                                                 */
+} dn_status;
+
+typedef enum {
+    DN_NU_NODAL = 0,       /* nu given at the nodes, Q1-interpolated to the Gauss points    */
+    DN_NU_KL_GAUSS = 1     /* nu evaluated from the KL weights at the Gauss points; no field stored */
+} dn_nu_mode;
+
+/* dn_problem.flags */
+#define DN_IMPOSE_BC_ON_LOAD 1u  /* read u as if its x faces held bc_x0 / bc_x1 (u itself is not written) */
+#define DN_NO_MASK           2u  /* keep the raw residual at Dirichlet nodes (tests)                      */
+#define DN_FORCE_GENERIC     4u  /* use the any-size kernels even where a tiled kernel applies (tests)    */
+
+#define DN_MAX_KL_MODES 8        /* largest m (KL modes per axis)                                         */
+#define DN_MAX_EXTENT 32768      /* largest nx, ny or nz                                                  */
+
+typedef struct {
+    int32_t dim;                 /* 2 or 3                                 */
+    int32_t nx, ny, nz;          /* nodes per axis; nz is ignored when dim == 2 */
+} dn_grid;
+
+/* Statement of one batched problem: grid size, batch, diffusivity (KL coefficients or a
+ * nodal field), boundary values and forcing. */
+typedef struct {
+    dn_grid grid;
+    int32_t batch;               /* B >= 1                                                         */
+    int32_t nu_mode;             /* dn_nu_mode                                                     */
+    const float* nu;             /* [B][nz][ny][nx], used when nu_mode == DN_NU_NODAL              */
+    int32_t kl_modes;            /* m, used when nu_mode == DN_NU_KL_GAUSS                         */
+    const float* kl_w;           /* [B][m]^dim, index [b][i-1][j-1]([k-1]); i <-> x, j <-> y, k <-> z */
+    float f_const;               /* forcing when f == NULL                                         */
+    const float* f;              /* optional nodal forcing [B][nz][ny][nx], Q1-interpolated        */
+    float bc_x0, bc_x1;          /* Dirichlet values on x = 0 and x = 1                            */
+    uint32_t flags;              /* DN_* flags above                                               */
+} dn_problem;
+
+/* Bytes of device scratch that dn_energy / dn_energy_grad need for this problem (per-block
+ * energy partials and cosine tables).  0 if the problem is invalid.  The workspace must be
+ * 256-byte aligned; its contents need not be preserved between calls, and two calls that
+ * may overlap on the device need separate workspaces. */
+size_t dn_workspace_bytes(const dn_problem* problem);
+
+/* Bytes of device staging that dn_energy_grad_host needs (u, r, J, weights / nodal fields,
+ * plus dn_workspace_bytes).  0 if the problem is invalid. */
+size_t dn_host_staging_bytes(const dn_problem* problem);
+
+/* Diffusivity sampling ("DiffNets": coefficients nu are sampled per minibatch): writes
+ *   nu[b][node] = exp( sum_{i,j(,k)=1..m} w[b][i-1][j-1]([k-1]) cos(i pi x) cos(j pi y) (cos(k pi z))
+ *                      / (1 + i^2 + j^2 (+ k^2)) )
+ * at the nodes.  kl_w: [B][m]^dim floats; nu_out: [B][nz][ny][nx] floats.  Needs no workspace. */
+dn_status dn_kl_field(const dn_grid* grid, int32_t batch, int32_t kl_modes, const float* kl_w,
+                      float* nu_out, void* stream);
+
+/* Energy only (Eq. (pde_loss) in its variational form): J[b], b < B.  u: [B][nz][ny][nx].
+ * Same value as the J output of dn_energy_grad. */
+dn_status dn_energy(const dn_problem* problem, const float* u, float* J, void* workspace,
+                    size_t workspace_bytes, void* stream);
+
+/* Energy and its exact gradient in one pass over u (Algorithm 1: loss, then its gradient
+ * for back-propagation):  r = K(nu) u - F, zeroed at Dirichlet nodes unless DN_NO_MASK,
+ * multiplied by gJ[b] when gJ != NULL (the upstream dLoss/dJ_b).
+ * J may be NULL (residual only).  r must not overlap u.  gJ: [B] floats or NULL. */
+dn_status dn_energy_grad(const dn_problem* problem, const float* u, const float* gJ, float* J, float* r,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* Boundary operator B(u) = b (Eq. (pde)): overwrites the two Dirichlet faces of a field in
+ * place.  mode 0: field = bc_x0 at ix = 0 and bc_x1 at ix = nx-1;  mode 1: both faces = 0
+ * (e.g. to mask a gradient). */
+dn_status dn_apply_bc(const dn_grid* grid, int32_t batch, float bc_x0, float bc_x1, int32_t mode,
+                      float* field_inout, void* stream);
+
+/* dn_energy_grad with HOST buffers: copies u (and nu / f / kl_w / gJ when present) to the
+ * device staging area, runs the same kernels, copies J and r back, and waits for the last
+ * copy.  In `problem`, nu / kl_w / f are HOST pointers here.  u_host, r_host: [B][..] floats;
+ * J_host: [B] floats or NULL; staging: device memory of dn_host_staging_bytes(problem) bytes,
+ * 256-byte aligned.  Use pinned host memory for full copy bandwidth. */
+dn_status dn_energy_grad_host(const dn_problem* problem, const float* u_host, const float* gJ_host,
+                              float* J_host, float* r_host, void* staging, size_t staging_bytes,
+                              void* stream);
+
+/* Number of kernel launches the last-validated path of this problem enqueues per
+ * dn_energy_grad call (for launch accounting); 0 if the problem is invalid. */
+int32_t dn_launches_per_call(const dn_problem* problem);
+
+/* Name of the kernel family that dn_energy_grad would use ("tiled2d", "tiled3d", "generic"). */
+const char* dn_path_name(const dn_problem* problem);
+
+const char* dn_status_string(dn_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DN_H_ */

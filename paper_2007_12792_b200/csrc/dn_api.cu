@@ -1,0 +1,268 @@
+// C-ABI entry points: validation, workspace layout, choice of kernel family, launches.
+// Host code only; the arithmetic lives in the kernels of the other translation units.
+#include <cstdio>
+#include <cstring>
+
+#include "dn_internal.cuh"
+
+namespace dn {
+
+static bool valid_grid(const dn_grid& g, dn_status& st) {
+    if (g.dim != 2 && g.dim != 3) { st = DN_ERR_DIM; return false; }
+    const int nz = (g.dim == 3) ? g.nz : 2;
+    if (g.nx < 2 || g.ny < 2 || nz < 2 || g.nx > DN_MAX_EXTENT || g.ny > DN_MAX_EXTENT || nz > DN_MAX_EXTENT) {
+        st = DN_ERR_SIZE; return false;
+    }
+    return true;
+}
+
+static dn_status validate(const dn_problem* p) {
+    if (!p) return DN_ERR_NULL;
+    dn_status st = DN_OK;
+    if (!valid_grid(p->grid, st)) return st;
+    if (p->batch < 1 || p->batch > 65535) return DN_ERR_SIZE;
+    if (p->nu_mode == DN_NU_NODAL) {
+        if (!p->nu) return DN_ERR_NULL;
+    } else if (p->nu_mode == DN_NU_KL_GAUSS) {
+        if (p->kl_modes < 1 || p->kl_modes > DN_MAX_KL_MODES) return DN_ERR_MODE;
+        if (!p->kl_w) return DN_ERR_NULL;
+    } else {
+        return DN_ERR_MODE;
+    }
+    return DN_OK;
+}
+
+static long long nodes_per_sample(const dn_grid& g) {
+    return (long long)g.nx * g.ny * ((g.dim == 3) ? g.nz : 1);
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+Launch choose_launch(const dn_problem& p, const float* u, const float* r) {
+    const bool vec_ok = aligned16(u) && aligned16(r) && (p.nu_mode != DN_NU_NODAL || aligned16(p.nu));
+    if (!(p.flags & DN_FORCE_GENERIC) && vec_ok && p.f == nullptr) {
+        if (tiled2d_applicable(p)) return tiled2d_geometry(p);
+        if (tiled3d_applicable(p)) return tiled3d_geometry(p);
+    }
+    Launch l{};
+    l.path = PATH_GENERIC;
+    l.nblk = generic_blocks_per_sample(nodes_per_sample(p.grid));
+    return l;
+}
+
+// The workspace is sized for the largest of the kernel families that could be chosen for
+// this problem, so that the size does not depend on pointer alignment.
+static int max_nblk(const dn_problem& p) {
+    int n = generic_blocks_per_sample(nodes_per_sample(p.grid));
+    if (tiled2d_applicable(p)) { int t = tiled2d_geometry(p).nblk; if (t > n) n = t; }
+    if (tiled3d_applicable(p)) { int t = tiled3d_geometry(p).nblk; if (t > n) n = t; }
+    return n;
+}
+
+WsLayout make_layout(const dn_problem& p, const Launch& l) {
+    WsLayout w{};
+    const int dim = p.grid.dim;
+    const int m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
+    w.nblk = l.nblk;
+    size_t off = 0;
+    w.partials = off; off += align_up(sizeof(double) * 2 * (size_t)p.batch * max_nblk(p));
+    size_t mpow = 1;
+    for (int a = 0; a < dim; ++a) mpow *= (size_t)m;
+    w.ckl = off; off += align_up(sizeof(float) * (size_t)p.batch * (m ? mpow : 0) + 16);
+    const int n[3] = {p.grid.nx, p.grid.ny, (dim == 3) ? p.grid.nz : 1};
+    for (int a = 0; a < 3; ++a) {
+        const int ng = (a < dim) ? 2 * (n[a] - 1) : 0;
+        w.gstride[a] = (ng + 3) / 4 * 4 + 8;     // slack so that vector reads past the last point stay inside
+        w.cg[a] = off;
+        off += align_up(sizeof(float) * (size_t)m * w.gstride[a] + 16);
+    }
+    w.total = off;
+    return w;
+}
+
+static Params make_params(const dn_problem& p, const WsLayout& w, const float* u, const float* gJ, float* r, void* ws) {
+    Params P{};
+    P.dim = p.grid.dim; P.nx = p.grid.nx; P.ny = p.grid.ny; P.nz = (p.grid.dim == 3) ? p.grid.nz : 1;
+    P.batch = p.batch; P.nu_mode = p.nu_mode; P.m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
+    P.flags = p.flags; P.f_const = p.f_const; P.bc_x0 = p.bc_x0; P.bc_x1 = p.bc_x1;
+    P.hx = (float)(1.0 / (P.nx - 1)); P.hy = (float)(1.0 / (P.ny - 1));
+    P.hz = (P.dim == 3) ? (float)(1.0 / (P.nz - 1)) : 1.0f;
+    P.u = u; P.nu = p.nu; P.f = p.f; P.gJ = gJ; P.r = r;
+    char* base = static_cast<char*>(ws);
+    P.partials = reinterpret_cast<double*>(base + w.partials);
+    P.ckl = reinterpret_cast<const float*>(base + w.ckl);
+    for (int a = 0; a < 3; ++a) { P.cg[a] = reinterpret_cast<const float*>(base + w.cg[a]); P.gstride[a] = w.gstride[a]; }
+    P.nblk = w.nblk;
+    P.nodes = nodes_per_sample(p.grid);
+    return P;
+}
+
+static dn_status run(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
+                     size_t ws_bytes, void* stream) {
+    dn_status st = validate(p);
+    if (st != DN_OK) return st;
+    if (!u) return DN_ERR_NULL;
+    if (r) {
+        const size_t bytes = sizeof(float) * (size_t)p->batch * nodes_per_sample(p->grid);
+        const char* a = reinterpret_cast<const char*>(u);
+        const char* b = reinterpret_cast<const char*>(r);
+        if (a < b + bytes && b < a + bytes) return DN_ERR_ALIAS;
+    }
+    const Launch l = choose_launch(*p, u, r);
+    const WsLayout w = make_layout(*p, l);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign) != 0 || ws_bytes < w.total) return DN_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Params P = make_params(*p, w, u, gJ, r, ws);
+    cudaError_t e = cudaSuccess;
+    if (p->nu_mode == DN_NU_KL_GAUSS) {
+        char* base = static_cast<char*>(ws);
+        float* cg[3] = {reinterpret_cast<float*>(base + w.cg[0]), reinterpret_cast<float*>(base + w.cg[1]),
+                        reinterpret_cast<float*>(base + w.cg[2])};
+        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, s);
+        if (e != cudaSuccess) return DN_ERR_CUDA;
+    }
+    if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
+    else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
+    else e = launch_generic(P, s);
+    if (e != cudaSuccess) return DN_ERR_CUDA;
+    if (J) {
+        e = launch_finalize(P.partials, w.nblk, p->batch, J, s);
+        if (e != cudaSuccess) return DN_ERR_CUDA;
+    }
+    return DN_OK;
+}
+
+}  // namespace dn
+
+using namespace dn;
+
+extern "C" {
+
+size_t dn_workspace_bytes(const dn_problem* p) {
+    if (validate(p) != DN_OK) return 0;
+    Launch l{};
+    l.nblk = 1;
+    return make_layout(*p, l).total;
+}
+
+size_t dn_host_staging_bytes(const dn_problem* p) {
+    if (validate(p) != DN_OK) return 0;
+    const size_t field = align_up(sizeof(float) * (size_t)p->batch * nodes_per_sample(p->grid));
+    size_t total = 2 * field;                                   // u, r
+    total += 2 * align_up(sizeof(float) * (size_t)p->batch);    // J, gJ
+    if (p->nu_mode == DN_NU_NODAL) total += field;
+    if (p->f) total += field;
+    size_t mpow = 1;
+    for (int a = 0; a < p->grid.dim; ++a) mpow *= (size_t)((p->nu_mode == DN_NU_KL_GAUSS) ? p->kl_modes : 0);
+    total += align_up(sizeof(float) * (size_t)p->batch * mpow + 16);
+    return total + dn_workspace_bytes(p);
+}
+
+dn_status dn_energy(const dn_problem* p, const float* u, float* J, void* ws, size_t ws_bytes, void* stream) {
+    if (!J) return DN_ERR_NULL;
+    return run(p, u, nullptr, J, nullptr, ws, ws_bytes, stream);
+}
+
+dn_status dn_energy_grad(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
+                         size_t ws_bytes, void* stream) {
+    if (!r) return DN_ERR_NULL;
+    return run(p, u, gJ, J, r, ws, ws_bytes, stream);
+}
+
+dn_status dn_kl_field(const dn_grid* g, int32_t batch, int32_t m, const float* kl_w, float* nu, void* stream) {
+    if (!g || !kl_w || !nu) return DN_ERR_NULL;
+    dn_status st = DN_OK;
+    if (!valid_grid(*g, st)) return st;
+    if (batch < 1 || batch > 65535) return DN_ERR_SIZE;
+    if (m < 1 || m > DN_MAX_KL_MODES) return DN_ERR_MODE;
+    return launch_kl_field(*g, batch, m, kl_w, nu, static_cast<cudaStream_t>(stream)) == cudaSuccess ? DN_OK : DN_ERR_CUDA;
+}
+
+dn_status dn_apply_bc(const dn_grid* g, int32_t batch, float b0, float b1, int32_t mode, float* field, void* stream) {
+    if (!g || !field) return DN_ERR_NULL;
+    dn_status st = DN_OK;
+    if (!valid_grid(*g, st)) return st;
+    if (batch < 1 || batch > 65535) return DN_ERR_SIZE;
+    if (mode != 0 && mode != 1) return DN_ERR_MODE;
+    return launch_apply_bc(*g, batch, b0, b1, mode, field, static_cast<cudaStream_t>(stream)) == cudaSuccess ? DN_OK
+                                                                                                            : DN_ERR_CUDA;
+}
+
+dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const float* gJ_host, float* J_host,
+                              float* r_host, void* staging, size_t staging_bytes, void* stream) {
+    dn_status st = validate(p);
+    if (st != DN_OK) return st;
+    if (!u_host || !r_host) return DN_ERR_NULL;
+    if (!staging || (reinterpret_cast<uintptr_t>(staging) % kAlign) != 0 || staging_bytes < dn_host_staging_bytes(p))
+        return DN_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t nfield = (size_t)p->batch * nodes_per_sample(p->grid);
+    const size_t field = align_up(sizeof(float) * nfield);
+    const size_t small = align_up(sizeof(float) * (size_t)p->batch);
+    char* base = static_cast<char*>(staging);
+    size_t off = 0;
+    float* d_u = reinterpret_cast<float*>(base + off); off += field;
+    float* d_r = reinterpret_cast<float*>(base + off); off += field;
+    float* d_J = reinterpret_cast<float*>(base + off); off += small;
+    float* d_g = reinterpret_cast<float*>(base + off); off += small;
+    dn_problem q = *p;
+#define DN_TRY(x) do { if ((x) != cudaSuccess) return DN_ERR_CUDA; } while (0)
+    DN_TRY(cudaMemcpyAsync(d_u, u_host, sizeof(float) * nfield, cudaMemcpyHostToDevice, s));
+    if (p->nu_mode == DN_NU_NODAL) {
+        float* d = reinterpret_cast<float*>(base + off); off += field;
+        DN_TRY(cudaMemcpyAsync(d, p->nu, sizeof(float) * nfield, cudaMemcpyHostToDevice, s));
+        q.nu = d;
+    }
+    if (p->f) {
+        float* d = reinterpret_cast<float*>(base + off); off += field;
+        DN_TRY(cudaMemcpyAsync(d, p->f, sizeof(float) * nfield, cudaMemcpyHostToDevice, s));
+        q.f = d;
+    }
+    {
+        size_t mpow = 1;
+        for (int a = 0; a < p->grid.dim; ++a) mpow *= (size_t)((p->nu_mode == DN_NU_KL_GAUSS) ? p->kl_modes : 0);
+        float* d = reinterpret_cast<float*>(base + off); off += align_up(sizeof(float) * (size_t)p->batch * mpow + 16);
+        if (p->nu_mode == DN_NU_KL_GAUSS) {
+            DN_TRY(cudaMemcpyAsync(d, p->kl_w, sizeof(float) * (size_t)p->batch * mpow, cudaMemcpyHostToDevice, s));
+            q.kl_w = d;
+        }
+    }
+    if (gJ_host) DN_TRY(cudaMemcpyAsync(d_g, gJ_host, sizeof(float) * p->batch, cudaMemcpyHostToDevice, s));
+    st = run(&q, d_u, gJ_host ? d_g : nullptr, J_host ? d_J : nullptr, d_r, base + off, staging_bytes - off, s);
+    if (st != DN_OK) return st;
+    DN_TRY(cudaMemcpyAsync(r_host, d_r, sizeof(float) * nfield, cudaMemcpyDeviceToHost, s));
+    if (J_host) DN_TRY(cudaMemcpyAsync(J_host, d_J, sizeof(float) * p->batch, cudaMemcpyDeviceToHost, s));
+    DN_TRY(cudaStreamSynchronize(s));
+#undef DN_TRY
+    return DN_OK;
+}
+
+int32_t dn_launches_per_call(const dn_problem* p) {
+    if (validate(p) != DN_OK) return 0;
+    return 2 + (p->nu_mode == DN_NU_KL_GAUSS ? 1 : 0);
+}
+
+const char* dn_path_name(const dn_problem* p) {
+    if (validate(p) != DN_OK) return "invalid";
+    if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr) {
+        if (tiled2d_applicable(*p)) return "tiled2d";
+        if (tiled3d_applicable(*p)) return "tiled3d";
+    }
+    return "generic";
+}
+
+const char* dn_status_string(dn_status s) {
+    switch (s) {
+        case DN_OK: return "ok";
+        case DN_ERR_NULL: return "a required pointer is NULL";
+        case DN_ERR_DIM: return "dim must be 2 or 3";
+        case DN_ERR_SIZE: return "grid extent or batch out of range";
+        case DN_ERR_MODE: return "unknown mode or kl_modes out of range";
+        case DN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case DN_ERR_CUDA: return "CUDA runtime error";
+        case DN_ERR_ALIAS: return "r overlaps u";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,99 @@
+// Internal declarations shared by the CUDA translation units of libdn.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "dn.h"
+
+namespace dn {
+
+// Gauss abscissae of the 2-point rule mapped to [0,1]: (1 -/+ 1/sqrt(3)) / 2.
+#define DN_GA 0.21132486540518711775f
+#define DN_GB 0.78867513459481288225f
+
+constexpr int kAlign = 256;
+
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+enum Path { PATH_GENERIC = 0, PATH_TILED2D = 1, PATH_TILED3D = 2 };
+
+// Where things live inside the caller's workspace (byte offsets, all 256-B aligned).
+struct WsLayout {
+    size_t partials;      // double [B][nblk][2]  (diffusion part, load part)
+    size_t ckl;           // float  [B][m^dim]    KL weights * log2(e) / (1 + i^2 + j^2 (+ k^2))
+    size_t cg[3];         // float  [m][gstride[a]] cos(i pi x) at the Gauss abscissae of axis a
+    int gstride[3];       // padded row length of cg[a] (multiple of 4)
+    int nblk;             // energy partials per sample
+    size_t total;
+};
+
+// Everything a kernel needs, passed by value.
+struct Params {
+    int dim, nx, ny, nz, batch;
+    int nu_mode, m;
+    unsigned flags;
+    float f_const, bc_x0, bc_x1;
+    float hx, hy, hz;
+    const float* u;
+    const float* nu;
+    const float* f;
+    const float* gJ;
+    float* r;             // may be NULL (energy only)
+    double* partials;
+    const float* ckl;
+    const float* cg[3];
+    int gstride[3];
+    int nblk;
+    long long nodes;      // per sample
+};
+
+struct Launch {           // tiled-path launch geometry chosen on the host
+    int path;
+    int nblk;             // blocks (energy partials) per sample
+    int chunk;            // rows (2D) or planes (3D) of elements per block
+    int variant;          // kernel template variant
+};
+
+Launch choose_launch(const dn_problem& p, const float* u, const float* r);
+WsLayout make_layout(const dn_problem& p, const Launch& l);
+
+cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], cudaStream_t s);
+cudaError_t launch_generic(const Params& P, cudaStream_t s);
+cudaError_t launch_tiled2d(const Params& P, const Launch& l, cudaStream_t s);
+cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s);
+cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s);
+cudaError_t launch_kl_field(const dn_grid& g, int batch, int m, const float* kl_w, float* nu, cudaStream_t s);
+cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int mode, float* field, cudaStream_t s);
+
+int generic_blocks_per_sample(long long nodes);
+bool tiled2d_applicable(const dn_problem& p);
+bool tiled3d_applicable(const dn_problem& p);
+Launch tiled2d_geometry(const dn_problem& p);
+Launch tiled3d_geometry(const dn_problem& p);
+
+#ifdef __CUDACC__
+// Sum (d, l) over the block in a fixed order and let thread 0 store the pair.
+// Every thread of the block must call this.  blockDim.x * blockDim.y <= 1024.
+__device__ __forceinline__ void block_reduce_store(double d, double l, double* slot) {
+    __shared__ double sd[32], sl[32];
+    const int tid = threadIdx.y * blockDim.x + threadIdx.x;
+    const int nthreads = blockDim.x * blockDim.y;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        d += __shfl_down_sync(0xffffffffu, d, o);
+        l += __shfl_down_sync(0xffffffffu, l, o);
+    }
+    if ((tid & 31) == 0) { sd[tid >> 5] = d; sl[tid >> 5] = l; }
+    __syncthreads();
+    if (tid == 0) {
+        const int nw = (nthreads + 31) >> 5;
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < nw; ++w) { a += sd[w]; b += sl[w]; }
+        slot[0] = a; slot[1] = b;
+    }
+}
+#endif
+
+}  // namespace dn

@@ -1,0 +1,7 @@
+// Tiled 2D kernel (placeholder: not yet applicable to any problem).
+#include "dn_internal.cuh"
+namespace dn {
+bool tiled2d_applicable(const dn_problem&) { return false; }
+Launch tiled2d_geometry(const dn_problem&) { return Launch{}; }
+cudaError_t launch_tiled2d(const Params&, const Launch&, cudaStream_t) { return cudaErrorNotSupported; }
+}  // namespace dn

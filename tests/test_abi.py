@@ -1,0 +1,101 @@
+"""The C-ABI library loads, exports every symbol the header declares, and rejects bad
+arguments on the host (no kernel is launched, so this runs without a GPU)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2007_12792_b200 import build, binding
+    build.build()
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "dn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dn_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    from paper_2007_12792_b200 import binding
+    names = declared_symbols()
+    assert len(names) >= 9
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(binding.EXPORTS) == set(names)
+
+
+def test_status_strings(L):
+    from paper_2007_12792_b200 import binding
+    seen = {binding.status_string(s) for s in range(0, 8)}
+    assert len(seen) == 8 and binding.status_string(0) == "ok"
+
+
+def test_host_side_validation(L):
+    from paper_2007_12792_b200 import binding as B
+    fake = 0x1000  # never dereferenced: validation fails first
+
+    def prob(**kw):
+        p = B.DnProblem()
+        p.grid = B.DnGrid(kw.get("dim", 2), kw.get("nx", 8), kw.get("ny", 8), kw.get("nz", 1))
+        p.batch = kw.get("batch", 1)
+        p.nu_mode = kw.get("nu_mode", B.DN_NU_KL_GAUSS)
+        p.kl_modes = kw.get("kl_modes", 2)
+        p.kl_w = kw.get("kl_w", fake)
+        p.nu = kw.get("nu", None)
+        return p
+
+    def eg(p, u=fake, r=fake * 1024, ws=fake * 4096, ws_bytes=1 << 30):
+        return L.dn_energy_grad(C.byref(p), u, None, None, r, ws, ws_bytes, None)
+
+    assert L.dn_workspace_bytes(C.byref(prob())) > 0
+    assert L.dn_workspace_bytes(C.byref(prob())) % 256 == 0
+    assert L.dn_host_staging_bytes(C.byref(prob())) > L.dn_workspace_bytes(C.byref(prob()))
+    assert L.dn_workspace_bytes(None) == 0
+    assert L.dn_energy_grad(None, fake, None, None, fake, fake, 0, None) == B.DN_ERR_NULL
+    assert eg(prob(dim=4)) == B.DN_ERR_DIM
+    assert eg(prob(nx=1)) == B.DN_ERR_SIZE
+    assert eg(prob(dim=3, nz=1)) == B.DN_ERR_SIZE
+    assert eg(prob(batch=0)) == B.DN_ERR_SIZE
+    assert eg(prob(nx=40000)) == B.DN_ERR_SIZE
+    assert eg(prob(nu_mode=7)) == B.DN_ERR_MODE
+    assert eg(prob(kl_modes=0)) == B.DN_ERR_MODE
+    assert eg(prob(kl_modes=B.DN_MAX_KL_MODES + 1)) == B.DN_ERR_MODE
+    assert eg(prob(kl_w=None)) == B.DN_ERR_NULL
+    assert eg(prob(nu_mode=B.DN_NU_NODAL, nu=None)) == B.DN_ERR_NULL
+    assert eg(prob(), u=None) == B.DN_ERR_NULL
+    assert eg(prob(), r=None) == B.DN_ERR_NULL
+    assert eg(prob(), r=fake + 16) == B.DN_ERR_ALIAS
+    assert eg(prob(), ws=None) == B.DN_ERR_WORKSPACE
+    assert eg(prob(), ws=fake * 4096 + 8) == B.DN_ERR_WORKSPACE
+    assert eg(prob(), ws_bytes=16) == B.DN_ERR_WORKSPACE
+    assert L.dn_energy(C.byref(prob()), fake, None, fake * 4096, 1 << 30, None) == B.DN_ERR_NULL
+    g = B.DnGrid(2, 8, 8, 1)
+    assert L.dn_kl_field(C.byref(g), 1, 0, fake, fake, None) == B.DN_ERR_MODE
+    assert L.dn_kl_field(C.byref(g), 1, 2, None, fake, None) == B.DN_ERR_NULL
+    assert L.dn_kl_field(C.byref(B.DnGrid(5, 8, 8, 1)), 1, 2, fake, fake, None) == B.DN_ERR_DIM
+    assert L.dn_apply_bc(C.byref(g), 1, 1.0, 0.0, 3, fake, None) == B.DN_ERR_MODE
+    assert L.dn_apply_bc(C.byref(g), 0, 1.0, 0.0, 0, fake, None) == B.DN_ERR_SIZE
+    assert L.dn_apply_bc(C.byref(g), 1, 1.0, 0.0, 0, None, None) == B.DN_ERR_NULL
+    assert L.dn_energy_grad_host(C.byref(prob()), fake, None, None, fake, None, 0, None) == B.DN_ERR_WORKSPACE
+    assert L.dn_launches_per_call(C.byref(prob())) == 3
+    assert L.dn_launches_per_call(C.byref(prob(dim=9))) == 0
+    assert L.dn_path_name(C.byref(prob(nx=7))) == b"generic"
+
+
+def test_binding_rejects_host_tensors_and_missing_library(monkeypatch):
+    import torch
+    from paper_2007_12792_b200 import binding as B
+    p = B.Problem(dim=2, nx=8, ny=8, batch=1, kl_modes=2, kl_w=torch.zeros(1, 2, 2))
+    with pytest.raises(ValueError):
+        p.c_struct()                      # host tensor where a device tensor is required: no CPU path
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libdn.so")
+    with pytest.raises(RuntimeError):
+        B.lib()
