@@ -1,0 +1,286 @@
+#!/usr/bin/env python
+"""Benchmark of the fused FEM energy+residual path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--nu-mode kl|nodal]
+    python bench.py --impl reference ...      # the fp64 CPU oracle on the host cores
+
+One "step" is one pass of the whole hot path over one synthetic batch: a single
+``dn_energy_grad`` call (KL tables -> fused energy+residual kernel -> energy
+finaliser).  Prints ONE JSON line (rank 0).  With N > 1 ranks every rank
+processes its own batch of the same shape (samples are independent: weak
+scaling, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2007_12792_b200 import inputs  # noqa: E402
+
+METRIC = "fused FEM energy+residual Gelements/s"
+UNIT = "Gelements/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/; None where the kernel has changed since the capture.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.1] or [r for _, r in self.rows]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample_run(cfg: int, mode: str, target_seconds: float = 12.0):
+    """Times the oracle (as it stands) on a bounded sample of the workload: whole samples of the batch."""
+    import oracle
+    wl = inputs.WORKLOADS[cfg]
+    nu_mode = oracle.NU_KL_GAUSS if mode == "kl" else oracle.NU_NODAL
+
+    def run(samples):
+        inp = inputs.make_inputs(cfg, samples=samples)
+        nu = None
+        if nu_mode == oracle.NU_NODAL:
+            nu = oracle.kl_field(inp.dim, inp.nx, inp.ny, inp.nz, inp.batch, inp.kl_modes, inp.kl_w).astype(np.float32)
+        p = oracle.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=nu_mode, nu=nu,
+                           kl_modes=inp.kl_modes, kl_w=inp.kl_w, f_const=inp.f_const, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1)
+        t = time.perf_counter()
+        oracle.energy_grad(p, inp.u)
+        return time.perf_counter() - t
+
+    t1 = run([0])
+    n = int(max(1, min(wl.batch, round(target_seconds / max(t1, 1e-3)))))
+    t = run(list(range(n))) if n > 1 else t1
+    return {"value": wl.elements * n / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n} of {wl.batch} samples of {wl.name} ({wl.elements * n} elements, energy + full residual), "
+                      f"{t:.2f} s wall"}, t, n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = inputs.WORKLOADS[args.config]
+    times, base, n = [], None, 1
+    for it in range(args.warmup + args.steps):
+        base, t, n = oracle_sample_run(args.config, args.nu_mode, target_seconds=4.0)
+        if it >= args.warmup:
+            times.append(t)
+    ms = 1e3 * sum(times) / len(times)
+    value = wl.elements * n / (ms * 1e-3) / 1e9
+    base["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "nu_mode": args.nu_mode, "step": f"oracle pass over {n} sample(s)"},
+            "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (default: 2D 2048^2, batch 16)")
+    ap.add_argument("--nu-mode", default="kl", choices=["kl", "nodal"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2007_12792_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()
+
+    wl = inputs.WORKLOADS[args.config]
+    # every rank draws its own batch: sample indices rank*B .. rank*B + B-1 of the same recipe
+    inp = inputs.make_inputs(args.config, samples=range(rank * wl.batch, (rank + 1) * wl.batch))
+    u = torch.from_numpy(inp.u).cuda()
+    w = torch.from_numpy(inp.kl_w).cuda()
+    nu = None
+    mode = B.DN_NU_KL_GAUSS if args.nu_mode == "kl" else B.DN_NU_NODAL
+    if mode == B.DN_NU_NODAL:
+        nu = torch.empty_like(u)
+        B.dn_kl_field(inp.dim, inp.nx, inp.ny, inp.nz, inp.batch, inp.kl_modes, w, nu)
+    prob = B.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=mode, nu=nu,
+                     kl_modes=inp.kl_modes, kl_w=w, f_const=inp.f_const, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1)
+    r = torch.empty_like(u)
+    J = torch.empty(inp.batch, device="cuda")
+    ws = B.new_workspace(prob)
+    cs = prob.c_struct()
+    field_bytes = u.numel() * 4
+    l2_bytes = torch.cuda.get_device_properties(local).L2_cache_size
+    traffic_bytes = 2 * field_bytes + (field_bytes if nu is not None else 0)
+    flush = None
+    if traffic_bytes < 2 * l2_bytes:
+        flush = torch.empty(max(2 * l2_bytes, 256 << 20), dtype=torch.uint8, device="cuda")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K = args.steps
+    ev_step = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    ev_main = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b_ in ev_step + ev_main:            # create the underlying CUDA events
+        a.record(); b_.record()
+    for _ in range(args.warmup):
+        if flush is not None:
+            flush.zero_()
+        B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    t0 = time.time()
+    for k in range(K):
+        if flush is not None:
+            flush.zero_()                      # evict L2 between timed steps (outside the per-step events)
+        ev_step[k][0].record()
+        B.dn_energy_grad_traced(prob, u, None, J, r, ws, ev_main[k][0], ev_main[k][1], _cstruct=cs)
+        ev_step[k][1].record()
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    step_ms = sum(a.elapsed_time(b_) for a, b_ in ev_step) / K
+    main_ms = sum(a.elapsed_time(b_) for a, b_ in ev_main) / K
+    Jsum = float(J.double().sum())
+
+    # ---- end to end: host buffers in, host buffers out, through the C-ABI host entry point ----------
+    u_h = torch.from_numpy(inp.u).pin_memory()
+    w_h = torch.from_numpy(inp.kl_w).pin_memory()
+    nu_h = nu.cpu().pin_memory() if nu is not None else None
+    r_h = torch.empty(u.shape).pin_memory()
+    J_h = torch.empty(inp.batch).pin_memory()
+    prob_h = B.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=mode, nu=nu_h,
+                       kl_modes=inp.kl_modes, kl_w=w_h, f_const=inp.f_const, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1)
+    staging = B.new_host_staging(prob_h)
+    B.dn_energy_grad_host(prob_h, u_h, None, J_h, r_h, staging)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.e2e_steps):
+        B.dn_energy_grad_host(prob_h, u_h, None, J_h, r_h, staging)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+    h2d = field_bytes + w.numel() * 4 + (field_bytes if nu is not None else 0)
+    d2h = field_bytes + inp.batch * 4
+
+    t = torch.tensor([step_ms, main_ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    step_ms, main_ms, e2e_ms = (float(x) for x in t.cpu())
+
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        elements = wl.elements * inp.batch
+        nodes = wl.nodes * inp.batch
+        alg_bytes = nodes * (8 if mode == B.DN_NU_KL_GAUSS else 12)
+        achieved = alg_bytes / (main_ms * 1e-3) / 1e9
+        path = B.dn_path_name(prob)
+        key = f"{path}:{wl.name}:{args.nu_mode}"
+        line = {
+            "metric": METRIC, "value": world * elements / (step_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "nu_mode": args.nu_mode, "kernel_path": path,
+                       "elements_per_step_per_gpu": elements, "sharding": "independent batches per rank",
+                       "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps"},
+            "clocks": clocks,
+            "e2e": {"value": world * elements / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
+                    "entry": "dn_energy_grad_host (pinned host buffers)"},
+            "gpu_launches": K * B.dn_launches_per_call(prob),
+            "roofline": {"bound": "hbm", "kernel": f"fused energy+residual ({path})", "achieved": achieved,
+                         "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                         "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": main_ms,
+                         "traffic": NCU_TRAFFIC_BYTES.get(key)},
+            "checksum_J": Jsum,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = oracle_sample_run(args.config, args.nu_mode)[0]
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

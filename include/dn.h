@@ -115,6 +115,15 @@ dn_status dn_energy(const dn_problem* problem, const float* u, float* J, void* w
 dn_status dn_energy_grad(const dn_problem* problem, const float* u, const float* gJ, float* J, float* r,
                          void* workspace, size_t workspace_bytes, void* stream);
 
+/* dn_energy_grad that also records two caller-owned CUDA events (cudaEvent_t passed as void*)
+ * on `stream`: event_before just before the fused energy+residual kernel is enqueued and
+ * event_after just after it, so that a caller can time that kernel alone while the table and
+ * finaliser kernels of the same call are excluded.  Either event may be NULL.  A measurement
+ * aid (Algorithm 1 has no counterpart); results are identical to dn_energy_grad. */
+dn_status dn_energy_grad_traced(const dn_problem* problem, const float* u, const float* gJ, float* J, float* r,
+                                void* workspace, size_t workspace_bytes, void* stream,
+                                void* event_before, void* event_after);
+
 /* Boundary operator B(u) = b (Eq. (pde)): overwrites the two Dirichlet faces of a field in
  * place.  mode 0: field = bc_x0 at ix = 0 and bc_x1 at ix = nx-1;  mode 1: both faces = 0
  * (e.g. to mask a gradient). */

@@ -28,7 +28,7 @@ DN_FORCE_GENERIC = 4
 DN_MAX_KL_MODES = 8
 
 EXPORTS = ("dn_workspace_bytes", "dn_host_staging_bytes", "dn_kl_field", "dn_energy", "dn_energy_grad",
-           "dn_apply_bc", "dn_energy_grad_host", "dn_launches_per_call", "dn_path_name", "dn_status_string")
+           "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced", "dn_launches_per_call", "dn_path_name", "dn_status_string")
 
 
 class DnGrid(C.Structure):
@@ -67,12 +67,14 @@ def lib():
         L.dn_kl_field.argtypes = [PG, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.dn_energy.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.dn_energy_grad.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.dn_energy_grad_traced.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                            C.c_void_p, C.c_void_p, C.c_void_p]
         L.dn_apply_bc.argtypes = [PG, C.c_int32, C.c_float, C.c_float, C.c_int32, C.c_void_p, C.c_void_p]
         L.dn_energy_grad_host.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.dn_launches_per_call.argtypes = [PP]; L.dn_launches_per_call.restype = C.c_int32
         L.dn_path_name.argtypes = [PP]; L.dn_path_name.restype = C.c_char_p
         L.dn_status_string.argtypes = [C.c_int]; L.dn_status_string.restype = C.c_char_p
-        for f in ("dn_kl_field", "dn_energy", "dn_energy_grad", "dn_apply_bc", "dn_energy_grad_host"):
+        for f in ("dn_kl_field", "dn_energy", "dn_energy_grad", "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced"):
             getattr(L, f).restype = C.c_int
         _lib = L
     return _lib
@@ -188,6 +190,20 @@ def dn_energy_grad(problem: Problem, u: torch.Tensor, gJ: Optional[torch.Tensor]
     p = problem.c_struct()
     _check(lib().dn_energy_grad(C.byref(p), _ptr(u, "u"), _ptr(gJ, "gJ"), _ptr(J, "J"), _ptr(r, "r"),
                                 workspace.data_ptr(), workspace.numel(), _stream(stream)), "dn_energy_grad")
+    return J, r
+
+
+def dn_energy_grad_traced(problem: Problem, u: torch.Tensor, gJ: Optional[torch.Tensor], J: Optional[torch.Tensor],
+                          r: torch.Tensor, workspace: torch.Tensor, event_before: Optional[torch.cuda.Event],
+                          event_after: Optional[torch.cuda.Event], stream=None, _cstruct=None):
+    """dn_energy_grad that records the two (already created, timing-enabled) torch CUDA events around
+    the fused kernel.  ``_cstruct`` lets a tight loop reuse a marshalled ``dn_problem``."""
+    p = _cstruct if _cstruct is not None else problem.c_struct()
+    eb = None if event_before is None else event_before.cuda_event
+    ea = None if event_after is None else event_after.cuda_event
+    _check(lib().dn_energy_grad_traced(C.byref(p), _ptr(u, "u"), _ptr(gJ, "gJ"), _ptr(J, "J"), _ptr(r, "r"),
+                                       workspace.data_ptr(), workspace.numel(), _stream(stream), eb, ea),
+           "dn_energy_grad_traced")
     return J, r
 
 

@@ -98,7 +98,7 @@ static Params make_params(const dn_problem& p, const WsLayout& w, const float* u
 }
 
 static dn_status run(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
-                     size_t ws_bytes, void* stream) {
+                     size_t ws_bytes, void* stream, void* ev_before = nullptr, void* ev_after = nullptr) {
     dn_status st = validate(p);
     if (st != DN_OK) return st;
     if (!u) return DN_ERR_NULL;
@@ -121,10 +121,12 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
         e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, s);
         if (e != cudaSuccess) return DN_ERR_CUDA;
     }
+    if (ev_before && cudaEventRecord(static_cast<cudaEvent_t>(ev_before), s) != cudaSuccess) return DN_ERR_CUDA;
     if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
     else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
     else e = launch_generic(P, s);
     if (e != cudaSuccess) return DN_ERR_CUDA;
+    if (ev_after && cudaEventRecord(static_cast<cudaEvent_t>(ev_after), s) != cudaSuccess) return DN_ERR_CUDA;
     if (J) {
         e = launch_finalize(P.partials, w.nblk, p->batch, J, s);
         if (e != cudaSuccess) return DN_ERR_CUDA;
@@ -167,6 +169,12 @@ dn_status dn_energy_grad(const dn_problem* p, const float* u, const float* gJ, f
                          size_t ws_bytes, void* stream) {
     if (!r) return DN_ERR_NULL;
     return run(p, u, gJ, J, r, ws, ws_bytes, stream);
+}
+
+dn_status dn_energy_grad_traced(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
+                                size_t ws_bytes, void* stream, void* ev_before, void* ev_after) {
+    if (!r) return DN_ERR_NULL;
+    return run(p, u, gJ, J, r, ws, ws_bytes, stream, ev_before, ev_after);
 }
 
 dn_status dn_kl_field(const dn_grid* g, int32_t batch, int32_t m, const float* kl_w, float* nu, void* stream) {

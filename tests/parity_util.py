@@ -43,4 +43,4 @@ def check(Jg, rg, Jo, ro, what=""):
     err = np.abs(rg - ro).max()
     assert np.isfinite(rg).all(), f"{what}: non-finite residual"
     assert err <= R_RTOL * scale, f"{what}: r max err {err:.3e} vs scale {scale:.3e} ({err / scale:.3e})"
-    return (0.0 if Jg is None else float((np.abs(Jg - Jo) / np.abs(Jo)).max())), float(err / scale)
+    return (0.0 if Jg is None else float((np.abs(Jg - Jo) / np.abs(Jo)).max())), float(err / max(scale, 1e-300))
