@@ -65,6 +65,7 @@ typedef enum {
 
 #define DN_MAX_KL_MODES 8        /* largest m (KL modes per axis)                                         */
 #define DN_MAX_EXTENT 32768      /* largest nx, ny or nz                                                  */
+#define DN_STATIC_SCRATCH_BYTES (1u << 20)  /* scratch built into the library for dn_energy_grad_static   */
 
 typedef struct {
     int32_t dim;                 /* 2 or 3                                 */
@@ -123,6 +124,25 @@ dn_status dn_energy_grad(const dn_problem* problem, const float* u, const float*
 dn_status dn_energy_grad_traced(const dn_problem* problem, const float* u, const float* gJ, float* J, float* r,
                                 void* workspace, size_t workspace_bytes, void* stream,
                                 void* event_before, void* event_after);
+
+/* dn_energy_grad without a workspace argument, for callers that are not allowed to allocate
+ * device memory: code running inside another framework's memory plan, under a fixed memory
+ * budget, or at a point where cudaMalloc would stall the device.  (The paper has no counterpart;
+ * this is a calling convenience.)  The scratch that dn_energy_grad takes from the caller is here a
+ * fixed array of DN_STATIC_SCRATCH_BYTES (1 MiB) inside the library image; every GPU that loads the
+ * library holds it until the process exits.  The call itself allocates and frees nothing.
+ *  - Inputs, outputs and results are exactly those of dn_energy_grad.
+ *  - A problem that needs more scratch than the array holds (large grids on the any-size kernels,
+ *    very large batches) is refused with DN_ERR_WORKSPACE and nothing is enqueued; use
+ *    dn_energy_grad with your own workspace for those.
+ *  - The first call on each device looks up the array's device address (one runtime query, with
+ *    that device current); make that first call before starting any stream capture.
+ *  - All calls on a device share the one array and it keeps whatever the previous call left in it.
+ *    Nothing in it needs to start at zero (every entry is written before it is read), but two calls
+ *    that may run on the GPU at the same time (different streams) race on it: serialise them, or
+ *    use dn_energy_grad with separate workspaces. */
+dn_status dn_energy_grad_static(const dn_problem* problem, const float* u, const float* gJ, float* J, float* r,
+                                void* stream);
 
 /* Boundary operator B(u) = b (Eq. (pde)): overwrites the two Dirichlet faces of a field in
  * place.  mode 0: field = bc_x0 at ix = 0 and bc_x1 at ix = nx-1;  mode 1: both faces = 0

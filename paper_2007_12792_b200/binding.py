@@ -28,7 +28,7 @@ DN_FORCE_GENERIC = 4
 DN_MAX_KL_MODES = 8
 
 EXPORTS = ("dn_workspace_bytes", "dn_host_staging_bytes", "dn_kl_field", "dn_energy", "dn_energy_grad",
-           "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced", "dn_launches_per_call", "dn_path_name", "dn_status_string")
+           "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced", "dn_energy_grad_static", "dn_launches_per_call", "dn_path_name", "dn_status_string")
 
 
 class DnGrid(C.Structure):
@@ -69,6 +69,8 @@ def lib():
         L.dn_energy_grad.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.dn_energy_grad_traced.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                             C.c_void_p, C.c_void_p, C.c_void_p]
+        L.dn_energy_grad_static.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.dn_energy_grad_static.restype = C.c_int
         L.dn_apply_bc.argtypes = [PG, C.c_int32, C.c_float, C.c_float, C.c_int32, C.c_void_p, C.c_void_p]
         L.dn_energy_grad_host.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.dn_launches_per_call.argtypes = [PP]; L.dn_launches_per_call.restype = C.c_int32
@@ -204,6 +206,18 @@ def dn_energy_grad_traced(problem: Problem, u: torch.Tensor, gJ: Optional[torch.
     _check(lib().dn_energy_grad_traced(C.byref(p), _ptr(u, "u"), _ptr(gJ, "gJ"), _ptr(J, "J"), _ptr(r, "r"),
                                        workspace.data_ptr(), workspace.numel(), _stream(stream), eb, ea),
            "dn_energy_grad_traced")
+    return J, r
+
+
+def dn_energy_grad_static(problem: Problem, u: torch.Tensor, gJ: Optional[torch.Tensor], J: Optional[torch.Tensor],
+                          r: torch.Tensor, stream=None):
+    """dn_energy_grad for callers that may not allocate device memory (for instance code that runs under
+    another framework's fixed memory plan): no workspace is passed, the library's built-in 1 MiB scratch
+    array is used, and nothing is allocated here or in the library.  Problems that need more scratch raise
+    DnError(DN_ERR_WORKSPACE).  Calls on one device share that array, so do not overlap them on the GPU."""
+    p = problem.c_struct()
+    _check(lib().dn_energy_grad_static(C.byref(p), _ptr(u, "u"), _ptr(gJ, "gJ"), _ptr(J, "J"), _ptr(r, "r"),
+                                       _stream(stream)), "dn_energy_grad_static")
     return J, r
 
 

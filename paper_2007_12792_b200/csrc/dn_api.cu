@@ -59,13 +59,13 @@ static int max_nblk(const dn_problem& p) {
     return n;
 }
 
-WsLayout make_layout(const dn_problem& p, const Launch& l) {
+WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
     WsLayout w{};
     const int dim = p.grid.dim;
     const int m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
     w.nblk = l.nblk;
     size_t off = 0;
-    w.partials = off; off += align_up(sizeof(double) * 2 * (size_t)p.batch * max_nblk(p));
+    w.partials = off; off += align_up(sizeof(double) * 2 * (size_t)p.batch * (tight ? l.nblk : max_nblk(p)));
     size_t mpow = 1;
     for (int a = 0; a < dim; ++a) mpow *= (size_t)m;
     w.ckl = off; off += align_up(sizeof(float) * (size_t)p.batch * (m ? mpow : 0) + 16);
@@ -98,7 +98,8 @@ static Params make_params(const dn_problem& p, const WsLayout& w, const float* u
 }
 
 static dn_status run(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
-                     size_t ws_bytes, void* stream, void* ev_before = nullptr, void* ev_after = nullptr) {
+                     size_t ws_bytes, void* stream, void* ev_before = nullptr, void* ev_after = nullptr,
+                     bool tight = false) {
     dn_status st = validate(p);
     if (st != DN_OK) return st;
     if (!u) return DN_ERR_NULL;
@@ -109,7 +110,7 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
         if (a < b + bytes && b < a + bytes) return DN_ERR_ALIAS;
     }
     const Launch l = choose_launch(*p, u, r);
-    const WsLayout w = make_layout(*p, l);
+    const WsLayout w = make_layout(*p, l, tight);
     if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign) != 0 || ws_bytes < w.total) return DN_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Params P = make_params(*p, w, u, gJ, r, ws);
@@ -132,6 +133,12 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
         if (e != cudaSuccess) return DN_ERR_CUDA;
     }
     return DN_OK;
+}
+
+dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
+                    size_t ws_bytes, void* stream) {
+    if (!r) return DN_ERR_NULL;
+    return run(p, u, gJ, J, r, ws, ws_bytes, stream, nullptr, nullptr, true);
 }
 
 }  // namespace dn

@@ -57,7 +57,10 @@ struct Launch {           // tiled-path launch geometry chosen on the host
 };
 
 Launch choose_launch(const dn_problem& p, const float* u, const float* r);
-WsLayout make_layout(const dn_problem& p, const Launch& l);
+WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight = false);
+// dn_energy_grad with the workspace sized for the chosen kernel family only (tight = true).
+dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
+                    size_t ws_bytes, void* stream);
 
 cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], cudaStream_t s);
 cudaError_t launch_generic(const Params& P, cudaStream_t s);
