@@ -39,86 +39,33 @@ __device__ __forceinline__ float ex2_approx3(float x) {
     return y;
 }
 
-template <int M> struct Gs3 { static constexpr int value = ((M + 1) + 3) / 4 * 4; };
+typedef unsigned long long u64;
 
-template <int M>
-__device__ __forceinline__ float horner3(const float* g, float c) {
-    float e = g[M];
-#pragma unroll
-    for (int k = M - 1; k >= 0; --k) e = fmaf(e, c, g[k]);
-    return e;
+__device__ __forceinline__ u64 pack2_3(float lo, float hi) {
+    u64 v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void unpack2_3(u64 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 fma2_3(u64 a, u64 b, u64 c) {
+    u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
 }
 
-struct Contrib { float r000, r100, r010, r110, r001, r101, r011, r111; };
+// Register state of one staged node plane, for the 4 node columns of a thread.
+struct PlaneState { float u[4], h, e[4], s[4], txy[4]; };   // h: node right of the strip (lane 31)
 
-// One element.  nu[p][q][s]: p, q, s index the Gauss point along x, y, z.
-__device__ __forceinline__ void element3(float e0, float s0, float w0, float txy, float txz, float tyz, float txyz,
-                                         const float (&nu)[2][2][2], bool iso, float kx, float ky, float kz,
-                                         Contrib& o, float& en) {
-    const float a = DN_GA, b = DN_GB;
-    // d/dx (times hx) at (q, s)
-    const float Axa = fmaf(a, txy, e0), Axb = fmaf(b, txy, e0);
-    const float Bxa = fmaf(a, txyz, txz), Bxb = fmaf(b, txyz, txz);
-    const float Dx_aa = fmaf(a, Bxa, Axa), Dx_ab = fmaf(b, Bxa, Axa), Dx_ba = fmaf(a, Bxb, Axb), Dx_bb = fmaf(b, Bxb, Axb);
-    // d/dy (times hy) at (p, s)
-    const float Aya = fmaf(a, txy, s0), Ayb = fmaf(b, txy, s0);
-    const float Bya = fmaf(a, txyz, tyz), Byb = fmaf(b, txyz, tyz);
-    const float Dy_aa = fmaf(a, Bya, Aya), Dy_ab = fmaf(b, Bya, Aya), Dy_ba = fmaf(a, Byb, Ayb), Dy_bb = fmaf(b, Byb, Ayb);
-    // d/dz (times hz) at (p, q): (w + p txz) + q (tyz + p txyz)
-    const float Aza = fmaf(a, txz, w0), Azb = fmaf(b, txz, w0);
-    const float Dz_aa = fmaf(a, Bya, Aza), Dz_ab = fmaf(b, Bya, Aza), Dz_ba = fmaf(a, Byb, Azb), Dz_bb = fmaf(b, Byb, Azb);
-    // nu summed along the derivative's own axis
-    float Nx_aa = nu[0][0][0] + nu[1][0][0], Nx_ab = nu[0][0][1] + nu[1][0][1];     // (q, s)
-    float Nx_ba = nu[0][1][0] + nu[1][1][0], Nx_bb = nu[0][1][1] + nu[1][1][1];
-    float Ny_aa = nu[0][0][0] + nu[0][1][0], Ny_ab = nu[0][0][1] + nu[0][1][1];     // (p, s)
-    float Ny_ba = nu[1][0][0] + nu[1][1][0], Ny_bb = nu[1][0][1] + nu[1][1][1];
-    float Nz_aa = nu[0][0][0] + nu[0][0][1], Nz_ab = nu[0][1][0] + nu[0][1][1];     // (p, q)
-    float Nz_ba = nu[1][0][0] + nu[1][0][1], Nz_bb = nu[1][1][0] + nu[1][1][1];
-    if (!iso) {
-        Nx_aa *= kx; Nx_ab *= kx; Nx_ba *= kx; Nx_bb *= kx;
-        Ny_aa *= ky; Ny_ab *= ky; Ny_ba *= ky; Ny_bb *= ky;
-        Nz_aa *= kz; Nz_ab *= kz; Nz_ba *= kz; Nz_bb *= kz;
-    }
-    const float Gx_aa = Nx_aa * Dx_aa, Gx_ab = Nx_ab * Dx_ab, Gx_ba = Nx_ba * Dx_ba, Gx_bb = Nx_bb * Dx_bb;
-    const float Gy_aa = Ny_aa * Dy_aa, Gy_ab = Ny_ab * Dy_ab, Gy_ba = Ny_ba * Dy_ba, Gy_bb = Ny_bb * Dy_bb;
-    const float Gz_aa = Nz_aa * Dz_aa, Gz_ab = Nz_ab * Dz_ab, Gz_ba = Nz_ba * Dz_ba, Gz_bb = Nz_bb * Dz_bb;
-    float acc = Gx_aa * Dx_aa;
-    acc = fmaf(Gx_ab, Dx_ab, acc); acc = fmaf(Gx_ba, Dx_ba, acc); acc = fmaf(Gx_bb, Dx_bb, acc);
-    acc = fmaf(Gy_aa, Dy_aa, acc); acc = fmaf(Gy_ab, Dy_ab, acc); acc = fmaf(Gy_ba, Dy_ba, acc); acc = fmaf(Gy_bb, Dy_bb, acc);
-    acc = fmaf(Gz_aa, Dz_aa, acc); acc = fmaf(Gz_ab, Dz_ab, acc); acc = fmaf(Gz_ba, Dz_ba, acc); acc = fmaf(Gz_bb, Dz_bb, acc);
-    en += acc;
-    // adjoint of the three interpolations
-    const float AXa = Gx_aa + Gx_ab, AXb = Gx_ba + Gx_bb;
-    const float BXa = fmaf(b, Gx_ab, a * Gx_aa), BXb = fmaf(b, Gx_bb, a * Gx_ba);
-    const float AYa = Gy_aa + Gy_ab, AYb = Gy_ba + Gy_bb;
-    const float BYa = fmaf(b, Gy_ab, a * Gy_aa), BYb = fmaf(b, Gy_bb, a * Gy_ba);
-    const float AZa = Gz_aa + Gz_ab, AZb = Gz_ba + Gz_bb;
-    const float BZa = fmaf(b, Gz_ab, a * Gz_aa), BZb = fmaf(b, Gz_bb, a * Gz_ba);
-    const float dE = AXa + AXb, dS = AYa + AYb, dW = AZa + AZb;
-    float dXY = fmaf(b, AXb, a * AXa);
-    dXY = fmaf(a, AYa, dXY); dXY = fmaf(b, AYb, dXY);
-    float dXZ = BXa + BXb;
-    dXZ = fmaf(a, AZa, dXZ); dXZ = fmaf(b, AZb, dXZ);
-    float dYZ = (BYa + BYb) + (BZa + BZb);
-    float dXYZ = fmaf(b, BXb, a * BXa);
-    dXYZ = fmaf(a, BYa, dXYZ); dXYZ = fmaf(b, BYb, dXYZ);
-    dXYZ = fmaf(a, BZa, dXYZ); dXYZ = fmaf(b, BZb, dXYZ);
-    // chain rule to the corners
-    o.r111 = dXYZ;
-    o.r110 = dXY - dXYZ;
-    o.r101 = dXZ - dXYZ;
-    o.r011 = dYZ - dXYZ;
-    o.r100 = (dE - o.r110) - dXZ;
-    o.r010 = (dS - o.r110) - dYZ;
-    o.r001 = (dW - o.r101) - dYZ;
-    o.r000 = ((o.r011 - dW) + (dXY - dE)) + (dXZ - dS);
-}
+// Floats per Gauss row pair (q fixed, s = a and b interleaved) in the coefficient table.
+template <int M> struct Gs3p { static constexpr int value = (2 * (M + 1) + 3) / 4 * 4; };
 
-template <int M, bool WANT_R>
+template <int M, bool WANT_R, bool FULL>
 __global__ void __launch_bounds__(T3_THREADS, 1)
 tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const int ntile_y) {
     extern __shared__ __align__(16) float smem[];
-    constexpr int GS = Gs3<M>::value;
+    constexpr int GS = Gs3p<M>::value;                  // floats per (row q) line pair
     const int lane = threadIdx.x & 31;
     const int wid = threadIdx.x >> 5;
     const int wx = wid % WX, ty = wid / WX;
@@ -131,18 +78,19 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     const int x0 = wx * 128 + 4 * lane;
     const int p0 = zc * Z, p1 = min(p0 + Z, nz);
     const int kbeg = max(p0 - 1, 0), kend = min(p1 - 1, nz - 2);
-    const bool col_ok = x0 < nx;
+    const bool col_ok = FULL || (x0 < nx);
     const bool elem_row_ok = (y < ny - 1);
-    const bool node_row_ok = (y < ny);
-    const bool out_row = node_row_ok && (ty >= 1 || tile == 0);
+    const bool out_row = (y < ny) && (ty >= 1 || tile == 0);
     const bool top_row = (ty == TY - 1);
 
     // shared memory: two exchange buffers, then the KL coefficients of every Gauss line of the block
-    const int XOFF = 4 * TY * NXP;                     // floats before the cross-warp slots
+    const int TYNXP = TY * NXP;
+    const int XOFF = 4 * TYNXP;                        // floats before the cross-warp slots
     const int BUF = XOFF + TY * WX * 4;
     float* gam = smem + 2 * BUF;
 
-    // ---- prologue: KL polynomial coefficients for the Gauss lines (row q, plane s) of the block
+    // ---- prologue: KL polynomial coefficients; table index ((k - kbeg) * TY + row) * 2 + q, entries
+    // interleave the two Gauss planes s = a, b of the element plane: [coef][s]
     {
         const int nlines = (kend - kbeg + 1) * TY * 4;
         const float* c = P.ckl + (size_t)b * M * M * M;
@@ -177,8 +125,9 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
 #pragma unroll
                 for (int k = 0; k <= M; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
             }
+            float* dst = gam + (size_t)(t >> 1) * GS + s;
 #pragma unroll
-            for (int k = 0; k < GS; ++k) gam[(size_t)t * GS + k] = (k <= M) ? (float)acc[k <= M ? k : 0] : 0.f;
+            for (int k = 0; k <= M; ++k) dst[2 * k] = (float)acc[k];
         }
     }
 
@@ -188,63 +137,57 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     const float kap = iso ? kx : 1.f;                  // isotropic cells: one scale applied at the end
     const bool nomask = (P.flags & DN_NO_MASK) != 0;
     const bool impose = (P.flags & DN_IMPOSE_BC_ON_LOAD) != 0;
+    const float bc0 = P.bc_x0, bc1 = P.bc_x1;
     const float gs = (WANT_R && P.gJ) ? __ldg(P.gJ + b) : 1.f;
     const float fw = P.f_const * P.hx * P.hy * P.hz;  // nodal load of an interior node
+    const bool hasf = (P.f_const != 0.f);
     const float wy = (y == 0 || y == ny - 1) ? 0.5f : 1.f;
     const bool first_col = (x0 == 0), last_col = (x0 + 3 == nx - 1);
     const bool last_elem_missing = (x0 + 3 >= nx - 1);  // element right of node x0+3 does not exist
+    const bool halo_ok = (lane == 31) && (x0 + 4 < nx);
+    const float mfirst = first_col ? 0.f : 1.f, mlast = last_col ? 0.f : 1.f;
 
     const int yl = min(y, ny - 1);                     // rows beyond the grid load a valid address; unused
     const int ya = min(y + 1, ny - 1);
-    const float* ub = P.u + (size_t)b * P.nodes;
-    float* rb = WANT_R ? P.r + (size_t)b * P.nodes : nullptr;
     const size_t plane = (size_t)nx * ny;
+    const float* pu = P.u + (size_t)b * P.nodes + (size_t)yl * nx + x0;      // own row, plane 0
+    const float* pa = P.u + (size_t)b * P.nodes + (size_t)ya * nx + x0;      // row above (top warp row only)
+    float* pr = WANT_R ? P.r + (size_t)b * P.nodes + (size_t)yl * nx + x0 : nullptr;
 
-    float cpa[4], cpb[4];
-    if (col_ok) {
-        const float4 q0 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0));
-        const float4 q1 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0 + 4));
-        cpa[0] = q0.x; cpb[0] = q0.y; cpa[1] = q0.z; cpb[1] = q0.w;
-        cpa[2] = q1.x; cpb[2] = q1.y; cpa[3] = q1.z; cpb[3] = q1.w;
-    } else {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) { cpa[c] = 0.f; cpb[c] = 0.f; }
+    u64 cda[4], cdb[4];                                // cos(pi x) at the two Gauss columns, duplicated
+    {
+        float4 q0 = make_float4(0.f, 0.f, 0.f, 0.f), q1 = q0;
+        if (col_ok) {
+            q0 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0));
+            q1 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0 + 4));
+        }
+        cda[0] = pack2_3(q0.x, q0.x); cdb[0] = pack2_3(q0.y, q0.y); cda[1] = pack2_3(q0.z, q0.z); cdb[1] = pack2_3(q0.w, q0.w);
+        cda[2] = pack2_3(q1.x, q1.x); cdb[2] = pack2_3(q1.y, q1.y); cda[3] = pack2_3(q1.z, q1.z); cdb[3] = pack2_3(q1.w, q1.w);
     }
 
-    // ---- register state: plane kp = the last staged plane
-    float uk[4], ek[4], sk[4], txyk[4];
+    PlaneState S0, S1;
     float L0p[4], U0p[4], carry[4], L1p[4], U1p[4], Xp[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-        uk[c] = ek[c] = sk[c] = txyk[c] = 0.f;
+        S0.u[c] = S0.e[c] = S0.s[c] = S0.txy[c] = 0.f;
+        S1.u[c] = S1.e[c] = S1.s[c] = S1.txy[c] = 0.f;
+        S0.h = S1.h = 0.f;
         L0p[c] = U0p[c] = carry[c] = L1p[c] = U1p[c] = Xp[c] = 0.f;
     }
     float en = 0.f, enl = 0.f, ell = 0.f;
 
-    auto load_own = [&](int p, float (&v)[4], float& halo) {
+    auto load4 = [&](const float* ptr, float (&v)[4], float& halo) {
         if (col_ok) {
-            const float4 q = __ldg(reinterpret_cast<const float4*>(ub + (size_t)p * plane + (size_t)yl * nx + x0));
+            const float4 q = __ldg(reinterpret_cast<const float4*>(ptr));
             v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
         } else {
             v[0] = v[1] = v[2] = v[3] = 0.f;
         }
-        halo = (lane == 31 && x0 + 4 < nx) ? __ldg(ub + (size_t)p * plane + (size_t)yl * nx + x0 + 4) : 0.f;
+        halo = 0.f;
+        if (halo_ok) halo = __ldg(ptr + 4);
         if (impose) {
-            if (first_col) v[0] = P.bc_x0;
-            if (last_col) v[3] = P.bc_x1;
-        }
-    };
-    auto load_above = [&](int p, float (&v)[4], float& halo) {   // row y+1, top warp row of the tile only
-        if (col_ok) {
-            const float4 q = __ldg(reinterpret_cast<const float4*>(ub + (size_t)p * plane + (size_t)ya * nx + x0));
-            v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
-        } else {
-            v[0] = v[1] = v[2] = v[3] = 0.f;
-        }
-        halo = (lane == 31 && x0 + 4 < nx) ? __ldg(ub + (size_t)p * plane + (size_t)ya * nx + x0 + 4) : 0.f;
-        if (impose) {
-            if (first_col) v[0] = P.bc_x0;
-            if (last_col) v[3] = P.bc_x1;
+            if (first_col) v[0] = bc0;
+            if (last_col) v[3] = bc1;
         }
     };
     auto xdiffs = [&](const float (&v)[4], float halo, float (&e)[4]) {
@@ -253,43 +196,38 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
         e[0] = v[1] - v[0]; e[1] = v[2] - v[1]; e[2] = v[3] - v[2]; e[3] = rn - v[3];
     };
 
-    float un[4], unh, ua[4], uah;
-    load_own(kbeg, un, unh);
-    if (top_row) load_above(kbeg, ua, uah);
+    float ua[4], uah = 0.f;                            // prefetched row above (top warp row of the tile only)
+    ua[0] = ua[1] = ua[2] = ua[3] = 0.f;
+    if (kbeg & 1) load4(pu + (size_t)kbeg * plane, S1.u, S1.h); else load4(pu + (size_t)kbeg * plane, S0.u, S0.h);
+    if (top_row) load4(pa + (size_t)kbeg * plane, ua, uah);
 
-    // iteration p stages node plane p, computes element plane p-1, finishes node plane p-2
-    for (int p = kbeg; p <= kend + 2; ++p) {
-        const int par = p & 1;
-        float* sb = smem + par * BUF;
-        float* su = sb + (0 * TY + ty) * NXP + x0;
-        float* se = sb + (1 * TY + ty) * NXP + x0;
-        float* sL = sb + (2 * TY + ty) * NXP + x0;
-        float* sU = sb + (3 * TY + ty) * NXP + x0;
-        float* sX = sb + XOFF + (ty * WX + wx) * 4;
+    // Iteration p stages node plane p into `up`, computes element plane p-1 between `lo` and `up`,
+    // and finishes node plane p-2.  PAR = p & 1 selects the exchange buffer.
+    auto step = [&](PlaneState& lo, PlaneState& up, const int p, const int PAR) {
+        float* sb = smem + PAR * BUF + ty * NXP + x0;
+        float* sX = smem + PAR * BUF + XOFF + (ty * WX + wx) * 4;
         const bool stage = (p <= kend + 1);
-        float ep[4], vn[4], vnh, va[4], vah;
-        if (stage) {
-            xdiffs(un, unh, ep);
+        float w0[4];
+        if (stage) {                                   // up.u / up.h were prefetched by the previous step
+            xdiffs(up.u, up.h, up.e);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) w0[c] = up.u[c] - lo.u[c];
             if (col_ok) {
-                *reinterpret_cast<float4*>(su) = make_float4(un[0], un[1], un[2], un[3]);
-                *reinterpret_cast<float4*>(se) = make_float4(ep[0], ep[1], ep[2], ep[3]);
+                *reinterpret_cast<float4*>(sb) = make_float4(up.u[0], up.u[1], up.u[2], up.u[3]);
+                *reinterpret_cast<float4*>(sb + TYNXP) = make_float4(up.e[0], up.e[1], up.e[2], up.e[3]);
             }
-            if (p + 1 <= kend + 1) {                   // prefetch the next plane
-                load_own(p + 1, vn, vnh);
-                if (top_row) load_above(p + 1, va, vah);
-            }
-            // load energy of the staged plane (owned planes and rows only)
-            if (p >= p0 && p < p1 && out_row) {
-                float rs = (un[0] + un[1]) + (un[2] + un[3]);
-                if (first_col) rs -= 0.5f * un[0];
-                if (last_col) rs -= 0.5f * un[3];
+            if (p <= kend) load4(pu + (size_t)(p + 1) * plane, lo.u, lo.h);   // prefetch the next plane (lo.u is dead)
+            if (hasf && p >= p0 && p < p1 && out_row) { // load energy of the staged plane
+                float rs = (up.u[0] + up.u[1]) + (up.u[2] + up.u[3]);
+                if (first_col) rs -= 0.5f * up.u[0];
+                if (last_col) rs -= 0.5f * up.u[3];
                 const float wz = (p == 0 || p == nz - 1) ? 0.5f : 1.f;
                 ell = fmaf(fw * wy * wz, rs, ell);
             }
         }
         if (WANT_R && col_ok) {                        // contributions of the previous element step to row y+1
-            *reinterpret_cast<float4*>(sL) = make_float4(L1p[0], L1p[1], L1p[2], L1p[3]);
-            *reinterpret_cast<float4*>(sU) = make_float4(U1p[0], U1p[1], U1p[2], U1p[3]);
+            *reinterpret_cast<float4*>(sb + 2 * TYNXP) = make_float4(L1p[0], L1p[1], L1p[2], L1p[3]);
+            *reinterpret_cast<float4*>(sb + 3 * TYNXP) = make_float4(U1p[0], U1p[1], U1p[2], U1p[3]);
             if (lane == 31) *reinterpret_cast<float4*>(sX) = make_float4(Xp[0], Xp[1], Xp[2], Xp[3]);
         }
         __syncthreads();
@@ -298,8 +236,8 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
         if (WANT_R && p - 2 >= kbeg) {
             float l1[4] = {0.f, 0.f, 0.f, 0.f}, u1[4] = {0.f, 0.f, 0.f, 0.f};
             if (ty > 0 && col_ok) {
-                const float4 a = *reinterpret_cast<const float4*>(sL - NXP);
-                const float4 c4 = *reinterpret_cast<const float4*>(sU - NXP);
+                const float4 a = *reinterpret_cast<const float4*>(sb + 2 * TYNXP - NXP);
+                const float4 c4 = *reinterpret_cast<const float4*>(sb + 3 * TYNXP - NXP);
                 l1[0] = a.x; l1[1] = a.y; l1[2] = a.z; l1[3] = a.w;
                 u1[0] = c4.x; u1[1] = c4.y; u1[2] = c4.z; u1[3] = c4.w;
             }
@@ -312,7 +250,6 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 }
             }
             const int pl = p - 2;                      // the plane being finished
-            const bool own_plane = (pl >= p0);
             const float wz = (pl == 0 || pl == nz - 1) ? 0.5f : 1.f;
             const float lw = fw * wy * wz;
             const float sc = gs * kap, nl = -gs * lw;
@@ -322,118 +259,151 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 const float raw = (L0p[c] + l1[c]) + carry[c];
                 carry[c] = U0p[c] + u1[c];
                 o[c] = fmaf(sc, raw, nl);
-                if (c == 0 && first_col) o[c] = nomask ? fmaf(sc, raw, 0.5f * nl) : 0.f;
-                if (c == 3 && last_col) o[c] = nomask ? fmaf(sc, raw, 0.5f * nl) : 0.f;
             }
-            if (own_plane && out_row && col_ok && pl <= kend)
-                *reinterpret_cast<float4*>(rb + (size_t)pl * plane + (size_t)y * nx + x0) = make_float4(o[0], o[1], o[2], o[3]);
+            if (!nomask) {
+                o[0] *= mfirst; o[3] *= mlast;
+            } else {
+                if (first_col) o[0] -= 0.5f * nl;      // Dirichlet columns carry half the nodal load
+                if (last_col) o[3] -= 0.5f * nl;
+            }
+            if (pl >= p0 && out_row && col_ok)
+                *reinterpret_cast<float4*>(pr + (size_t)pl * plane) = make_float4(o[0], o[1], o[2], o[3]);
         }
 
         // ---- finish staging plane p (needs row y+1) and compute element plane p-1
         if (stage) {
             float uab[4], eab[4];
             if (!top_row) {
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), c4 = a;
                 if (col_ok) {
-                    const float4 a = *reinterpret_cast<const float4*>(su + NXP);
-                    const float4 c4 = *reinterpret_cast<const float4*>(se + NXP);
-                    uab[0] = a.x; uab[1] = a.y; uab[2] = a.z; uab[3] = a.w;
-                    eab[0] = c4.x; eab[1] = c4.y; eab[2] = c4.z; eab[3] = c4.w;
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) { uab[c] = 0.f; eab[c] = 0.f; }
+                    a = *reinterpret_cast<const float4*>(sb + NXP);
+                    c4 = *reinterpret_cast<const float4*>(sb + TYNXP + NXP);
                 }
+                uab[0] = a.x; uab[1] = a.y; uab[2] = a.z; uab[3] = a.w;
+                eab[0] = c4.x; eab[1] = c4.y; eab[2] = c4.z; eab[3] = c4.w;
             } else {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) uab[c] = ua[c];
                 xdiffs(ua, uah, eab);
+                if (p <= kend) load4(pa + (size_t)(p + 1) * plane, ua, uah);
             }
-            float sp[4], txyp[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) { sp[c] = uab[c] - un[c]; txyp[c] = eab[c] - ep[c]; }
+            for (int c = 0; c < 4; ++c) { up.s[c] = uab[c] - up.u[c]; up.txy[c] = eab[c] - up.e[c]; }
 
             if (p > kbeg) {
                 const int k = p - 1;
-                const bool own_step = (k >= p0);      // the warm-up step only seeds the carried contributions
-                Contrib prev;
-                float l1n[4], u1n[4];
-                prev.r100 = prev.r110 = prev.r101 = prev.r111 = 0.f;
-                const float* gl = gam + ((size_t)((k - kbeg) * TY + ty) * 4) * GS;
-                float g_aa[GS], g_ab[GS], g_ba[GS], g_bb[GS];      // (q, s) lines
+                const bool own_energy = (k >= p0) && (ty >= 1 || tile == 0);
+                float L0[5], L1[5], U0[5], U1[5];
 #pragma unroll
-                for (int i = 0; i < GS / 4; ++i) {
-                    const float4 t0 = reinterpret_cast<const float4*>(gl)[i];
-                    const float4 t1 = reinterpret_cast<const float4*>(gl + GS)[i];
-                    const float4 t2 = reinterpret_cast<const float4*>(gl + 2 * GS)[i];
-                    const float4 t3 = reinterpret_cast<const float4*>(gl + 3 * GS)[i];
-                    g_aa[4 * i] = t0.x; g_aa[4 * i + 1] = t0.y; g_aa[4 * i + 2] = t0.z; g_aa[4 * i + 3] = t0.w;
-                    g_ab[4 * i] = t1.x; g_ab[4 * i + 1] = t1.y; g_ab[4 * i + 2] = t1.z; g_ab[4 * i + 3] = t1.w;
-                    g_ba[4 * i] = t2.x; g_ba[4 * i + 1] = t2.y; g_ba[4 * i + 2] = t2.z; g_ba[4 * i + 3] = t2.w;
-                    g_bb[4 * i] = t3.x; g_bb[4 * i + 1] = t3.y; g_bb[4 * i + 2] = t3.z; g_bb[4 * i + 3] = t3.w;
-                }
+                for (int c = 0; c < 5; ++c) { L0[c] = 0.f; L1[c] = 0.f; U0[c] = 0.f; U1[c] = 0.f; }
                 float enrow = 0.f, enlast = 0.f;
                 if (elem_row_ok) {
+                    const ulonglong2* gl = reinterpret_cast<const ulonglong2*>(gam + (size_t)(((k - kbeg) * TY + ty) * 2) * GS);
+                    u64 gq_a[GS / 2], gq_b[GS / 2];       // Gauss row q = a / b; each entry holds (plane s = a, s = b)
+#pragma unroll
+                    for (int i = 0; i < GS / 4; ++i) {
+                        const ulonglong2 t0 = gl[i], t1 = gl[GS / 4 + i];
+                        gq_a[2 * i] = t0.x; gq_a[2 * i + 1] = t0.y; gq_b[2 * i] = t1.x; gq_b[2 * i + 1] = t1.y;
+                    }
+                    const float a = DN_GA, bq = DN_GB;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        float nu[2][2][2];
-                        nu[0][0][0] = ex2_approx3(horner3<M>(g_aa, cpa[c])); nu[1][0][0] = ex2_approx3(horner3<M>(g_aa, cpb[c]));
-                        nu[0][0][1] = ex2_approx3(horner3<M>(g_ab, cpa[c])); nu[1][0][1] = ex2_approx3(horner3<M>(g_ab, cpb[c]));
-                        nu[0][1][0] = ex2_approx3(horner3<M>(g_ba, cpa[c])); nu[1][1][0] = ex2_approx3(horner3<M>(g_ba, cpb[c]));
-                        nu[0][1][1] = ex2_approx3(horner3<M>(g_bb, cpa[c])); nu[1][1][1] = ex2_approx3(horner3<M>(g_bb, cpb[c]));
-                        Contrib o;
-                        float e1 = 0.f;
-                        element3(ek[c], sk[c], un[c] - uk[c], txyk[c], ep[c] - ek[c], sp[c] - sk[c], txyp[c] - txyk[c],
-                                 nu, iso, kx, ky, kz, o, e1);
+                        // nu[p][q][s] at the 8 Gauss points: 4 packed Horner chains (column p, row q) x (s = a, b)
+                        u64 h_aa = gq_a[M], h_ab = gq_b[M], h_ba = gq_a[M], h_bb = gq_b[M];   // h_{p q}
+#pragma unroll
+                        for (int i = M - 1; i >= 0; --i) {
+                            h_aa = fma2_3(h_aa, cda[c], gq_a[i]); h_ab = fma2_3(h_ab, cda[c], gq_b[i]);
+                            h_ba = fma2_3(h_ba, cdb[c], gq_a[i]); h_bb = fma2_3(h_bb, cdb[c], gq_b[i]);
+                        }
+                        float n000, n001, n010, n011, n100, n101, n110, n111;               // n p q s
+                        unpack2_3(h_aa, n000, n001); unpack2_3(h_ab, n010, n011);
+                        unpack2_3(h_ba, n100, n101); unpack2_3(h_bb, n110, n111);
+                        n000 = ex2_approx3(n000); n001 = ex2_approx3(n001); n010 = ex2_approx3(n010); n011 = ex2_approx3(n011);
+                        n100 = ex2_approx3(n100); n101 = ex2_approx3(n101); n110 = ex2_approx3(n110); n111 = ex2_approx3(n111);
+                        float Nx_aa = n000 + n100, Nx_ab = n001 + n101, Nx_ba = n010 + n110, Nx_bb = n011 + n111;   // (q, s)
+                        float Ny_aa = n000 + n010, Ny_ab = n001 + n011, Ny_ba = n100 + n110, Ny_bb = n101 + n111;   // (p, s)
+                        float Nz_aa = n000 + n001, Nz_ab = n010 + n011, Nz_ba = n100 + n101, Nz_bb = n110 + n111;   // (p, q)
+                        if (!iso) {
+                            Nx_aa *= kx; Nx_ab *= kx; Nx_ba *= kx; Nx_bb *= kx;
+                            Ny_aa *= ky; Ny_ab *= ky; Ny_ba *= ky; Ny_bb *= ky;
+                            Nz_aa *= kz; Nz_ab *= kz; Nz_ba *= kz; Nz_bb *= kz;
+                        }
+                        // hierarchical coordinates of the element
+                        const float e0 = lo.e[c], s0 = lo.s[c];
+                        const float txy = lo.txy[c], txz = up.e[c] - e0, tyz = up.s[c] - s0, txyz = up.txy[c] - txy;
+                        const float Axa = fmaf(a, txy, e0), Axb = fmaf(bq, txy, e0);
+                        const float Bxa = fmaf(a, txyz, txz), Bxb = fmaf(bq, txyz, txz);
+                        const float Dx_aa = fmaf(a, Bxa, Axa), Dx_ab = fmaf(bq, Bxa, Axa), Dx_ba = fmaf(a, Bxb, Axb), Dx_bb = fmaf(bq, Bxb, Axb);
+                        const float Aya = fmaf(a, txy, s0), Ayb = fmaf(bq, txy, s0);
+                        const float Bya = fmaf(a, txyz, tyz), Byb = fmaf(bq, txyz, tyz);
+                        const float Dy_aa = fmaf(a, Bya, Aya), Dy_ab = fmaf(bq, Bya, Aya), Dy_ba = fmaf(a, Byb, Ayb), Dy_bb = fmaf(bq, Byb, Ayb);
+                        const float Aza = fmaf(a, txz, w0[c]), Azb = fmaf(bq, txz, w0[c]);
+                        const float Dz_aa = fmaf(a, Bya, Aza), Dz_ab = fmaf(bq, Bya, Aza), Dz_ba = fmaf(a, Byb, Azb), Dz_bb = fmaf(bq, Byb, Azb);
+                        const float Gx_aa = Nx_aa * Dx_aa, Gx_ab = Nx_ab * Dx_ab, Gx_ba = Nx_ba * Dx_ba, Gx_bb = Nx_bb * Dx_bb;
+                        const float Gy_aa = Ny_aa * Dy_aa, Gy_ab = Ny_ab * Dy_ab, Gy_ba = Ny_ba * Dy_ba, Gy_bb = Ny_bb * Dy_bb;
+                        const float Gz_aa = Nz_aa * Dz_aa, Gz_ab = Nz_ab * Dz_ab, Gz_ba = Nz_ba * Dz_ba, Gz_bb = Nz_bb * Dz_bb;
+                        // adjoint of the three interpolations
+                        const float AXa = Gx_aa + Gx_ab, AXb = Gx_ba + Gx_bb;
+                        const float BXa = fmaf(bq, Gx_ab, a * Gx_aa), BXb = fmaf(bq, Gx_bb, a * Gx_ba);
+                        const float AYa = Gy_aa + Gy_ab, AYb = Gy_ba + Gy_bb;
+                        const float BYa = fmaf(bq, Gy_ab, a * Gy_aa), BYb = fmaf(bq, Gy_bb, a * Gy_ba);
+                        const float AZa = Gz_aa + Gz_ab, AZb = Gz_ba + Gz_bb;
+                        const float BZa = fmaf(bq, Gz_ab, a * Gz_aa), BZb = fmaf(bq, Gz_bb, a * Gz_ba);
+                        float dE = AXa + AXb, dS = AYa + AYb, dW = AZa + AZb;
+                        float dXY = fmaf(bq, AXb, a * AXa);
+                        dXY = fmaf(a, AYa, dXY); dXY = fmaf(bq, AYb, dXY);
+                        float dXZ = BXa + BXb;
+                        dXZ = fmaf(a, AZa, dXZ); dXZ = fmaf(bq, AZb, dXZ);
+                        float dYZ = (BYa + BYb) + (BZa + BZb);
+                        float dXYZ = fmaf(bq, BXb, a * BXa);
+                        dXYZ = fmaf(a, BYa, dXYZ); dXYZ = fmaf(bq, BYb, dXYZ);
+                        dXYZ = fmaf(a, BZa, dXYZ); dXYZ = fmaf(bq, BZb, dXYZ);
+                        // the element energy is a quadratic form of its 7 coordinates: Euler's identity
+                        float e1 = dE * e0;
+                        e1 = fmaf(dS, s0, e1); e1 = fmaf(dW, w0[c], e1); e1 = fmaf(dXY, txy, e1);
+                        e1 = fmaf(dXZ, txz, e1); e1 = fmaf(dYZ, tyz, e1); e1 = fmaf(dXYZ, txyz, e1);
                         if (c == 3) enlast = e1; else enrow += e1;
                         if (WANT_R) {
-                            if (c == 3 && last_elem_missing) {
-                                o.r000 = o.r100 = o.r010 = o.r110 = o.r001 = o.r101 = o.r011 = o.r111 = 0.f;
-                            }
-                            if (c > 0) {
-                                L0p[c] = o.r000 + prev.r100; l1n[c] = o.r010 + prev.r110;
-                                U0p[c] = o.r001 + prev.r101; u1n[c] = o.r011 + prev.r111;
-                            } else {
-                                L0p[0] = o.r000; l1n[0] = o.r010; U0p[0] = o.r001; u1n[0] = o.r011;
-                            }
-                            prev = o;
+                            if (c == 3 && nomask && last_elem_missing) { dE = dS = dW = dXY = dXZ = dYZ = dXYZ = 0.f; }
+                            // chain rule to the corners
+                            const float r110 = dXY - dXYZ, r101 = dXZ - dXYZ, r011 = dYZ - dXYZ;
+                            const float r100 = (dE - r110) - dXZ, r010 = (dS - r110) - dYZ, r001 = (dW - r101) - dYZ;
+                            const float r000 = ((r011 - dW) + (dXY - dE)) + (dXZ - dS);
+                            if (c == 0) { L0[0] = r000; L1[0] = r010; U0[0] = r001; U1[0] = r011; }
+                            else { L0[c] += r000; L1[c] += r010; U0[c] += r001; U1[c] += r011; }
+                            L0[c + 1] = r100; L1[c + 1] = r110; U0[c + 1] = r101; U1[c + 1] = dXYZ;
                         }
                     }
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) { L0p[c] = 0.f; l1n[c] = 0.f; U0p[c] = 0.f; u1n[c] = 0.f; }
                 }
                 if (WANT_R) {
                     // the left neighbour's last element feeds this thread's first node column
-                    const float a100 = __shfl_up_sync(0xffffffffu, prev.r100, 1), a110 = __shfl_up_sync(0xffffffffu, prev.r110, 1);
-                    const float a101 = __shfl_up_sync(0xffffffffu, prev.r101, 1), a111 = __shfl_up_sync(0xffffffffu, prev.r111, 1);
-                    if (lane > 0) { L0p[0] += a100; l1n[0] += a110; U0p[0] += a101; u1n[0] += a111; }
-                    Xp[0] = prev.r100; Xp[1] = prev.r110; Xp[2] = prev.r101; Xp[3] = prev.r111;
+                    const float a100 = __shfl_up_sync(0xffffffffu, L0[4], 1), a110 = __shfl_up_sync(0xffffffffu, L1[4], 1);
+                    const float a101 = __shfl_up_sync(0xffffffffu, U0[4], 1), a111 = __shfl_up_sync(0xffffffffu, U1[4], 1);
+                    if (lane > 0) { L0[0] += a100; L1[0] += a110; U0[0] += a101; U1[0] += a111; }
+                    Xp[0] = L0[4]; Xp[1] = L1[4]; Xp[2] = U0[4]; Xp[3] = U1[4];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) { L1p[c] = l1n[c]; U1p[c] = u1n[c]; }
+                    for (int c = 0; c < 4; ++c) { L0p[c] = L0[c]; U0p[c] = U0[c]; L1p[c] = L1[c]; U1p[c] = U1[c]; }
                 }
-                if (own_step && elem_row_ok) {
-                    // energy of element row y belongs to the tile that computes it as a non-halo row
-                    if (ty >= 1 || tile == 0) {
-                        en += enrow;
-                        if (!last_elem_missing) enl += enlast;
-                    }
-                }
-            }
-            // the staged plane becomes the state
-#pragma unroll
-            for (int c = 0; c < 4; ++c) { uk[c] = un[c]; ek[c] = ep[c]; sk[c] = sp[c]; txyk[c] = txyp[c]; }
-            if (p + 1 <= kend + 1) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) un[c] = vn[c];
-                unh = vnh;
-                if (top_row) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) ua[c] = va[c];
-                    uah = vah;
+                if (own_energy && elem_row_ok) {
+                    en += enrow;
+                    if (!last_elem_missing) enl += enlast;
                 }
             }
         } else if (WANT_R) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) { L0p[c] = 0.f; U0p[c] = 0.f; L1p[c] = 0.f; U1p[c] = 0.f; Xp[c] = 0.f; }
+        }
+    };
+
+    // ---- march; even planes are staged into S0, odd planes into S1
+    {
+        int p = kbeg;
+        if (p & 1) { step(S0, S1, p, 1); ++p; }
+        while (p <= kend + 2) {
+            step(S1, S0, p, 0);
+            if (++p > kend + 2) break;
+            step(S0, S1, p, 1);
+            ++p;
         }
     }
 
@@ -443,12 +413,10 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
         const float sc = gs * kap, nl = -gs * lw;
         float o[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            o[c] = fmaf(sc, carry[c], nl);
-            if (c == 0 && first_col) o[c] = nomask ? fmaf(sc, carry[c], 0.5f * nl) : 0.f;
-            if (c == 3 && last_col) o[c] = nomask ? fmaf(sc, carry[c], 0.5f * nl) : 0.f;
-        }
-        *reinterpret_cast<float4*>(rb + (size_t)(nz - 1) * plane + (size_t)y * nx + x0) = make_float4(o[0], o[1], o[2], o[3]);
+        for (int c = 0; c < 4; ++c) o[c] = fmaf(sc, carry[c], nl);
+        if (!nomask) { o[0] *= mfirst; o[3] *= mlast; }
+        else { if (first_col) o[0] -= 0.5f * nl; if (last_col) o[3] -= 0.5f * nl; }
+        *reinterpret_cast<float4*>(pr + (size_t)(nz - 1) * plane) = make_float4(o[0], o[1], o[2], o[3]);
     }
     const double etot = 0.5 * (double)kap * ((double)en + (double)enl);
     block_reduce_store(etot, (double)ell, P.partials + 2 * ((size_t)b * P.nblk + blockIdx.x));
@@ -473,14 +441,14 @@ Geo3 geometry3(const dn_problem& p) {
     if (g.TY > ny) g.TY = (ny < 2) ? 2 : ny;
     g.ntile_y = (ny - 1 + (g.TY - 1) - 1) / (g.TY - 1);
     const int m = p.kl_modes;
-    g.GS = ((m + 1) + 3) / 4 * 4;
+    g.GS = (2 * (m + 1) + 3) / 4 * 4;               // floats per Gauss-row line pair
     const long long slots = sm_count3();
     const size_t fixed = sizeof(float) * 2 * ((size_t)4 * g.TY * g.WX * 128 + (size_t)g.TY * g.WX * 4);
     long long best = -1;
     int bestZ = 8;
     for (int Z = 4; Z <= 256; ++Z) {
         if (Z > nz && Z > 4) break;
-        const size_t sm = fixed + sizeof(float) * (size_t)(Z + 1) * g.TY * 4 * g.GS;
+        const size_t sm = fixed + sizeof(float) * (size_t)(Z + 1) * g.TY * 2 * g.GS;
         if (sm > 200 * 1024) break;
         const long long nch = (nz + Z - 1) / Z;
         const long long blocks = (long long)p.batch * g.ntile_y * nch;
@@ -490,25 +458,30 @@ Geo3 geometry3(const dn_problem& p) {
     }
     g.Z = bestZ;
     g.nchunk_z = (nz + g.Z - 1) / g.Z;
-    g.smem = fixed + sizeof(float) * (size_t)(g.Z + 1) * g.TY * 4 * g.GS;
+    g.smem = fixed + sizeof(float) * (size_t)(g.Z + 1) * g.TY * 2 * g.GS;
     return g;
 }
 
-template <int M>
-cudaError_t launch_m(const Params& P, const Geo3& g, cudaStream_t s) {
+template <int M, bool FULL>
+cudaError_t launch_mf(const Params& P, const Geo3& g, cudaStream_t s) {
     dim3 grid((unsigned)(g.ntile_y * g.nchunk_z), (unsigned)P.batch);
     const int threads = 32 * g.WX * g.TY;
     cudaError_t e;
     if (P.r) {
-        e = cudaFuncSetAttribute(tiled3d_kernel<M, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+        e = cudaFuncSetAttribute(tiled3d_kernel<M, true, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
         if (e != cudaSuccess) return e;
-        tiled3d_kernel<M, true><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y);
+        tiled3d_kernel<M, true, FULL><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y);
     } else {
-        e = cudaFuncSetAttribute(tiled3d_kernel<M, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+        e = cudaFuncSetAttribute(tiled3d_kernel<M, false, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
         if (e != cudaSuccess) return e;
-        tiled3d_kernel<M, false><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y);
+        tiled3d_kernel<M, false, FULL><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y);
     }
     return cudaGetLastError();
+}
+
+template <int M>
+cudaError_t launch_m(const Params& P, const Geo3& g, cudaStream_t s) {
+    return (g.WX * 128 == P.nx) ? launch_mf<M, true>(P, g, s) : launch_mf<M, false>(P, g, s);
 }
 
 }  // namespace
