@@ -4,9 +4,13 @@
 // warp 32*NE consecutive nodes, W warps side by side cover the row (nx <= 32*NE*W); WY such warp
 // rows share a block.  Each warp row marches over a chunk of node rows in y.  Per element row the
 // node row below lives in registers (values, horizontal differences, pending contributions); the
-// row above is loaded once with 128-bit loads, prefetched one row ahead; three row buffers rotate
-// by name (the row loop is unrolled three times), so nothing is copied.  The x+1 neighbour comes
-// from the next lane by shuffle, across warps from global memory (one scalar per row).  Every
+// row above arrives in one of two ways.  KL mode (issue-bound): 128-bit loads one row ahead into
+// registers.  Nodal mode (two input fields, latency-bound): the rows stream through a ring in
+// shared memory; every lane copies its own 16-byte pieces asynchronously (cp.async, 4 rows in
+// flight) and reads back only what it copied, so the ring needs no barrier.  Either way each row is
+// read from HBM once, and the register row buffers rotate by name (the row loop is unrolled three
+// times), so nothing is copied.  The x+1 neighbour comes from the next lane by shuffle, across
+// warps from global memory (one scalar per row).  Every
 // element is computed exactly once per block: its contributions to its two left nodes stay in the
 // thread, those to its right nodes go to the owner of the next element (shuffle; shared memory
 // between warps, one named barrier per row), those to the upper row are carried to the next step.
@@ -48,6 +52,21 @@ __device__ __forceinline__ void named_barrier(int id, int nthreads) {
 
 typedef unsigned long long u64;
 
+// Asynchronous global -> shared copies (each thread later reads back only what it copied itself,
+// so completion of its own copy groups is all the synchronisation the ring needs).
+__device__ __forceinline__ void cp_async16(float* smem_dst, const float* gsrc) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async4(float* smem_dst, const float* gsrc) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+constexpr int T2_STAGES = 4;                            // rows in flight per warp row (ring in shared memory)
+
 __device__ __forceinline__ u64 pack2(float lo, float hi) {
     u64 v;
     asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
@@ -67,7 +86,7 @@ template <int M> struct GamStride { static constexpr int value = (2 * (M + 1) + 
 
 template <int NE> struct Row { float v[NE]; float halo; };
 
-template <int K, int M, bool WANT_R, bool FULL>
+template <int K, int M, bool WANT_R, bool FULL, bool RING>
 __global__ void __launch_bounds__(256, 2)
 tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
     extern __shared__ __align__(16) float smem[];
@@ -89,6 +108,11 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
     const int gam_rows = R + 1;
     float* gam = smem + (size_t)wy * gam_rows * GS;
     float* xch = smem + (size_t)WY * gam_rows * (KL ? GS : 0) + (size_t)wy * 2 * T2_MAX_WARPS * 2;
+    // ring of T2_STAGES node rows per warp row (u, and nu in nodal mode): per lane NE floats, then one halo per warp
+    constexpr int NARR = KL ? 1 : 2;
+    const int ring_row = 32 * W * NE + 4 * ((W + 3) / 4);                      // floats per (stage, array)
+    float* ring = smem + (size_t)WY * gam_rows * (KL ? GS : 0) + (size_t)WY * 2 * T2_MAX_WARPS * 2 +
+                  (size_t)wy * T2_STAGES * NARR * ring_row;
 
     // ---- prologue: polynomial coefficients of the KL exponent for the Gauss rows of the chunk
     if constexpr (KL) if (!idle) {
@@ -157,6 +181,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
 #pragma unroll
         for (int k = 0; k < NE; ++k) em[k] = (x0 + k < nx - 1) ? 1.f : 0.f;
 
+        // direct variant: one row ahead in registers
         auto load_row = [&](Row<NE>& r, const float* __restrict__ base, int row) {
             const float* p = base + (size_t)row * nx + x0;
 #pragma unroll
@@ -170,6 +195,34 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             }
             r.halo = 0.f;
             if (lane == 31 && warp_has_halo) r.halo = __ldg(p + NE);
+        };
+        // ring variant: issue the copies of node row `row` into its ring slot (one commit group per row, possibly empty)
+        auto issue_row = [&](int row) {
+            if (row <= jend + 1) {
+                float* dst = ring + (size_t)(row & (T2_STAGES - 1)) * NARR * ring_row;
+#pragma unroll
+                for (int a = 0; a < NARR; ++a) {
+                    const float* p = ((a == 0) ? ub : nub) + (size_t)row * nx + x0;
+                    float* d = dst + a * ring_row;
+#pragma unroll
+                    for (int s = 0; s < K; ++s)
+                        if (act[s]) cp_async16(d + (wx * 32 + lane) * NE + 4 * s, p + 4 * s);
+                    if (lane == 31 && warp_has_halo) cp_async4(d + 32 * W * NE + wx, p + NE);
+                }
+            }
+            cp_async_commit();
+        };
+        // read this lane's part of a landed row back into registers
+        auto read_row = [&](Row<NE>& r, int row, int a) {
+            const float* d = ring + ((size_t)(row & (T2_STAGES - 1)) * NARR + a) * ring_row;
+#pragma unroll
+            for (int s = 0; s < K; ++s) {
+                float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (act[s]) q = *reinterpret_cast<const float4*>(d + (wx * 32 + lane) * NE + 4 * s);
+                r.v[4 * s] = q.x; r.v[4 * s + 1] = q.y; r.v[4 * s + 2] = q.z; r.v[4 * s + 3] = q.w;
+            }
+            r.halo = 0.f;
+            if (lane == 31 && warp_has_halo) r.halo = d[32 * W * NE + wx];
         };
         auto fix_bc = [&](Row<NE>& r) {
             if (impose) {
@@ -205,7 +258,14 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
         // ---- state of the node row below the current element row
         float ehor[NE], U[NE], hnu[NE], nlr = 0.f;
         Row<NE> A, B, C, nA, nB, nC;
-        load_row(A, ub, jbeg);
+        if constexpr (RING) {
+#pragma unroll
+            for (int d = 0; d < T2_STAGES; ++d) issue_row(jbeg + d);
+            cp_async_wait<T2_STAGES - 1>();             // row jbeg has landed
+            read_row(A, jbeg, 0);
+        } else {
+            load_row(A, ub, jbeg);
+        }
         fix_bc(A);
         {
             const float rn = right_nb(A);
@@ -216,17 +276,26 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             }
         }
         if constexpr (!KL) {
-            load_row(nA, nub, jbeg);
+            if constexpr (RING) read_row(nA, jbeg, 1); else load_row(nA, nub, jbeg);
             nlr = right_nb(nA);
 #pragma unroll
             for (int k = 0; k < NE; ++k) hnu[k] = nA.v[k] + ((k + 1 < NE) ? nA.v[(k + 1 < NE) ? k + 1 : k] : nlr);
         }
-        load_row(B, ub, jbeg + 1);
-        if constexpr (!KL) load_row(nB, nub, jbeg + 1);
 
-        // One element row: lo / cur are node rows j and j+1, nxt receives row j+2.
+        if constexpr (!RING) {
+            load_row(B, ub, jbeg + 1);
+            if constexpr (!KL) load_row(nB, nub, jbeg + 1);
+        }
+
+        // One element row: lo holds node row j, cur node row j+1 (read from the ring, or loaded by the
+        // previous step); the direct variant loads row j+2 into nxt.
         auto step = [&](Row<NE>& lo, Row<NE>& cur, Row<NE>& nxt, Row<NE>& nlo, Row<NE>& ncur, Row<NE>& nnxt, const int j) {
-            if (j < jend) {
+            if constexpr (RING) {
+                issue_row(j + T2_STAGES);               // its slot held row j, which is in registers already
+                cp_async_wait<T2_STAGES - 1>();         // row j+1 has landed
+                read_row(cur, j + 1, 0);
+                if constexpr (!KL) read_row(ncur, j + 1, 1);
+            } else if (j < jend) {
                 load_row(nxt, ub, j + 2);
                 if constexpr (!KL) load_row(nnxt, nub, j + 2);
             }
@@ -361,7 +430,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             if constexpr (!KL) nlr = nhr;
         };
 
-        // ---- march: the three row buffers rotate by name
+        // ---- march: the row buffers rotate by name
         int j = jbeg;
         Row<NE> fin;                                    // the last node row reached (for the top-row epilogue)
         while (true) {
@@ -372,6 +441,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             step(C, A, B, nC, nA, nB, j);
             if (++j > jend) { fin = A; break; }
         }
+        if constexpr (RING) cp_async_wait<0>();
 
         // ---- the top node row of the domain has no element row above it
         if (n1 == ny) {
@@ -427,7 +497,7 @@ Geo2 geometry(const dn_problem& p) {
     const int m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
     g.GS = m ? (2 * (m + 1) + 3) / 4 * 4 : 0;
     const long long slots = 2ll * sm_count();
-    const int rmax_smem = g.GS ? (int)(40960 / ((size_t)g.WY * g.GS * 4)) - 1 : 4096;
+    const int rmax_smem = g.GS ? (int)(32768 / ((size_t)g.WY * g.GS * 4)) - 1 : 4096;
     long long best = -1;
     int bestR = 16;
     for (int R = 8; R <= 512 && R <= rmax_smem; ++R) {
@@ -441,7 +511,9 @@ Geo2 geometry(const dn_problem& p) {
     g.R = bestR;
     const int nch = (ny + g.R - 1) / g.R;
     g.nblkx = (nch + g.WY - 1) / g.WY;
-    g.smem = sizeof(float) * ((size_t)g.WY * (g.R + 1) * g.GS + (size_t)g.WY * 2 * T2_MAX_WARPS * 2);
+    const size_t ring_row = (size_t)32 * g.W * 4 * g.K + 4 * ((g.W + 3) / 4);
+    g.smem = sizeof(float) * ((size_t)g.WY * (g.R + 1) * g.GS + (size_t)g.WY * 2 * T2_MAX_WARPS * 2 +
+                              (m ? 0 : (size_t)g.WY * T2_STAGES * 2 * ring_row));      // the ring serves the nodal variant
     return g;
 }
 
@@ -450,8 +522,16 @@ cudaError_t launch_kmf(const Params& P, const Geo2& g, cudaStream_t s) {
     dim3 grid((unsigned)g.nblkx, (unsigned)P.batch);
     const int threads = 32 * g.W * g.WY;
     // the energy-only kernel sums element energies; the fused kernel takes J from the residual
-    if (P.r) tiled2d_kernel<K, M, true, FULL><<<grid, threads, g.smem, s>>>(P, g.W, g.WY, g.R);
-    else tiled2d_kernel<K, M, false, FULL><<<grid, threads, g.smem, s>>>(P, g.W, g.WY, g.R);
+    cudaError_t e;
+    if (P.r) {
+        e = cudaFuncSetAttribute(tiled2d_kernel<K, M, true, FULL, (M == 0)>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+        if (e != cudaSuccess) return e;
+        tiled2d_kernel<K, M, true, FULL, (M == 0)><<<grid, threads, g.smem, s>>>(P, g.W, g.WY, g.R);
+    } else {
+        e = cudaFuncSetAttribute(tiled2d_kernel<K, M, false, FULL, (M == 0)>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+        if (e != cudaSuccess) return e;
+        tiled2d_kernel<K, M, false, FULL, (M == 0)><<<grid, threads, g.smem, s>>>(P, g.W, g.WY, g.R);
+    }
     return cudaGetLastError();
 }
 

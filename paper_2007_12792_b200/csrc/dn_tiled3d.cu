@@ -166,14 +166,15 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     }
 
     PlaneState S0, S1;
-    float L0p[4], U0p[4], carry[4], L1p[4], U1p[4], Xp[4];
+    float L0p[5], U0p[5], carry[4];                    // pending contributions to this row (5th: column of the next lane)
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         S0.u[c] = S0.e[c] = S0.s[c] = S0.txy[c] = 0.f;
         S1.u[c] = S1.e[c] = S1.s[c] = S1.txy[c] = 0.f;
         S0.h = S1.h = 0.f;
-        L0p[c] = U0p[c] = carry[c] = L1p[c] = U1p[c] = Xp[c] = 0.f;
+        L0p[c] = U0p[c] = carry[c] = 0.f;
     }
+    L0p[4] = U0p[4] = 0.f;
     float en = 0.f, enl = 0.f, ell = 0.f;
 
     auto load4 = [&](const float* ptr, float (&v)[4], float& halo) {
@@ -224,11 +225,6 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 const float wz = (p == 0 || p == nz - 1) ? 0.5f : 1.f;
                 ell = fmaf(fw * wy * wz, rs, ell);
             }
-        }
-        if (WANT_R && col_ok) {                        // contributions of the previous element step to row y+1
-            *reinterpret_cast<float4*>(sb + 2 * TYNXP) = make_float4(L1p[0], L1p[1], L1p[2], L1p[3]);
-            *reinterpret_cast<float4*>(sb + 3 * TYNXP) = make_float4(U1p[0], U1p[1], U1p[2], U1p[3]);
-            if (lane == 31) *reinterpret_cast<float4*>(sX) = make_float4(Xp[0], Xp[1], Xp[2], Xp[3]);
         }
         __syncthreads();
 
@@ -293,9 +289,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
             if (p > kbeg) {
                 const int k = p - 1;
                 const bool own_energy = (k >= p0) && (ty >= 1 || tile == 0);
-                float L0[5], L1[5], U0[5], U1[5];
-#pragma unroll
-                for (int c = 0; c < 5; ++c) { L0[c] = 0.f; L1[c] = 0.f; U0[c] = 0.f; U1[c] = 0.f; }
+                float L1[5], U1[5];                    // contributions to row y+1 (lower / upper plane)
                 float enrow = 0.f, enlast = 0.f;
                 if (elem_row_ok) {
                     const ulonglong2* gl = reinterpret_cast<const ulonglong2*>(gam + (size_t)(((k - kbeg) * TY + ty) * 2) * GS);
@@ -369,29 +363,37 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                             const float r110 = dXY - dXYZ, r101 = dXZ - dXYZ, r011 = dYZ - dXYZ;
                             const float r100 = (dE - r110) - dXZ, r010 = (dS - r110) - dYZ, r001 = (dW - r101) - dYZ;
                             const float r000 = ((r011 - dW) + (dXY - dE)) + (dXZ - dS);
-                            if (c == 0) { L0[0] = r000; L1[0] = r010; U0[0] = r001; U1[0] = r011; }
-                            else { L0[c] += r000; L1[c] += r010; U0[c] += r001; U1[c] += r011; }
-                            L0[c + 1] = r100; L1[c + 1] = r110; U0[c + 1] = r101; U1[c + 1] = dXYZ;
+                            if (c == 0) { L0p[0] = r000; L1[0] = r010; U0p[0] = r001; U1[0] = r011; }
+                            else { L0p[c] += r000; L1[c] += r010; U0p[c] += r001; U1[c] += r011; }
+                            L0p[c + 1] = r100; L1[c + 1] = r110; U0p[c + 1] = r101; U1[c + 1] = dXYZ;
                         }
                     }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 5; ++c) { L0p[c] = 0.f; L1[c] = 0.f; U0p[c] = 0.f; U1[c] = 0.f; }
                 }
                 if (WANT_R) {
                     // the left neighbour's last element feeds this thread's first node column
-                    const float a100 = __shfl_up_sync(0xffffffffu, L0[4], 1), a110 = __shfl_up_sync(0xffffffffu, L1[4], 1);
-                    const float a101 = __shfl_up_sync(0xffffffffu, U0[4], 1), a111 = __shfl_up_sync(0xffffffffu, U1[4], 1);
-                    if (lane > 0) { L0[0] += a100; L1[0] += a110; U0[0] += a101; U1[0] += a111; }
-                    Xp[0] = L0[4]; Xp[1] = L1[4]; Xp[2] = U0[4]; Xp[3] = U1[4];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) { L0p[c] = L0[c]; U0p[c] = U0[c]; L1p[c] = L1[c]; U1p[c] = U1[c]; }
+                    const float a100 = __shfl_up_sync(0xffffffffu, L0p[4], 1), a110 = __shfl_up_sync(0xffffffffu, L1[4], 1);
+                    const float a101 = __shfl_up_sync(0xffffffffu, U0p[4], 1), a111 = __shfl_up_sync(0xffffffffu, U1[4], 1);
+                    if (lane > 0) { L0p[0] += a100; L1[0] += a110; U0p[0] += a101; U1[0] += a111; }
+                    // what goes to row y+1 and to the warp on the right is published by the next step's
+                    // barrier: write it into the other exchange buffer now (its readers finished before
+                    // this step's barrier)
+                    float* so = smem + (PAR ^ 1) * BUF + ty * NXP + x0;
+                    if (col_ok) {
+                        *reinterpret_cast<float4*>(so + 2 * TYNXP) = make_float4(L1[0], L1[1], L1[2], L1[3]);
+                        *reinterpret_cast<float4*>(so + 3 * TYNXP) = make_float4(U1[0], U1[1], U1[2], U1[3]);
+                    }
+                    if (lane == 31)
+                        *reinterpret_cast<float4*>(smem + (PAR ^ 1) * BUF + XOFF + (ty * WX + wx) * 4) =
+                            make_float4(L0p[4], L1[4], U0p[4], U1[4]);
                 }
                 if (own_energy && elem_row_ok) {
                     en += enrow;
                     if (!last_elem_missing) enl += enlast;
                 }
             }
-        } else if (WANT_R) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) { L0p[c] = 0.f; U0p[c] = 0.f; L1p[c] = 0.f; U1p[c] = 0.f; Xp[c] = 0.f; }
         }
     };
 
