@@ -1,5 +1,5 @@
 // Tiled 3D kernel: fused element quadrature, energy reduction, node gather, mask and store on
-// hexahedra, for DN_NU_KL_GAUSS with constant forcing.
+// hexahedra, for both diffusivity modes, with constant forcing.
 //
 // Layout of the work.  A block owns a tile of TY node rows (y) across the whole x extent
 // (WX warps of 128 nodes, 4 consecutive nodes per lane) and marches over a chunk of node planes
@@ -56,7 +56,11 @@ __device__ __forceinline__ u64 fma2_3(u64 a, u64 b, u64 c) {
 }
 
 // Register state of one staged node plane, for the 4 node columns of a thread.
-struct PlaneState { float u[4], h, e[4], s[4], txy[4]; };   // h: node right of the strip (lane 31)
+struct PlaneState {
+    float u[4], h, e[4], s[4], txy[4];     // h: node right of the strip (lane 31)
+    float n[4], nh;                        // nodal mode: staged diffusivity of the own row (prefetch target)
+    float v[4][4];                         // nodal mode: nu interpolated to the 4 (xi, eta) points of each element, on this plane
+};
 
 // Floats per Gauss row pair (q fixed, s = a and b interleaved) in the coefficient table.
 template <int M> struct Gs3p { static constexpr int value = (2 * (M + 1) + 3) / 4 * 4; };
@@ -65,7 +69,10 @@ template <int M, bool WANT_R, bool FULL>
 __global__ void __launch_bounds__(T3_THREADS, 1)
 tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const int ntile_y) {
     extern __shared__ __align__(16) float smem[];
-    constexpr int GS = Gs3p<M>::value;                  // floats per (row q) line pair
+    constexpr bool KL = (M > 0);
+    constexpr int MM = KL ? M : 1;
+    constexpr int GS = Gs3p<MM>::value;                 // floats per (row q) line pair
+    constexpr int NARR = KL ? 4 : 5;                    // exchange arrays: u, e, L1, U1 (, nu)
     const int lane = threadIdx.x & 31;
     const int wid = threadIdx.x >> 5;
     const int wx = wid % WX, ty = wid / WX;
@@ -85,20 +92,20 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
 
     // shared memory: two exchange buffers, then the KL coefficients of every Gauss line of the block
     const int TYNXP = TY * NXP;
-    const int XOFF = 4 * TYNXP;                        // floats before the cross-warp slots
+    const int XOFF = NARR * TYNXP;                     // floats before the cross-warp slots
     const int BUF = XOFF + TY * WX * 4;
     float* gam = smem + 2 * BUF;
 
     // ---- prologue: KL polynomial coefficients; table index ((k - kbeg) * TY + row) * 2 + q, entries
     // interleave the two Gauss planes s = a, b of the element plane: [coef][s]
-    {
+    if constexpr (KL) {
         const int nlines = (kend - kbeg + 1) * TY * 4;
         const float* c = P.ckl + (size_t)b * M * M * M;
         for (int t = threadIdx.x; t < nlines; t += blockDim.x) {
             const int s = t & 1, q = (t >> 1) & 1, row = (t >> 2) % TY, kk = (t >> 2) / TY;
             const int gy = min(2 * (y0 + row) + q, 2 * (ny - 1) - 1);
             const int gz = 2 * (kbeg + kk) + s;
-            double g[M];
+            double g[MM];
 #pragma unroll
             for (int i = 0; i < M; ++i) {
                 double acc = 0.0;
@@ -112,14 +119,14 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 }
                 g[i] = acc;
             }
-            double acc[M + 1], tp[M + 1], tc[M + 1];
+            double acc[MM + 1], tp[MM + 1], tc[MM + 1];
 #pragma unroll
             for (int k = 0; k <= M; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
 #pragma unroll
             for (int i = 1; i <= M; ++i) {
 #pragma unroll
                 for (int k = 0; k <= M; ++k) acc[k] += g[i - 1] * tc[k];
-                double tn[M + 1];
+                double tn[MM + 1];
 #pragma unroll
                 for (int k = 0; k <= M; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
 #pragma unroll
@@ -152,10 +159,12 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     const size_t plane = (size_t)nx * ny;
     const float* pu = P.u + (size_t)b * P.nodes + (size_t)yl * nx + x0;      // own row, plane 0
     const float* pa = P.u + (size_t)b * P.nodes + (size_t)ya * nx + x0;      // row above (top warp row only)
+    const float* pn = KL ? nullptr : P.nu + (size_t)b * P.nodes + (size_t)yl * nx + x0;
+    const float* pna = KL ? nullptr : P.nu + (size_t)b * P.nodes + (size_t)ya * nx + x0;
     float* pr = WANT_R ? P.r + (size_t)b * P.nodes + (size_t)yl * nx + x0 : nullptr;
 
     u64 cda[4], cdb[4];                                // cos(pi x) at the two Gauss columns, duplicated
-    {
+    if constexpr (KL) {
         float4 q0 = make_float4(0.f, 0.f, 0.f, 0.f), q1 = q0;
         if (col_ok) {
             q0 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0));
@@ -172,11 +181,24 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
         S0.u[c] = S0.e[c] = S0.s[c] = S0.txy[c] = 0.f;
         S1.u[c] = S1.e[c] = S1.s[c] = S1.txy[c] = 0.f;
         S0.h = S1.h = 0.f;
+        S0.n[c] = S1.n[c] = 0.f;
+#pragma unroll
+        for (int d = 0; d < 4; ++d) { S0.v[c][d] = 0.f; S1.v[c][d] = 0.f; }
         L0p[c] = U0p[c] = carry[c] = 0.f;
     }
     L0p[4] = U0p[4] = 0.f;
+    S0.nh = S1.nh = 0.f;
     float en = 0.f, enl = 0.f, ell = 0.f;
 
+    auto load4n = [&](const float* ptr, float (&v)[4], float& halo) {     // plain (diffusivity)
+        v[0] = v[1] = v[2] = v[3] = 0.f;
+        if (col_ok) {
+            const float4 q = __ldg(reinterpret_cast<const float4*>(ptr));
+            v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+        }
+        halo = 0.f;
+        if (halo_ok) halo = __ldg(ptr + 4);
+    };
     auto load4 = [&](const float* ptr, float (&v)[4], float& halo) {
         if (col_ok) {
             const float4 q = __ldg(reinterpret_cast<const float4*>(ptr));
@@ -201,6 +223,12 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     ua[0] = ua[1] = ua[2] = ua[3] = 0.f;
     if (kbeg & 1) load4(pu + (size_t)kbeg * plane, S1.u, S1.h); else load4(pu + (size_t)kbeg * plane, S0.u, S0.h);
     if (top_row) load4(pa + (size_t)kbeg * plane, ua, uah);
+    float na[4], nah = 0.f;                            // nodal mode: prefetched diffusivity of the row above (top warp row)
+    na[0] = na[1] = na[2] = na[3] = 0.f;
+    if constexpr (!KL) {
+        if (kbeg & 1) load4n(pn + (size_t)kbeg * plane, S1.n, S1.nh); else load4n(pn + (size_t)kbeg * plane, S0.n, S0.nh);
+        if (top_row) load4n(pna + (size_t)kbeg * plane, na, nah);
+    }
 
     // Iteration p stages node plane p into `up`, computes element plane p-1 between `lo` and `up`,
     // and finishes node plane p-2.  PAR = p & 1 selects the exchange buffer.
@@ -217,7 +245,13 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 *reinterpret_cast<float4*>(sb) = make_float4(up.u[0], up.u[1], up.u[2], up.u[3]);
                 *reinterpret_cast<float4*>(sb + TYNXP) = make_float4(up.e[0], up.e[1], up.e[2], up.e[3]);
             }
-            if (p <= kend) load4(pu + (size_t)(p + 1) * plane, lo.u, lo.h);   // prefetch the next plane (lo.u is dead)
+            if constexpr (!KL) {
+                if (col_ok) *reinterpret_cast<float4*>(sb + 4 * TYNXP) = make_float4(up.n[0], up.n[1], up.n[2], up.n[3]);
+            }
+            if (p <= kend) {                           // prefetch the next plane (lo.u / lo.n are dead)
+                load4(pu + (size_t)(p + 1) * plane, lo.u, lo.h);
+                if constexpr (!KL) load4n(pn + (size_t)(p + 1) * plane, lo.n, lo.nh);
+            }
             if (hasf && p >= p0 && p < p1 && out_row) { // load energy of the staged plane
                 float rs = (up.u[0] + up.u[1]) + (up.u[2] + up.u[3]);
                 if (first_col) rs -= 0.5f * up.u[0];
@@ -285,6 +319,36 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
             }
 #pragma unroll
             for (int c = 0; c < 4; ++c) { up.s[c] = uab[c] - up.u[c]; up.txy[c] = eab[c] - up.e[c]; }
+            if constexpr (!KL) {
+                // nu of the staged plane at the 4 (xi, eta) points of each element: x lerp on rows y and y+1, then y lerp
+                float nab[5];
+                if (!top_row) {
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float a4 = 0.f;
+                    if (col_ok) {
+                        a = *reinterpret_cast<const float4*>(sb + 4 * TYNXP + NXP);
+                        if (x0 + 4 < nx) a4 = sb[4 * TYNXP + NXP + 4];
+                    }
+                    nab[0] = a.x; nab[1] = a.y; nab[2] = a.z; nab[3] = a.w; nab[4] = a4;
+                } else {
+                    float rn = __shfl_down_sync(0xffffffffu, na[0], 1);
+                    if (lane == 31) rn = nah;
+                    nab[0] = na[0]; nab[1] = na[1]; nab[2] = na[2]; nab[3] = na[3]; nab[4] = rn;
+                    if (p <= kend) load4n(pna + (size_t)(p + 1) * plane, na, nah);
+                }
+                float nrn = __shfl_down_sync(0xffffffffu, up.n[0], 1);
+                if (lane == 31) nrn = up.nh;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float n0 = up.n[c], n1 = (c < 3) ? up.n[c < 3 ? c + 1 : c] : nrn;
+                    const float dl = n1 - n0, dh = nab[c + 1] - nab[c];
+                    const float la = fmaf(DN_GA, dl, n0), lb = fmaf(DN_GB, dl, n0);          // row y at xi = a, b
+                    const float ha = fmaf(DN_GA, dh, nab[c]), hb = fmaf(DN_GB, dh, nab[c]);  // row y+1
+                    const float da = ha - la, db = hb - lb;
+                    up.v[c][0] = fmaf(DN_GA, da, la); up.v[c][1] = fmaf(DN_GB, da, la);      // (p = a; q = a, b)
+                    up.v[c][2] = fmaf(DN_GA, db, lb); up.v[c][3] = fmaf(DN_GB, db, lb);      // (p = b; q = a, b)
+                }
+            }
 
             if (p > kbeg) {
                 const int k = p - 1;
@@ -292,28 +356,40 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 float L1[5], U1[5];                    // contributions to row y+1 (lower / upper plane)
                 float enrow = 0.f, enlast = 0.f;
                 if (elem_row_ok) {
-                    const ulonglong2* gl = reinterpret_cast<const ulonglong2*>(gam + (size_t)(((k - kbeg) * TY + ty) * 2) * GS);
                     u64 gq_a[GS / 2], gq_b[GS / 2];       // Gauss row q = a / b; each entry holds (plane s = a, s = b)
+                    if constexpr (KL) {
+                        const ulonglong2* gl = reinterpret_cast<const ulonglong2*>(gam + (size_t)(((k - kbeg) * TY + ty) * 2) * GS);
 #pragma unroll
-                    for (int i = 0; i < GS / 4; ++i) {
-                        const ulonglong2 t0 = gl[i], t1 = gl[GS / 4 + i];
-                        gq_a[2 * i] = t0.x; gq_a[2 * i + 1] = t0.y; gq_b[2 * i] = t1.x; gq_b[2 * i + 1] = t1.y;
+                        for (int i = 0; i < GS / 4; ++i) {
+                            const ulonglong2 t0 = gl[i], t1 = gl[GS / 4 + i];
+                            gq_a[2 * i] = t0.x; gq_a[2 * i + 1] = t0.y; gq_b[2 * i] = t1.x; gq_b[2 * i + 1] = t1.y;
+                        }
                     }
                     const float a = DN_GA, bq = DN_GB;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        // nu[p][q][s] at the 8 Gauss points: 4 packed Horner chains (column p, row q) x (s = a, b)
-                        u64 h_aa = gq_a[M], h_ab = gq_b[M], h_ba = gq_a[M], h_bb = gq_b[M];   // h_{p q}
-#pragma unroll
-                        for (int i = M - 1; i >= 0; --i) {
-                            h_aa = fma2_3(h_aa, cda[c], gq_a[i]); h_ab = fma2_3(h_ab, cda[c], gq_b[i]);
-                            h_ba = fma2_3(h_ba, cdb[c], gq_a[i]); h_bb = fma2_3(h_bb, cdb[c], gq_b[i]);
-                        }
                         float n000, n001, n010, n011, n100, n101, n110, n111;               // n p q s
-                        unpack2_3(h_aa, n000, n001); unpack2_3(h_ab, n010, n011);
-                        unpack2_3(h_ba, n100, n101); unpack2_3(h_bb, n110, n111);
-                        n000 = ex2_approx3(n000); n001 = ex2_approx3(n001); n010 = ex2_approx3(n010); n011 = ex2_approx3(n011);
-                        n100 = ex2_approx3(n100); n101 = ex2_approx3(n101); n110 = ex2_approx3(n110); n111 = ex2_approx3(n111);
+                        if constexpr (KL) {
+                            // nu[p][q][s] at the 8 Gauss points: 4 packed Horner chains (column p, row q) x (s = a, b)
+                            u64 h_aa = gq_a[MM], h_ab = gq_b[MM], h_ba = gq_a[MM], h_bb = gq_b[MM];   // h_{p q}
+#pragma unroll
+                            for (int i = MM - 1; i >= 0; --i) {
+                                h_aa = fma2_3(h_aa, cda[c], gq_a[i]); h_ab = fma2_3(h_ab, cda[c], gq_b[i]);
+                                h_ba = fma2_3(h_ba, cdb[c], gq_a[i]); h_bb = fma2_3(h_bb, cdb[c], gq_b[i]);
+                            }
+                            unpack2_3(h_aa, n000, n001); unpack2_3(h_ab, n010, n011);
+                            unpack2_3(h_ba, n100, n101); unpack2_3(h_bb, n110, n111);
+                            n000 = ex2_approx3(n000); n001 = ex2_approx3(n001); n010 = ex2_approx3(n010); n011 = ex2_approx3(n011);
+                            n100 = ex2_approx3(n100); n101 = ex2_approx3(n101); n110 = ex2_approx3(n110); n111 = ex2_approx3(n111);
+                        } else {
+                            // nodal mode: z lerp between the (xi, eta)-interpolated values of planes k and k+1
+                            const float d0 = up.v[c][0] - lo.v[c][0], d1 = up.v[c][1] - lo.v[c][1];
+                            const float d2 = up.v[c][2] - lo.v[c][2], d3 = up.v[c][3] - lo.v[c][3];
+                            n000 = fmaf(a, d0, lo.v[c][0]); n001 = fmaf(bq, d0, lo.v[c][0]);
+                            n010 = fmaf(a, d1, lo.v[c][1]); n011 = fmaf(bq, d1, lo.v[c][1]);
+                            n100 = fmaf(a, d2, lo.v[c][2]); n101 = fmaf(bq, d2, lo.v[c][2]);
+                            n110 = fmaf(a, d3, lo.v[c][3]); n111 = fmaf(bq, d3, lo.v[c][3]);
+                        }
                         float Nx_aa = n000 + n100, Nx_ab = n001 + n101, Nx_ba = n010 + n110, Nx_bb = n011 + n111;   // (q, s)
                         float Ny_aa = n000 + n010, Ny_ab = n001 + n011, Ny_ba = n100 + n110, Ny_bb = n101 + n111;   // (p, s)
                         float Nz_aa = n000 + n001, Nz_ab = n010 + n011, Nz_ba = n100 + n101, Nz_bb = n110 + n111;   // (p, q)
@@ -442,10 +518,10 @@ Geo3 geometry3(const dn_problem& p) {
     g.TY = (T3_THREADS / 32) / g.WX;
     if (g.TY > ny) g.TY = (ny < 2) ? 2 : ny;
     g.ntile_y = (ny - 1 + (g.TY - 1) - 1) / (g.TY - 1);
-    const int m = p.kl_modes;
-    g.GS = (2 * (m + 1) + 3) / 4 * 4;               // floats per Gauss-row line pair
+    const int m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
+    g.GS = m ? (2 * (m + 1) + 3) / 4 * 4 : 0;               // floats per Gauss-row line pair
     const long long slots = sm_count3();
-    const size_t fixed = sizeof(float) * 2 * ((size_t)4 * g.TY * g.WX * 128 + (size_t)g.TY * g.WX * 4);
+    const size_t fixed = sizeof(float) * 2 * ((size_t)(m ? 4 : 5) * g.TY * g.WX * 128 + (size_t)g.TY * g.WX * 4);
     long long best = -1;
     int bestZ = 8;
     for (int Z = 4; Z <= 256; ++Z) {
@@ -489,7 +565,7 @@ cudaError_t launch_m(const Params& P, const Geo3& g, cudaStream_t s) {
 }  // namespace
 
 bool tiled3d_applicable(const dn_problem& p) {
-    return p.grid.dim == 3 && p.nu_mode == DN_NU_KL_GAUSS && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 512 &&
+    return p.grid.dim == 3 && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 512 &&
            p.grid.ny >= 2 && p.grid.nz >= 2;
 }
 
@@ -510,6 +586,7 @@ cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s) {
     const Geo3 g = geometry3(p);
     (void)l;
     switch (P.m) {
+        case 0: return launch_m<0>(P, g, s);
         case 1: return launch_m<1>(P, g, s);
         case 2: return launch_m<2>(P, g, s);
         case 3: return launch_m<3>(P, g, s);
