@@ -31,9 +31,31 @@ from paper_2007_12792_b200 import inputs  # noqa: E402
 METRIC = "fused FEM energy+residual Gelements/s"
 UNIT = "Gelements/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/; None where the kernel has changed since the capture.
-NCU_TRAFFIC_BYTES = {}
+FP32_PEAK_LANE_OPS = 148 * 128 * 1.965e9     # SMs x FP32 lanes x max SM clock: the FP32 issue roof (lane-ops/s)
+# Counters of the dominant kernel from the ncu captures summarised under profiles/: DRAM bytes per
+# launch (dram__bytes_read.sum + dram__bytes_write.sum) and executed FP32 lane-operations per element
+# (FADD + FMUL + FFMA + 2 FFMA2).  Each entry names the kernel source it was taken from and the first 16
+# hex digits of its sha256: once that file changes the entry no longer applies and null is reported.
+NCU_CAPTURES = {
+    "tiled2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 500950272, "fp32_ops_per_element": 55.2,
+                                          "src": "dn_tiled2d.cu", "sha": "0050c2f08c260d14"},
+    "tiled3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 497360128, "fp32_ops_per_element": 171.7,
+                                        "src": "dn_tiled3d.cu", "sha": "e8a35cdd8d0b0d65"},
+}
+
+
+def ncu_capture(key):
+    import hashlib
+    c = NCU_CAPTURES.get(key)
+    if not c:
+        return None
+    try:
+        with open(os.path.join(ROOT, "paper_2007_12792_b200", "csrc", c["src"]), "rb") as fh:
+            if hashlib.sha256(fh.read()).hexdigest()[:16] != c["sha"]:
+                return None
+    except OSError:
+        return None
+    return c
 
 
 def measured_peak():
@@ -257,6 +279,13 @@ def main():
         achieved = alg_bytes / (main_ms * 1e-3) / 1e9
         path = B.dn_path_name(prob)
         key = f"{path}:{wl.name}:{args.nu_mode}"
+        cap = ncu_capture(key)
+        alu = None
+        if cap:
+            ops = cap["fp32_ops_per_element"] * elements / (main_ms * 1e-3)
+            alu = {"bound": "alu", "achieved": ops / 1e12, "peak": FP32_PEAK_LANE_OPS / 1e12, "unit": "T FP32 lane-ops/s",
+                   "frac": ops / FP32_PEAK_LANE_OPS, "fp32_ops_per_element": cap["fp32_ops_per_element"],
+                   "note": "executed FP32 operations (ncu) / kernel time, against SMs x 128 lanes x max clock"}
         line = {
             "metric": METRIC, "value": world * elements / (step_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
@@ -272,7 +301,8 @@ def main():
             "roofline": {"bound": "hbm", "kernel": f"fused energy+residual ({path})", "achieved": achieved,
                          "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                          "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": main_ms,
-                         "traffic": NCU_TRAFFIC_BYTES.get(key)},
+                         "traffic": cap["traffic"] if cap else None},
+            "roofline_alu": alu,
             "checksum_J": Jsum,
         }
         if not args.no_cpu_baseline and world == 1:
