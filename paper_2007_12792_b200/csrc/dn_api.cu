@@ -76,6 +76,8 @@ WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
         w.cg[a] = off;
         off += align_up(sizeof(float) * (size_t)m * w.gstride[a] + 16);
     }
+    w.seam = off;
+    if ((tight ? l.path == PATH_TILED3D : tiled3d_applicable(p))) off += align_up(sizeof(float) * tiled3d_seam_floats(p) + 16);
     w.total = off;
     return w;
 }
@@ -93,6 +95,7 @@ static Params make_params(const dn_problem& p, const WsLayout& w, const float* u
     P.ckl = reinterpret_cast<const float*>(base + w.ckl);
     for (int a = 0; a < 3; ++a) { P.cg[a] = reinterpret_cast<const float*>(base + w.cg[a]); P.gstride[a] = w.gstride[a]; }
     P.nblk = w.nblk;
+    P.seam = reinterpret_cast<float*>(base + w.seam);
     P.nodes = nodes_per_sample(p.grid);
     return P;
 }
@@ -254,7 +257,8 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
 
 int32_t dn_launches_per_call(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
-    return 2 + (p->nu_mode == DN_NU_KL_GAUSS ? 1 : 0);
+    const bool t3 = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
+    return 2 + (p->nu_mode == DN_NU_KL_GAUSS ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
 }
 
 const char* dn_path_name(const dn_problem* p) {

@@ -24,6 +24,7 @@ struct WsLayout {
     size_t partials;      // double [B][nblk][2]  (diffusion part, load part)
     size_t ckl;           // float  [B][m^dim]    KL weights * log2(e) / (1 + i^2 + j^2 (+ k^2))
     size_t cg[3];         // float  [m][gstride[a]] cos(i pi x) at the Gauss abscissae of axis a
+    size_t seam;          // float  [B][nseam][nz][nx] contributions across tile seams (tiled 3D kernel)
     int gstride[3];       // padded row length of cg[a] (multiple of 4)
     int nblk;             // energy partials per sample
     size_t total;
@@ -47,6 +48,8 @@ struct Params {
     int gstride[3];
     int nblk;
     long long nodes;      // per sample
+    float* seam;          // tiled 3D: contributions of a tile's top element row to the next tile's first node row
+    int nseam;
 };
 
 struct Launch {           // tiled-path launch geometry chosen on the host
@@ -75,6 +78,7 @@ bool tiled2d_applicable(const dn_problem& p);
 bool tiled3d_applicable(const dn_problem& p);
 Launch tiled2d_geometry(const dn_problem& p);
 Launch tiled3d_geometry(const dn_problem& p);
+size_t tiled3d_seam_floats(const dn_problem& p);   // scratch floats the tiled 3D kernel needs for its tile seams
 
 #ifdef __CUDACC__
 // Sum (d, l) over the block in a fixed order and let thread 0 store the pair.

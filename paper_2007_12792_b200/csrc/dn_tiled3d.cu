@@ -11,8 +11,10 @@
 // lane by shuffle (to the next warp through shared memory), those to row y+1 through shared
 // memory, those to plane k+1 are carried to the next step.  One barrier per plane: the exchange
 // of a step's row-(y+1) contributions rides on the barrier of the next step, so a node plane is
-// finished two steps after it was staged.  The first row of a tile and the first plane of a
-// chunk are recomputed by the neighbouring block (1/TY and 1/Z redundancy).
+// finished two steps after it was staged.  Tiles do not overlap in y: the top element row of a
+// tile writes what it contributes to the next tile's first node row into a global scratch array
+// (seam), and a small second kernel adds those rows to r in a fixed order.  The first plane of a z
+// chunk is recomputed by the chunk below (1/Z redundancy).
 //
 // Arithmetic of one element, with the corner values u_ijk (i, j, k the x, y, z bits):
 //   e = u100-u000, s = u010-u000, w = u001-u000                      (edge differences at the low corner)
@@ -80,15 +82,17 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     const int tile = blockIdx.x % ntile_y, zc = blockIdx.x / ntile_y;
     const int nx = P.nx, ny = P.ny, nz = P.nz;
     const int NXP = WX * 128;
-    const int y0 = tile * (TY - 1);
+    const int y0 = tile * TY;
     const int y = y0 + ty;                             // node row and element row of this thread
     const int x0 = wx * 128 + 4 * lane;
     const int p0 = zc * Z, p1 = min(p0 + Z, nz);
     const int kbeg = max(p0 - 1, 0), kend = min(p1 - 1, nz - 2);
     const bool col_ok = FULL || (x0 < nx);
     const bool elem_row_ok = (y < ny - 1);
-    const bool out_row = (y < ny) && (ty >= 1 || tile == 0);
+    const bool out_row = (y < ny);
     const bool top_row = (ty == TY - 1);
+    // the top element row of a tile also feeds the first node row of the next tile: through global scratch
+    const bool seam_row = WANT_R && top_row && (tile + 1 < ntile_y) && (y + 1 < ny);
 
     // shared memory: two exchange buffers, then the KL coefficients of every Gauss line of the block
     const int TYNXP = TY * NXP;
@@ -161,6 +165,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     const float* pa = P.u + (size_t)b * P.nodes + (size_t)ya * nx + x0;      // row above (top warp row only)
     const float* pn = KL ? nullptr : P.nu + (size_t)b * P.nodes + (size_t)yl * nx + x0;
     const float* pna = KL ? nullptr : P.nu + (size_t)b * P.nodes + (size_t)ya * nx + x0;
+    float* pseam = seam_row ? P.seam + (((size_t)b * (ntile_y - 1) + tile) * nz) * nx + x0 : nullptr;
     float* pr = WANT_R ? P.r + (size_t)b * P.nodes + (size_t)yl * nx + x0 : nullptr;
 
     u64 cda[4], cdb[4];                                // cos(pi x) at the two Gauss columns, duplicated
@@ -176,6 +181,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
 
     PlaneState S0, S1;
     float L0p[5], U0p[5], carry[4];                    // pending contributions to this row (5th: column of the next lane)
+    float scarry[4] = {0.f, 0.f, 0.f, 0.f};            // seam rows: upper-plane contributions to the next tile's first row
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         S0.u[c] = S0.e[c] = S0.s[c] = S0.txy[c] = 0.f;
@@ -280,6 +286,26 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 }
             }
             const int pl = p - 2;                      // the plane being finished
+            if (seam_row) {                            // same finish for the node row above, which the next tile owns
+                float l1v[4] = {0.f, 0.f, 0.f, 0.f}, u1v[4] = {0.f, 0.f, 0.f, 0.f};
+                if (col_ok) {
+                    const float4 a = *reinterpret_cast<const float4*>(sb + 2 * TYNXP);
+                    const float4 c4 = *reinterpret_cast<const float4*>(sb + 3 * TYNXP);
+                    l1v[0] = a.x; l1v[1] = a.y; l1v[2] = a.z; l1v[3] = a.w;
+                    u1v[0] = c4.x; u1v[1] = c4.y; u1v[2] = c4.z; u1v[3] = c4.w;
+                }
+                if (lane == 0 && wx > 0) {
+                    const float4 me = *reinterpret_cast<const float4*>(sX - 4);
+                    l1v[0] += me.y; u1v[0] += me.w;
+                }
+                const float scs = gs * kap;
+                float o[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) { o[c] = scs * (l1v[c] + scarry[c]); scarry[c] = u1v[c]; }
+                if (!nomask) { o[0] *= mfirst; o[3] *= mlast; }
+                if (pl >= p0 && col_ok)
+                    *reinterpret_cast<float4*>(pseam + (size_t)pl * nx) = make_float4(o[0], o[1], o[2], o[3]);
+            }
             const float wz = (pl == 0 || pl == nz - 1) ? 0.5f : 1.f;
             const float lw = fw * wy * wz;
             const float sc = gs * kap, nl = -gs * lw;
@@ -352,7 +378,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
 
             if (p > kbeg) {
                 const int k = p - 1;
-                const bool own_energy = (k >= p0) && (ty >= 1 || tile == 0);
+                const bool own_energy = (k >= p0);
                 float L1[5], U1[5];                    // contributions to row y+1 (lower / upper plane)
                 float enrow = 0.f, enlast = 0.f;
                 if (elem_row_ok) {
@@ -496,11 +522,37 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
         else { if (first_col) o[0] -= 0.5f * nl; if (last_col) o[3] -= 0.5f * nl; }
         *reinterpret_cast<float4*>(pr + (size_t)(nz - 1) * plane) = make_float4(o[0], o[1], o[2], o[3]);
     }
+    if (seam_row && p1 == nz && col_ok) {
+        const float scs = gs * kap;
+        float o[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) o[c] = scs * scarry[c];
+        if (!nomask) { o[0] *= mfirst; o[3] *= mlast; }
+        *reinterpret_cast<float4*>(pseam + (size_t)(nz - 1) * nx) = make_float4(o[0], o[1], o[2], o[3]);
+    }
     const double etot = 0.5 * (double)kap * ((double)en + (double)enl);
     block_reduce_store(etot, (double)ell, P.partials + 2 * ((size_t)b * P.nblk + blockIdx.x));
 }
 
-struct Geo3 { int WX, TY, Z, ntile_y, nchunk_z, GS; size_t smem; };
+// Adds the seam contributions to the first node row of every tile but the first (fixed order: deterministic).
+__global__ void seam_fixup_kernel(float* __restrict__ r, const float* __restrict__ seam, int nx, int ny, int nz,
+                                  int TY, int nseam, long long total4) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total4) return;
+    const int nx4 = nx / 4;
+    const int x4 = (int)(i % nx4);
+    long long t = i / nx4;
+    const int pl = (int)(t % nz); t /= nz;
+    const int sm = (int)(t % nseam);
+    const int b = (int)(t / nseam);
+    const float4 a = __ldg(reinterpret_cast<const float4*>(seam) + i);
+    float4* dst = reinterpret_cast<float4*>(r + (((size_t)b * nz + pl) * ny + (size_t)(sm + 1) * TY) * nx) + x4;
+    float4 v = *dst;
+    v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+    *dst = v;
+}
+
+struct Geo3 { int WX, TY, Z, ntile_y, nchunk_z, GS, bps; size_t smem; };
 
 int sm_count3() {
     int dev = 0, n = 0;
@@ -512,32 +564,45 @@ int sm_count3() {
 }
 
 Geo3 geometry3(const dn_problem& p) {
-    Geo3 g{};
+    Geo3 best{};
     const int nx = p.grid.nx, ny = p.grid.ny, nz = p.grid.nz;
-    g.WX = (nx + 127) / 128;
-    g.TY = (T3_THREADS / 32) / g.WX;
-    if (g.TY > ny) g.TY = (ny < 2) ? 2 : ny;
-    g.ntile_y = (ny - 1 + (g.TY - 1) - 1) / (g.TY - 1);
+    const int WX = (nx + 127) / 128;
     const int m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
-    g.GS = m ? (2 * (m + 1) + 3) / 4 * 4 : 0;               // floats per Gauss-row line pair
-    const long long slots = sm_count3();
-    const size_t fixed = sizeof(float) * 2 * ((size_t)(m ? 4 : 5) * g.TY * g.WX * 128 + (size_t)g.TY * g.WX * 4);
-    long long best = -1;
-    int bestZ = 8;
-    for (int Z = 4; Z <= 256; ++Z) {
-        if (Z > nz && Z > 4) break;
-        const size_t sm = fixed + sizeof(float) * (size_t)(Z + 1) * g.TY * 2 * g.GS;
-        if (sm > 200 * 1024) break;
-        const long long nch = (nz + Z - 1) / Z;
-        const long long blocks = (long long)p.batch * g.ntile_y * nch;
-        const long long waves = (blocks + slots - 1) / slots;
-        const long long cost = waves * (Z + 3) * 1000 + 1000 / Z;
-        if (best < 0 || cost < best) { best = cost; bestZ = Z; }
+    const int GS = m ? (2 * (m + 1) + 3) / 4 * 4 : 0;               // floats per Gauss-row line pair
+    const int sms = sm_count3();
+    double best_cost = -1.0;
+    const int ty_max = (T3_THREADS / 32) / WX;
+    // Tiles do not overlap, so any tile height works.  Pick (TY, Z) by a cost model fitted to sweeps on
+    // B200: work grows with the warm-up plane of every z chunk, blocks should fill whole waves, an SM
+    // wants 16 resident warps (128 registers each) in more than one block (barriers), and very flat tiles
+    // pay more seam traffic.
+    for (int TY = 2; TY <= ty_max; ++TY) {
+        if (TY > ny && TY > 2) break;
+        int bps = 16 / (WX * TY);                                    // blocks per SM by registers
+        if (bps < 1) bps = 1;
+        if (bps > 4) bps = 4;
+        const int warps = bps * WX * TY;
+        const long long ntile = (ny + TY - 1) / TY;
+        const size_t fixed = sizeof(float) * 2 * ((size_t)(m ? 4 : 5) * TY * WX * 128 + (size_t)TY * WX * 4);
+        for (int Z = 4; Z <= 256; ++Z) {
+            if (Z > nz && Z > 4) break;
+            const size_t sm = fixed + sizeof(float) * (size_t)(Z + 1) * TY * 2 * GS;
+            if (sm * bps > 200 * 1024) break;
+            const long long nch = (nz + Z - 1) / Z;
+            const long long blocks = (long long)p.batch * ntile * nch;
+            const long long slots = (long long)sms * bps;
+            const long long waves = (blocks + slots - 1) / slots;
+            const double work = (double)blocks * (Z + 3) * TY;
+            const double imbalance = (double)waves * slots / (double)blocks;
+            const double cost = work * imbalance * (16.0 / warps) * (1.0 + 0.1 / TY) * (1.0 + 0.05 / bps);
+            if (best_cost < 0 || cost < best_cost) {
+                best_cost = cost;
+                best.WX = WX; best.TY = TY; best.Z = Z; best.ntile_y = (int)ntile; best.nchunk_z = (int)nch;
+                best.GS = GS; best.bps = bps; best.smem = sm;
+            }
+        }
     }
-    g.Z = bestZ;
-    g.nchunk_z = (nz + g.Z - 1) / g.Z;
-    g.smem = fixed + sizeof(float) * (size_t)(g.Z + 1) * g.TY * 2 * g.GS;
-    return g;
+    return best;
 }
 
 template <int M, bool FULL>
@@ -549,6 +614,11 @@ cudaError_t launch_mf(const Params& P, const Geo3& g, cudaStream_t s) {
         e = cudaFuncSetAttribute(tiled3d_kernel<M, true, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
         if (e != cudaSuccess) return e;
         tiled3d_kernel<M, true, FULL><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y);
+        if (g.ntile_y > 1) {
+            const long long total4 = (long long)P.batch * (g.ntile_y - 1) * P.nz * (P.nx / 4);
+            seam_fixup_kernel<<<(unsigned)((total4 + 255) / 256), 256, 0, s>>>(P.r, P.seam, P.nx, P.ny, P.nz, g.TY,
+                                                                              g.ntile_y - 1, total4);
+        }
     } else {
         e = cudaFuncSetAttribute(tiled3d_kernel<M, false, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
         if (e != cudaSuccess) return e;
@@ -567,6 +637,12 @@ cudaError_t launch_m(const Params& P, const Geo3& g, cudaStream_t s) {
 bool tiled3d_applicable(const dn_problem& p) {
     return p.grid.dim == 3 && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 512 &&
            p.grid.ny >= 2 && p.grid.nz >= 2;
+}
+
+size_t tiled3d_seam_floats(const dn_problem& p) {
+    if (!tiled3d_applicable(p)) return 0;
+    const Geo3 g = geometry3(p);
+    return (size_t)p.batch * (g.ntile_y - 1) * p.grid.nz * p.grid.nx;
 }
 
 Launch tiled3d_geometry(const dn_problem& p) {
