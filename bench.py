@@ -26,7 +26,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2007_12792_b200 import inputs  # noqa: E402
+from paper_2007_12792_b200 import inputs, sharding  # noqa: E402
 
 METRIC = "fused FEM energy+residual Gelements/s"
 UNIT = "Gelements/s"
@@ -190,8 +190,9 @@ def main():
     B.lib()
 
     wl = inputs.WORKLOADS[args.config]
-    # every rank draws its own batch: sample indices rank*B .. rank*B + B-1 of the same recipe
-    inp = inputs.make_inputs(args.config, samples=range(rank * wl.batch, (rank + 1) * wl.batch))
+    # every rank draws its own contiguous piece of the global mini-batch (world * B samples of the same recipe)
+    inp = inputs.make_inputs(args.config, samples=sharding.minibatch_indices(world * wl.batch, world * wl.batch,
+                                                                           world, rank, 0))
     u = torch.from_numpy(inp.u).cuda()
     w = torch.from_numpy(inp.kl_w).cuda()
     nu = None
@@ -266,10 +267,8 @@ def main():
     h2d = field_bytes + w.numel() * 4 + (field_bytes if nu is not None else 0)
     d2h = field_bytes + inp.batch * 4
 
-    t = torch.tensor([step_ms, main_ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    step_ms, main_ms, e2e_ms = (float(x) for x in t.cpu())
+    step_ms, main_ms, e2e_ms = sharding.max_over_ranks([step_ms, main_ms, e2e_ms])
+    Jmean = sharding.mean_over_ranks(Jsum, inp.batch)          # the averaged loss of Algorithm 1 (one scalar all-reduce)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -303,7 +302,7 @@ def main():
                          "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": main_ms,
                          "traffic": cap["traffic"] if cap else None},
             "roofline_alu": alu,
-            "checksum_J": Jsum,
+            "checksum_J": Jsum, "mean_J_all_ranks": Jmean,
         }
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = oracle_sample_run(args.config, args.nu_mode)[0]
