@@ -247,6 +247,26 @@ def test_nodal_mode_trapezoid_energy_and_three_point_rule(dim, nx, ny, nz):
     assert np.abs(a[3] - b[3]).max() < 1e-12 * np.abs(a[3]).max()
 
 
+def test_single_element_interpolated_nodal_nu_closed_form():
+    """One element, u = x y (z): the integrand nu |grad u|^2 is a polynomial, integrated by hand from 1-D moments
+    int (1-t) dt = int t dt = 1/2,  int (1-t) t^2 dt = 1/12,  int t^3 dt = 1/4.  Fails if nu is not interpolated to
+    the Gauss points (an element-mean nu gives a different number)."""
+    m0 = {0: 0.5, 1: 0.5}            # int w_i(t) dt
+    m2 = {0: 1.0 / 12.0, 1: 0.25}    # int w_i(t) t^2 dt
+    rng = np.random.default_rng(12)
+    nu = rng.uniform(0.5, 3.0, (1, 2, 2)).astype(np.float32)
+    u = np.array([[[0.0, 0.0], [0.0, 1.0]]])                       # u = x y at the corners
+    ref = 0.5 * sum(float(nu[0, j, i]) * (m0[i] * m2[j] + m2[i] * m0[j]) for i in (0, 1) for j in (0, 1))
+    p = Problem(dim=2, nx=2, ny=2, batch=1, nu_mode=NU_NODAL, nu=nu)
+    assert oracle.energy_grad(p, u, want_r=False)[0][0] == pytest.approx(ref, rel=1e-14)
+    nu3 = rng.uniform(0.5, 3.0, (1, 2, 2, 2)).astype(np.float32)
+    u3 = np.zeros((1, 2, 2, 2)); u3[0, 1, 1, 1] = 1.0             # u = x y z
+    ref3 = 0.5 * sum(float(nu3[0, k, j, i]) * (m0[i] * m2[j] * m2[k] + m2[i] * m0[j] * m2[k] + m2[i] * m2[j] * m0[k])
+                     for i in (0, 1) for j in (0, 1) for k in (0, 1))
+    p3 = Problem(dim=3, nx=2, ny=2, nz=2, batch=1, nu_mode=NU_NODAL, nu=nu3)
+    assert oracle.energy_grad(p3, u3, want_r=False)[0][0] == pytest.approx(ref3, rel=1e-14)
+
+
 # ---- P13 + KL-at-Gauss position pins ------------------------------------------------------------
 def test_kl_field_closed_forms():
     nx, ny = 9, 6
