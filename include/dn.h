@@ -88,7 +88,8 @@ typedef struct {
 } dn_problem;
 
 /* Bytes of device scratch that dn_energy / dn_energy_grad need for this problem (per-block
- * energy partials and cosine tables).  0 if the problem is invalid.  The workspace must be
+ * energy partials, cosine tables and, for 3D grids, the contributions exchanged across tile seams:
+ * about 1/4 of one field).  0 if the problem is invalid.  The workspace must be
  * 256-byte aligned; its contents need not be preserved between calls, and two calls that
  * may overlap on the device need separate workspaces. */
 size_t dn_workspace_bytes(const dn_problem* problem);
