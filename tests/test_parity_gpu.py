@@ -162,3 +162,29 @@ def test_closed_form_on_gpu():
         Jg, rg = run_gpu(pg, u)
         assert np.allclose(Jg, 1.25, rtol=1e-5)
         assert np.abs(rg).max() < 1e-5 * 2.5 / n
+
+
+def test_side_stream_and_graph_replay():
+    """Work is enqueued on the caller's stream only, and a captured dn_energy_grad replays to the same bits."""
+    for cfg, samples in ((1, range(4)), (3, range(2))):
+        inp = inputs.make_inputs(cfg, samples=samples)
+        _, pg = make_problems(inp, B.DN_NU_KL_GAUSS)
+        ud = dev(inp.u)
+        ws = B.new_workspace(pg)
+        r0 = torch.empty(pg.shape, device="cuda"); J0 = torch.empty(pg.batch, device="cuda")
+        B.dn_energy_grad(pg, ud, None, J0, r0, ws)
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        r1 = torch.zeros_like(r0); J1 = torch.zeros_like(J0)
+        with torch.cuda.stream(side):
+            B.dn_energy_grad(pg, ud, None, J1, r1, ws)
+        side.synchronize()
+        assert torch.equal(r0, r1) and torch.equal(J0, J1)
+        r2 = torch.zeros_like(r0); J2 = torch.zeros_like(J0)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            B.dn_energy_grad(pg, ud, None, J2, r2, ws)
+        r2.zero_(); J2.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(r0, r2) and torch.equal(J0, J2)
