@@ -154,7 +154,8 @@ dn_status dn_apply_bc(const dn_grid* grid, int32_t batch, float bc_x0, float bc_
 
 /* dn_energy_grad with HOST buffers: copies u (and nu / f / kl_w / gJ when present) to the
  * device staging area, runs the same kernels, copies J and r back, and waits for the last
- * copy.  In `problem`, nu / kl_w / f are HOST pointers here.  u_host, r_host: [B][..] floats;
+ * copy.  The batch is pipelined in chunks of whole samples over two internal copy streams (created
+ * and destroyed inside the call) so that both directions of the host link overlap with the kernels.  In `problem`, nu / kl_w / f are HOST pointers here.  u_host, r_host: [B][..] floats;
  * J_host: [B] floats or NULL; staging: device memory of dn_host_staging_bytes(problem) bytes,
  * 256-byte aligned.  Use pinned host memory for full copy bandwidth. */
 dn_status dn_energy_grad_host(const dn_problem* problem, const float* u_host, const float* gJ_host,

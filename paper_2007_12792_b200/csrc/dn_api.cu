@@ -206,6 +206,37 @@ dn_status dn_apply_bc(const dn_grid* g, int32_t batch, float b0, float b1, int32
                                                                                                             : DN_ERR_CUDA;
 }
 
+namespace {
+// Streams and events of one dn_energy_grad_host call (created and destroyed inside the call).
+struct HostPipe {
+    static constexpr int kMaxChunks = 32;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, copied[kMaxChunks] = {}, computed[kMaxChunks] = {};
+    bool create(int nchunks) {
+        if (cudaStreamCreateWithFlags(&in, cudaStreamNonBlocking) != cudaSuccess) return false;
+        if (cudaStreamCreateWithFlags(&out, cudaStreamNonBlocking) != cudaSuccess) return false;
+        if (cudaEventCreateWithFlags(&start, cudaEventDisableTiming) != cudaSuccess) return false;
+        for (int c = 0; c < nchunks; ++c) {
+            if (cudaEventCreateWithFlags(&copied[c], cudaEventDisableTiming) != cudaSuccess) return false;
+            if (cudaEventCreateWithFlags(&computed[c], cudaEventDisableTiming) != cudaSuccess) return false;
+        }
+        return true;
+    }
+    ~HostPipe() {
+        for (int c = 0; c < kMaxChunks; ++c) {
+            if (copied[c]) cudaEventDestroy(copied[c]);
+            if (computed[c]) cudaEventDestroy(computed[c]);
+        }
+        if (start) cudaEventDestroy(start);
+        if (in) cudaStreamDestroy(in);
+        if (out) cudaStreamDestroy(out);
+    }
+};
+}  // namespace
+
+// The batch is cut into chunks of whole samples that flow through three stages on three streams:
+// host->device copy, kernels (on the caller's stream), device->host copy.  Chunk c+1 is copied in
+// and chunk c-1 copied out while chunk c computes, so both directions of the host link stay busy.
 dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const float* gJ_host, float* J_host,
                               float* r_host, void* staging, size_t staging_bytes, void* stream) {
     dn_status st = validate(p);
@@ -214,43 +245,66 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
     if (!staging || (reinterpret_cast<uintptr_t>(staging) % kAlign) != 0 || staging_bytes < dn_host_staging_bytes(p))
         return DN_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t nfield = (size_t)p->batch * nodes_per_sample(p->grid);
+    const size_t nodes = (size_t)nodes_per_sample(p->grid);
+    const size_t nfield = (size_t)p->batch * nodes;
     const size_t field = align_up(sizeof(float) * nfield);
     const size_t small = align_up(sizeof(float) * (size_t)p->batch);
+    size_t mpow = 1;
+    for (int a = 0; a < p->grid.dim; ++a) mpow *= (size_t)((p->nu_mode == DN_NU_KL_GAUSS) ? p->kl_modes : 0);
     char* base = static_cast<char*>(staging);
     size_t off = 0;
     float* d_u = reinterpret_cast<float*>(base + off); off += field;
     float* d_r = reinterpret_cast<float*>(base + off); off += field;
     float* d_J = reinterpret_cast<float*>(base + off); off += small;
     float* d_g = reinterpret_cast<float*>(base + off); off += small;
-    dn_problem q = *p;
-#define DN_TRY(x) do { if ((x) != cudaSuccess) return DN_ERR_CUDA; } while (0)
-    DN_TRY(cudaMemcpyAsync(d_u, u_host, sizeof(float) * nfield, cudaMemcpyHostToDevice, s));
-    if (p->nu_mode == DN_NU_NODAL) {
-        float* d = reinterpret_cast<float*>(base + off); off += field;
-        DN_TRY(cudaMemcpyAsync(d, p->nu, sizeof(float) * nfield, cudaMemcpyHostToDevice, s));
-        q.nu = d;
-    }
-    if (p->f) {
-        float* d = reinterpret_cast<float*>(base + off); off += field;
-        DN_TRY(cudaMemcpyAsync(d, p->f, sizeof(float) * nfield, cudaMemcpyHostToDevice, s));
-        q.f = d;
-    }
+    float* d_nu = nullptr; float* d_f = nullptr;
+    if (p->nu_mode == DN_NU_NODAL) { d_nu = reinterpret_cast<float*>(base + off); off += field; }
+    if (p->f) { d_f = reinterpret_cast<float*>(base + off); off += field; }
+    float* d_w = reinterpret_cast<float*>(base + off); off += align_up(sizeof(float) * (size_t)p->batch * mpow + 16);
+    void* ws = base + off;
+    const size_t ws_bytes = staging_bytes - off;
+
+    // chunks of whole samples; one chunk if a chunk's workspace would not fit (its kernels may tile differently)
+    int csize = (p->batch + HostPipe::kMaxChunks - 1) / HostPipe::kMaxChunks;
+    int nchunks = (p->batch + csize - 1) / csize;
     {
-        size_t mpow = 1;
-        for (int a = 0; a < p->grid.dim; ++a) mpow *= (size_t)((p->nu_mode == DN_NU_KL_GAUSS) ? p->kl_modes : 0);
-        float* d = reinterpret_cast<float*>(base + off); off += align_up(sizeof(float) * (size_t)p->batch * mpow + 16);
-        if (p->nu_mode == DN_NU_KL_GAUSS) {
-            DN_TRY(cudaMemcpyAsync(d, p->kl_w, sizeof(float) * (size_t)p->batch * mpow, cudaMemcpyHostToDevice, s));
-            q.kl_w = d;
-        }
+        dn_problem q = *p;
+        q.batch = csize;
+        if (dn_workspace_bytes(&q) > ws_bytes) { csize = p->batch; nchunks = 1; }
     }
-    if (gJ_host) DN_TRY(cudaMemcpyAsync(d_g, gJ_host, sizeof(float) * p->batch, cudaMemcpyHostToDevice, s));
-    st = run(&q, d_u, gJ_host ? d_g : nullptr, J_host ? d_J : nullptr, d_r, base + off, staging_bytes - off, s);
-    if (st != DN_OK) return st;
-    DN_TRY(cudaMemcpyAsync(r_host, d_r, sizeof(float) * nfield, cudaMemcpyDeviceToHost, s));
-    if (J_host) DN_TRY(cudaMemcpyAsync(J_host, d_J, sizeof(float) * p->batch, cudaMemcpyDeviceToHost, s));
+    HostPipe pipe;
+    if (!pipe.create(nchunks)) return DN_ERR_CUDA;
+#define DN_TRY(x) do { if ((x) != cudaSuccess) return DN_ERR_CUDA; } while (0)
+    DN_TRY(cudaEventRecord(pipe.start, s));                       // the call is ordered after earlier work on `stream`
+    DN_TRY(cudaStreamWaitEvent(pipe.in, pipe.start, 0));
+    DN_TRY(cudaStreamWaitEvent(pipe.out, pipe.start, 0));
+    if (p->nu_mode == DN_NU_KL_GAUSS)
+        DN_TRY(cudaMemcpyAsync(d_w, p->kl_w, sizeof(float) * (size_t)p->batch * mpow, cudaMemcpyHostToDevice, pipe.in));
+    if (gJ_host) DN_TRY(cudaMemcpyAsync(d_g, gJ_host, sizeof(float) * p->batch, cudaMemcpyHostToDevice, pipe.in));
+    for (int c = 0; c < nchunks; ++c) {
+        const int b0 = c * csize;
+        const int nb = (b0 + csize <= p->batch) ? csize : p->batch - b0;
+        const size_t o = (size_t)b0 * nodes, n = (size_t)nb * nodes;
+        DN_TRY(cudaMemcpyAsync(d_u + o, u_host + o, sizeof(float) * n, cudaMemcpyHostToDevice, pipe.in));
+        if (d_nu) DN_TRY(cudaMemcpyAsync(d_nu + o, p->nu + o, sizeof(float) * n, cudaMemcpyHostToDevice, pipe.in));
+        if (d_f) DN_TRY(cudaMemcpyAsync(d_f + o, p->f + o, sizeof(float) * n, cudaMemcpyHostToDevice, pipe.in));
+        DN_TRY(cudaEventRecord(pipe.copied[c], pipe.in));
+        DN_TRY(cudaStreamWaitEvent(s, pipe.copied[c], 0));
+        dn_problem q = *p;
+        q.batch = nb;
+        q.nu = d_nu ? d_nu + o : nullptr;
+        q.f = d_f ? d_f + o : nullptr;
+        q.kl_w = (p->nu_mode == DN_NU_KL_GAUSS) ? d_w + (size_t)b0 * mpow : nullptr;
+        st = run(&q, d_u + o, gJ_host ? d_g + b0 : nullptr, J_host ? d_J + b0 : nullptr, d_r + o, ws, ws_bytes, s);
+        if (st != DN_OK) { cudaStreamSynchronize(pipe.in); cudaStreamSynchronize(s); cudaStreamSynchronize(pipe.out); return st; }
+        DN_TRY(cudaEventRecord(pipe.computed[c], s));
+        DN_TRY(cudaStreamWaitEvent(pipe.out, pipe.computed[c], 0));
+        DN_TRY(cudaMemcpyAsync(r_host + o, d_r + o, sizeof(float) * n, cudaMemcpyDeviceToHost, pipe.out));
+    }
+    if (J_host) DN_TRY(cudaMemcpyAsync(J_host, d_J, sizeof(float) * p->batch, cudaMemcpyDeviceToHost, pipe.out));
+    DN_TRY(cudaStreamSynchronize(pipe.in));
     DN_TRY(cudaStreamSynchronize(s));
+    DN_TRY(cudaStreamSynchronize(pipe.out));
 #undef DN_TRY
     return DN_OK;
 }
