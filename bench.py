@@ -145,7 +145,9 @@ def run_reference(args):
     wl = inputs.WORKLOADS[args.config]
     times, base, n = [], None, 1
     for it in range(args.warmup + args.steps):
-        base, t, n = oracle_sample_run(args.config, args.nu_mode, target_seconds=4.0)
+        # each step is a bounded sample sized so that the whole run stays within a few minutes
+        base, t, n = oracle_sample_run(args.config, args.nu_mode,
+                                       target_seconds=max(0.5, min(4.0, 150.0 / (args.steps + args.warmup))))
         if it >= args.warmup:
             times.append(t)
     ms = 1e3 * sum(times) / len(times)
@@ -246,6 +248,35 @@ def main():
     main_ms = sum(a.elapsed_time(b_) for a, b_ in ev_main) / K
     Jsum = float(J.double().sum())
 
+    # ---- L2-resident workloads: also time warm (no flush) and as a replayed CUDA graph (launch-bound cases)
+    extras = None
+    if flush is not None:
+        n_rep = 50
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n_rep):
+            B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
+        b_.record()
+        torch.cuda.synchronize()
+        warm_us = 1e3 * a.elapsed_time(b_) / n_rep
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs, stream=side)
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(n_rep):
+            graph.replay()
+        b_.record()
+        torch.cuda.synchronize()
+        extras = {"warm_us_per_call": warm_us, "graph_replay_us_per_call": 1e3 * a.elapsed_time(b_) / n_rep,
+                  "note": "workload fits in L2: back-to-back calls without flush, and the same call replayed from a CUDA graph"}
+    barrier()
+
     # ---- end to end: host buffers in, host buffers out, through the C-ABI host entry point ----------
     u_h = torch.from_numpy(inp.u).pin_memory()
     w_h = torch.from_numpy(inp.kl_w).pin_memory()
@@ -302,7 +333,7 @@ def main():
                          "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": main_ms,
                          "traffic": cap["traffic"] if cap else None},
             "roofline_alu": alu,
-            "checksum_J": Jsum, "mean_J_all_ranks": Jmean,
+            "checksum_J": Jsum, "mean_J_all_ranks": Jmean, "l2_resident_extras": extras,
         }
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = oracle_sample_run(args.config, args.nu_mode)[0]
