@@ -89,71 +89,132 @@ __device__ __forceinline__ float cos_node(int i, int ix, int nm1) {
 }
 
 constexpr int KLF_THREADS = 128;
-constexpr int KLF_ROWS = 16;
-constexpr int KLF_M = DN_MAX_KL_MODES;
+constexpr int KLF_LINES = 64;                           // grid lines (fixed y, z) per block
 
-template <int VEC>
+typedef unsigned long long klf_u64;
+__device__ __forceinline__ klf_u64 klf_pack2(float lo, float hi) {
+    klf_u64 v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void klf_unpack2(klf_u64 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ klf_u64 klf_fma2(klf_u64 a, klf_u64 b, klf_u64 c) {
+    klf_u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float klf_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// A block owns up to KLF_LINES consecutive grid lines (y, z flattened) and a strip of 4 * KLF_THREADS
+// nodes in x.  Along a line the exponent is a polynomial of degree m in c = cos(pi x) (cos(i pi x) =
+// T_i(c)); its coefficients are prepared per line in double and stored, duplicated, in shared memory,
+// so a pair of nodes costs m packed FMAs, two ex2 and half a 128-bit store: the kernel is write-bound.
+template <int M, int VEC>
 __global__ void __launch_bounds__(KLF_THREADS)
-kl_field_kernel(int dim, int nx, int ny, int nz, int m, const float* __restrict__ kl_w, float* __restrict__ nu) {
-    __shared__ float cy[KLF_ROWS][KLF_M];
-    __shared__ float cz[KLF_M];
-    __shared__ float g[KLF_ROWS][KLF_M];
+kl_field_kernel(int dim, int nx, int ny, int nz, const float* __restrict__ kl_w, float* __restrict__ nu) {
+    constexpr int GS = (2 * (M + 1) + 3) / 4 * 4;       // floats per line: (g_k, g_k) pairs, padded
+    __shared__ __align__(16) float gam[KLF_LINES][GS];
     const int b = blockIdx.z;
-    const int rows_y = (ny + KLF_ROWS - 1) / KLF_ROWS;
-    const int iz = blockIdx.x / rows_y;
-    const int y0 = (blockIdx.x % rows_y) * KLF_ROWS;
+    const long long nlines = (long long)ny * nz;
+    const long long l0 = (long long)blockIdx.x * KLF_LINES;
     const int tid = threadIdx.x;
-    long long mpow = (long long)m * m * (dim == 3 ? m : 1);
-    const float* w = kl_w + (long long)b * mpow;
-    if (tid < KLF_ROWS * m) {
-        const int row = tid / m, j = tid % m + 1;
-        const int iy = min(y0 + row, ny - 1);
-        cy[row][j - 1] = cos_node(j, iy, ny - 1);
-    }
-    if (tid < m) cz[tid] = (dim == 3) ? cos_node(tid + 1, iz, nz - 1) : 1.0f;
-    __syncthreads();
-    if (tid < KLF_ROWS * m) {
-        const int row = tid / m, i = tid % m + 1;
-        float acc = 0.0f;
-        for (int j = 1; j <= m; ++j) {
-            float inner = 0.0f;
-            if (dim == 3) {
-                for (int k = 1; k <= m; ++k)
-                    inner = fmaf(w[((i - 1) * m + (j - 1)) * m + (k - 1)] *
-                                     (float)(kLog2e / (1.0 + i * i + j * j + k * k)), cz[k - 1], inner);
-            } else {
-                inner = w[(i - 1) * m + (j - 1)] * (float)(kLog2e / (1.0 + i * i + j * j));
-            }
-            acc = fmaf(inner, cy[row][j - 1], acc);
+    const float* w = kl_w + (long long)b * M * M * (dim == 3 ? M : 1);
+    if (tid < KLF_LINES && l0 + tid < nlines) {
+        const long long l = l0 + tid;
+        const int iy = (int)(l % ny), iz = (int)(l / ny);
+        double cy[M], cz[M], g[M];
+#pragma unroll
+        for (int j = 0; j < M; ++j) {
+            cy[j] = (double)cos_node(j + 1, iy, ny - 1);
+            cz[j] = (dim == 3) ? (double)cos_node(j + 1, iz, nz - 1) : 1.0;
         }
-        g[row][i - 1] = acc;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            double acc = 0.0;
+#pragma unroll
+            for (int j = 0; j < M; ++j) {
+                double inner;
+                if (dim == 3) {
+                    inner = 0.0;
+#pragma unroll
+                    for (int k = 0; k < M; ++k)
+                        inner += (double)w[(i * M + j) * M + k] / (1.0 + (i + 1) * (i + 1) + (j + 1) * (j + 1) + (k + 1) * (k + 1)) * cz[k];
+                } else {
+                    inner = (double)w[i * M + j] / (1.0 + (i + 1) * (i + 1) + (j + 1) * (j + 1));
+                }
+                acc += inner * cy[j];
+            }
+            g[i] = acc * kLog2e;
+        }
+        // sum_i g_i T_i(c) in the monomial basis, T_{i+1} = 2 c T_i - T_{i-1}
+        double acc[M + 1], tp[M + 1], tc[M + 1];
+#pragma unroll
+        for (int k = 0; k <= M; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
+#pragma unroll
+        for (int i = 1; i <= M; ++i) {
+#pragma unroll
+            for (int k = 0; k <= M; ++k) acc[k] += g[i - 1] * tc[k];
+            double tn[M + 1];
+#pragma unroll
+            for (int k = 0; k <= M; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
+#pragma unroll
+            for (int k = 0; k <= M; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
+        }
+#pragma unroll
+        for (int k = 0; k <= M; ++k) { gam[tid][2 * k] = (float)acc[k]; gam[tid][2 * k + 1] = (float)acc[k]; }
     }
     __syncthreads();
     const int x0 = (blockIdx.y * KLF_THREADS + tid) * VEC;
     if (x0 >= nx) return;
-    float cx[KLF_M][VEC];
-    for (int i = 0; i < m; ++i)
+    float c[4];
 #pragma unroll
-        for (int v = 0; v < VEC; ++v) cx[i][v] = cos_node(i + 1, min(x0 + v, nx - 1), nx - 1);
-    for (int row = 0; row < KLF_ROWS; ++row) {
-        const int iy = y0 + row;
-        if (iy >= ny) break;
-        float e[VEC];
+    for (int v = 0; v < 4; ++v) c[v] = cos_node(1, min(x0 + v, nx - 1), nx - 1);
+    const klf_u64 c01 = klf_pack2(c[0], c[1]), c23 = klf_pack2(c[2], c[3]);
+    float* out = nu + (long long)b * nlines * nx + l0 * nx + x0;
+    const int lines = (int)min((long long)KLF_LINES, nlines - l0);
+    for (int row = 0; row < lines; ++row) {
+        klf_u64 g2[GS / 2];
+        const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(&gam[row][0]);
 #pragma unroll
-        for (int v = 0; v < VEC; ++v) e[v] = 0.0f;
-        for (int i = 0; i < m; ++i) {
-            const float gi = g[row][i];
+        for (int k = 0; k < GS / 4; ++k) { const ulonglong2 t = gp[k]; g2[2 * k] = t.x; g2[2 * k + 1] = t.y; }
+        klf_u64 e01 = g2[M], e23 = g2[M];
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) e[v] = fmaf(cx[i][v], gi, e[v]);
-        }
-        float* out = nu + (((long long)b * nz + iz) * ny + iy) * nx + x0;
+        for (int k = M - 1; k >= 0; --k) { e01 = klf_fma2(e01, c01, g2[k]); if (VEC == 4) e23 = klf_fma2(e23, c23, g2[k]); }
+        float e0, e1, e2, e3;
+        klf_unpack2(e01, e0, e1);
+        klf_unpack2(e23, e2, e3);
         if (VEC == 4) {
-            float4 o = make_float4(exp2f(e[0]), exp2f(e[1]), exp2f(e[2]), exp2f(e[3]));
-            *reinterpret_cast<float4*>(out) = o;
+            *reinterpret_cast<float4*>(out) = make_float4(klf_ex2(e0), klf_ex2(e1), klf_ex2(e2), klf_ex2(e3));
         } else {
-            out[0] = exp2f(e[0]);
+            out[0] = klf_ex2(e0);
         }
+        out += nx;
     }
+}
+
+template <int VEC>
+cudaError_t launch_kl_field_vec(const dn_grid& g, int nz, int batch, int m, const float* kl_w, float* nu, cudaStream_t s) {
+    const int per_block = KLF_THREADS * VEC;
+    const long long nlines = (long long)g.ny * nz;
+    dim3 grid((unsigned)((nlines + KLF_LINES - 1) / KLF_LINES), (g.nx + per_block - 1) / per_block, batch);
+    switch (m) {
+        case 1: kl_field_kernel<1, VEC><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, kl_w, nu); break;
+        case 2: kl_field_kernel<2, VEC><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, kl_w, nu); break;
+        case 3: kl_field_kernel<3, VEC><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, kl_w, nu); break;
+        case 4: kl_field_kernel<4, VEC><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, kl_w, nu); break;
+        case 5: kl_field_kernel<5, VEC><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, kl_w, nu); break;
+        case 6: kl_field_kernel<6, VEC><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, kl_w, nu); break;
+        case 7: kl_field_kernel<7, VEC><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, kl_w, nu); break;
+        case 8: kl_field_kernel<8, VEC><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, kl_w, nu); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
 }
 
 __global__ void apply_bc_kernel(long long lines, int nx, float v0, float v1, float* __restrict__ field) {
@@ -189,11 +250,7 @@ cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* 
 cudaError_t launch_kl_field(const dn_grid& g, int batch, int m, const float* kl_w, float* nu, cudaStream_t s) {
     const int nz = (g.dim == 3) ? g.nz : 1;
     const bool vec = (g.nx % 4 == 0) && ((reinterpret_cast<uintptr_t>(nu) & 15u) == 0);
-    const int per_block = KLF_THREADS * (vec ? 4 : 1);
-    dim3 grid(((g.ny + KLF_ROWS - 1) / KLF_ROWS) * nz, (g.nx + per_block - 1) / per_block, batch);
-    if (vec) kl_field_kernel<4><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, m, kl_w, nu);
-    else kl_field_kernel<1><<<grid, KLF_THREADS, 0, s>>>(g.dim, g.nx, g.ny, nz, m, kl_w, nu);
-    return cudaGetLastError();
+    return vec ? launch_kl_field_vec<4>(g, nz, batch, m, kl_w, nu, s) : launch_kl_field_vec<1>(g, nz, batch, m, kl_w, nu, s);
 }
 
 cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int mode, float* field, cudaStream_t s) {
