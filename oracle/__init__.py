@@ -29,6 +29,7 @@ _LIB = os.path.join(_HERE, "libdn_oracle.so")
 
 NU_NODAL = 0
 NU_KL_GAUSS = 1
+NU_KL_NODAL = 2
 IMPOSE_BC_ON_LOAD = 1
 NO_MASK = 2
 

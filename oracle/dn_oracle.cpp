@@ -25,7 +25,8 @@
 //              mode 1: the KL expansion
 //                 nu(x) = exp( sum_{i,j(,k)=1..m} w_ij(k) cos(i pi x) cos(j pi y)
 //                              (cos(k pi z)) / (1 + i^2 + j^2 (+ k^2)) )
-//              evaluated at the physical Gauss point.
+//              evaluated at the physical Gauss point;
+//              mode 2: the same KL expansion evaluated at the nodes (in double), then Q1 interpolation.
 //
 // Inputs are the same fp32 arrays the GPU gets, promoted to double on read.
 // Arrays are C-ordered [B][nz][ny][nx], x fastest.
@@ -47,7 +48,7 @@
 
 extern "C" {
 
-enum { ORC_NU_NODAL = 0, ORC_NU_KL_GAUSS = 1 };
+enum { ORC_NU_NODAL = 0, ORC_NU_KL_GAUSS = 1, ORC_NU_KL_NODAL = 2 };
 enum { ORC_IMPOSE_BC_ON_LOAD = 1u, ORC_NO_MASK = 2u };
 
 struct orc_problem {
@@ -166,6 +167,8 @@ void element(const orc_problem& p, const Geo& g, const Rule& rule, int b, const 
         const long idx = node_index(g, ix, iy, iz);
         uc[a] = u ? u_at(p, g, u, b, ix, iy, iz) : 0.0;
         nuc[a] = (p.nu_mode == ORC_NU_NODAL) ? (double)p.nu[(size_t)b * g.nodes + idx] : 0.0;
+        if (p.nu_mode == ORC_NU_KL_NODAL)
+            nuc[a] = kl_nu(p, b, ix * g.h[0], iy * g.h[1], (g.dim == 3) ? iz * g.h[2] : 0.0);
         fc[a] = p.f ? (double)p.f[(size_t)b * g.nodes + idx] : p.f_const;
     }
     Jdiff = 0.0; Jload = 0.0;
@@ -212,8 +215,8 @@ bool valid(const orc_problem& p) {
     if (p.nx < 2 || p.ny < 2 || (p.dim == 3 && p.nz < 2) || p.batch < 1) return false;
     if (p.nquad != 2 && p.nquad != 3) return false;
     if (p.nu_mode == ORC_NU_NODAL && !p.nu) return false;
-    if (p.nu_mode == ORC_NU_KL_GAUSS && (!p.kl_w || p.kl_modes < 1)) return false;
-    if (p.nu_mode != ORC_NU_NODAL && p.nu_mode != ORC_NU_KL_GAUSS) return false;
+    if ((p.nu_mode == ORC_NU_KL_GAUSS || p.nu_mode == ORC_NU_KL_NODAL) && (!p.kl_w || p.kl_modes < 1)) return false;
+    if (p.nu_mode != ORC_NU_NODAL && p.nu_mode != ORC_NU_KL_GAUSS && p.nu_mode != ORC_NU_KL_NODAL) return false;
     return true;
 }
 

@@ -10,7 +10,7 @@ import numpy as np
 import pytest
 
 import oracle
-from oracle import Problem, NU_NODAL, NU_KL_GAUSS, NO_MASK, IMPOSE_BC_ON_LOAD
+from oracle import Problem, NU_NODAL, NU_KL_GAUSS, NU_KL_NODAL, NO_MASK, IMPOSE_BC_ON_LOAD
 from paper_2007_12792_b200 import inputs
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
@@ -141,7 +141,7 @@ def _problem(dim, nx, ny, nz, mode, batch=1, m=2, f_const=0.7, seed=5):
     return p
 
 
-@pytest.mark.parametrize("mode", [NU_NODAL, NU_KL_GAUSS])
+@pytest.mark.parametrize("mode", [NU_NODAL, NU_KL_GAUSS, NU_KL_NODAL])
 @pytest.mark.parametrize("dim,nx,ny,nz", [(2, 8, 8, 1), (3, 5, 5, 5), (2, 7, 5, 1)])
 def test_quadratic_in_t_and_finite_differences(mode, dim, nx, ny, nz):
     p = _problem(dim, nx, ny, nz, mode)
@@ -167,7 +167,7 @@ def test_quadratic_in_t_and_finite_differences(mode, dim, nx, ny, nz):
 
 
 # ---- P5: residual vanishes at the discrete solution -------------------------------------------
-@pytest.mark.parametrize("mode", [NU_NODAL, NU_KL_GAUSS])
+@pytest.mark.parametrize("mode", [NU_NODAL, NU_KL_GAUSS, NU_KL_NODAL])
 @pytest.mark.parametrize("dim,nx,ny,nz", [(2, 6, 6, 1), (2, 9, 5, 1), (3, 4, 4, 4), (3, 5, 4, 3)])
 def test_residual_zero_at_direct_solution(mode, dim, nx, ny, nz):
     p = _problem(dim, nx, ny, nz, mode, f_const=1.0)
@@ -190,7 +190,7 @@ def test_residual_zero_at_direct_solution(mode, dim, nx, ny, nz):
 
 
 # ---- P7 / P8 / P12: partition of unity, Euler identity, symmetry ------------------------------
-@pytest.mark.parametrize("mode", [NU_NODAL, NU_KL_GAUSS])
+@pytest.mark.parametrize("mode", [NU_NODAL, NU_KL_GAUSS, NU_KL_NODAL])
 @pytest.mark.parametrize("dim,nx,ny,nz", GRIDS)
 def test_partition_of_unity_euler_symmetry(mode, dim, nx, ny, nz):
     p = _problem(dim, nx, ny, nz, mode, batch=2, f_const=0.9)
@@ -288,6 +288,31 @@ def test_kl_field_closed_forms():
                  * np.cos(3 * np.pi * z)[:, None, None] / 15.0)
     out = oracle.kl_field(3, nx, ny, nz, 2, 3, w3)
     assert np.all(out[0] == 1.0) and np.allclose(out[1], ref, rtol=1e-14)
+
+
+def test_kl_nodal_mode_closed_form_and_equivalence():
+    """KL evaluated at the nodes, then Q1-interpolated: for u = 1 - x the energy is the trapezoid sum of the
+    typed-out KL formula at the nodes; for general u it equals nodal mode fed with that field."""
+    for dim, nx, ny, nz in GRIDS:
+        w = inputs.draw_weights(np.random.default_rng(21), dim, 2)[None]
+        wd = w[0].astype(np.float64)
+        ax = [np.arange(n) / (n - 1) for n in (nx, ny, nz)]
+        if dim == 2:
+            e = sum(wd[i - 1, j - 1] * np.cos(i * np.pi * ax[0])[None, :] * np.cos(j * np.pi * ax[1])[:, None] / (1 + i * i + j * j)
+                    for i in (1, 2) for j in (1, 2))
+        else:
+            e = sum(wd[i - 1, j - 1, k - 1] * np.cos(i * np.pi * ax[0])[None, None, :] * np.cos(j * np.pi * ax[1])[None, :, None]
+                    * np.cos(k * np.pi * ax[2])[:, None, None] / (1 + i * i + j * j + k * k) for i in (1, 2) for j in (1, 2) for k in (1, 2))
+        nu = np.exp(e)
+        p = Problem(dim=dim, nx=nx, ny=ny, nz=nz, batch=1, nu_mode=NU_KL_NODAL, kl_modes=2, kl_w=w, f_const=0.4)
+        J = oracle.energy_grad(p, lin_profile(p.shape), want_r=False)
+        tw = trapezoid_weights(dim, nx, ny, nz)
+        assert J[1][0] == pytest.approx(0.5 * (tw * nu).sum(), rel=1e-13)            # diffusion part
+        q = Problem(dim=dim, nx=nx, ny=ny, nz=nz, batch=1, nu_mode=NU_NODAL, nu=nu[None].astype(np.float32), f_const=0.4)
+        u = RNG.standard_normal(p.shape)
+        a = oracle.energy_grad(p, u); b = oracle.energy_grad(q, u)
+        assert a[0][0] == pytest.approx(b[0][0], rel=1e-6)
+        assert np.abs(a[3] - b[3]).max() < 1e-6 * np.abs(b[3]).max()
 
 
 def test_kl_gauss_mode_zero_weights_equals_unit_nodal():
