@@ -55,7 +55,9 @@ typedef enum {
 
 typedef enum {
     DN_NU_NODAL = 0,       /* nu given at the nodes, Q1-interpolated to the Gauss points    */
-    DN_NU_KL_GAUSS = 1     /* nu evaluated from the KL weights at the Gauss points; no field stored */
+    DN_NU_KL_GAUSS = 1,    /* nu evaluated from the KL weights at the Gauss points; no field stored */
+    DN_NU_KL_NODAL = 2     /* nu evaluated from the KL weights at the nodes inside the kernel, then Q1-interpolated
+                              (the numbers of dn_kl_field + DN_NU_NODAL, without storing the field)          */
 } dn_nu_mode;
 
 /* dn_problem.flags */
@@ -79,7 +81,7 @@ typedef struct {
     int32_t batch;               /* B >= 1                                                         */
     int32_t nu_mode;             /* dn_nu_mode                                                     */
     const float* nu;             /* [B][nz][ny][nx], used when nu_mode == DN_NU_NODAL              */
-    int32_t kl_modes;            /* m, used when nu_mode == DN_NU_KL_GAUSS                         */
+    int32_t kl_modes;            /* m, used when nu_mode is DN_NU_KL_GAUSS or DN_NU_KL_NODAL       */
     const float* kl_w;           /* [B][m]^dim, index [b][i-1][j-1]([k-1]); i <-> x, j <-> y, k <-> z */
     float f_const;               /* forcing when f == NULL                                         */
     const float* f;              /* optional nodal forcing [B][nz][ny][nx], Q1-interpolated        */

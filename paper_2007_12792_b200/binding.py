@@ -22,6 +22,7 @@ DN_OK = 0
 DN_ERR_NULL, DN_ERR_DIM, DN_ERR_SIZE, DN_ERR_MODE, DN_ERR_WORKSPACE, DN_ERR_CUDA, DN_ERR_ALIAS = range(1, 8)
 DN_NU_NODAL = 0
 DN_NU_KL_GAUSS = 1
+DN_NU_KL_NODAL = 2
 DN_IMPOSE_BC_ON_LOAD = 1
 DN_NO_MASK = 2
 DN_FORCE_GENERIC = 4

@@ -23,7 +23,7 @@ static dn_status validate(const dn_problem* p) {
     if (p->batch < 1 || p->batch > 65535) return DN_ERR_SIZE;
     if (p->nu_mode == DN_NU_NODAL) {
         if (!p->nu) return DN_ERR_NULL;
-    } else if (p->nu_mode == DN_NU_KL_GAUSS) {
+    } else if (p->nu_mode == DN_NU_KL_GAUSS || p->nu_mode == DN_NU_KL_NODAL) {
         if (p->kl_modes < 1 || p->kl_modes > DN_MAX_KL_MODES) return DN_ERR_MODE;
         if (!p->kl_w) return DN_ERR_NULL;
     } else {
@@ -62,7 +62,7 @@ static int max_nblk(const dn_problem& p) {
 WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
     WsLayout w{};
     const int dim = p.grid.dim;
-    const int m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
+    const int m = (p.nu_mode != DN_NU_NODAL) ? p.kl_modes : 0;
     w.nblk = l.nblk;
     size_t off = 0;
     w.partials = off; off += align_up(sizeof(double) * 2 * (size_t)p.batch * (tight ? l.nblk : max_nblk(p)));
@@ -76,6 +76,11 @@ WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
         w.cg[a] = off;
         off += align_up(sizeof(float) * (size_t)m * w.gstride[a] + 16);
     }
+    for (int a = 0; a < 3; ++a) {
+        w.nstride[a] = (a < dim) ? (n[a] + 3) / 4 * 4 + 8 : 0;
+        w.cn[a] = off;
+        off += align_up(sizeof(float) * (size_t)m * w.nstride[a] + 16);
+    }
     w.seam = off;
     if ((tight ? l.path == PATH_TILED3D : tiled3d_applicable(p))) off += align_up(sizeof(float) * tiled3d_seam_floats(p) + 16);
     w.total = off;
@@ -85,7 +90,7 @@ WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
 static Params make_params(const dn_problem& p, const WsLayout& w, const float* u, const float* gJ, float* r, void* ws) {
     Params P{};
     P.dim = p.grid.dim; P.nx = p.grid.nx; P.ny = p.grid.ny; P.nz = (p.grid.dim == 3) ? p.grid.nz : 1;
-    P.batch = p.batch; P.nu_mode = p.nu_mode; P.m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
+    P.batch = p.batch; P.nu_mode = p.nu_mode; P.m = (p.nu_mode != DN_NU_NODAL) ? p.kl_modes : 0;
     P.flags = p.flags; P.f_const = p.f_const; P.bc_x0 = p.bc_x0; P.bc_x1 = p.bc_x1;
     P.hx = (float)(1.0 / (P.nx - 1)); P.hy = (float)(1.0 / (P.ny - 1));
     P.hz = (P.dim == 3) ? (float)(1.0 / (P.nz - 1)) : 1.0f;
@@ -94,6 +99,7 @@ static Params make_params(const dn_problem& p, const WsLayout& w, const float* u
     P.partials = reinterpret_cast<double*>(base + w.partials);
     P.ckl = reinterpret_cast<const float*>(base + w.ckl);
     for (int a = 0; a < 3; ++a) { P.cg[a] = reinterpret_cast<const float*>(base + w.cg[a]); P.gstride[a] = w.gstride[a]; }
+    for (int a = 0; a < 3; ++a) { P.cn[a] = reinterpret_cast<const float*>(base + w.cn[a]); P.nstride[a] = w.nstride[a]; }
     P.nblk = w.nblk;
     P.seam = reinterpret_cast<float*>(base + w.seam);
     P.nodes = nodes_per_sample(p.grid);
@@ -118,11 +124,13 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Params P = make_params(*p, w, u, gJ, r, ws);
     cudaError_t e = cudaSuccess;
-    if (p->nu_mode == DN_NU_KL_GAUSS) {
+    if (p->nu_mode != DN_NU_NODAL) {
         char* base = static_cast<char*>(ws);
         float* cg[3] = {reinterpret_cast<float*>(base + w.cg[0]), reinterpret_cast<float*>(base + w.cg[1]),
                         reinterpret_cast<float*>(base + w.cg[2])};
-        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, s);
+        float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
+                        reinterpret_cast<float*>(base + w.cn[2])};
+        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s);
         if (e != cudaSuccess) return DN_ERR_CUDA;
     }
     if (ev_before && cudaEventRecord(static_cast<cudaEvent_t>(ev_before), s) != cudaSuccess) return DN_ERR_CUDA;
@@ -165,7 +173,7 @@ size_t dn_host_staging_bytes(const dn_problem* p) {
     if (p->nu_mode == DN_NU_NODAL) total += field;
     if (p->f) total += field;
     size_t mpow = 1;
-    for (int a = 0; a < p->grid.dim; ++a) mpow *= (size_t)((p->nu_mode == DN_NU_KL_GAUSS) ? p->kl_modes : 0);
+    for (int a = 0; a < p->grid.dim; ++a) mpow *= (size_t)((p->nu_mode != DN_NU_NODAL) ? p->kl_modes : 0);
     total += align_up(sizeof(float) * (size_t)p->batch * mpow + 16);
     return total + dn_workspace_bytes(p);
 }
@@ -250,7 +258,7 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
     const size_t field = align_up(sizeof(float) * nfield);
     const size_t small = align_up(sizeof(float) * (size_t)p->batch);
     size_t mpow = 1;
-    for (int a = 0; a < p->grid.dim; ++a) mpow *= (size_t)((p->nu_mode == DN_NU_KL_GAUSS) ? p->kl_modes : 0);
+    for (int a = 0; a < p->grid.dim; ++a) mpow *= (size_t)((p->nu_mode != DN_NU_NODAL) ? p->kl_modes : 0);
     char* base = static_cast<char*>(staging);
     size_t off = 0;
     float* d_u = reinterpret_cast<float*>(base + off); off += field;
@@ -278,7 +286,7 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
     DN_TRY(cudaEventRecord(pipe.start, s));                       // the call is ordered after earlier work on `stream`
     DN_TRY(cudaStreamWaitEvent(pipe.in, pipe.start, 0));
     DN_TRY(cudaStreamWaitEvent(pipe.out, pipe.start, 0));
-    if (p->nu_mode == DN_NU_KL_GAUSS)
+    if (p->nu_mode != DN_NU_NODAL)
         DN_TRY(cudaMemcpyAsync(d_w, p->kl_w, sizeof(float) * (size_t)p->batch * mpow, cudaMemcpyHostToDevice, pipe.in));
     if (gJ_host) DN_TRY(cudaMemcpyAsync(d_g, gJ_host, sizeof(float) * p->batch, cudaMemcpyHostToDevice, pipe.in));
     for (int c = 0; c < nchunks; ++c) {
@@ -294,7 +302,7 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
         q.batch = nb;
         q.nu = d_nu ? d_nu + o : nullptr;
         q.f = d_f ? d_f + o : nullptr;
-        q.kl_w = (p->nu_mode == DN_NU_KL_GAUSS) ? d_w + (size_t)b0 * mpow : nullptr;
+        q.kl_w = (p->nu_mode != DN_NU_NODAL) ? d_w + (size_t)b0 * mpow : nullptr;
         st = run(&q, d_u + o, gJ_host ? d_g + b0 : nullptr, J_host ? d_J + b0 : nullptr, d_r + o, ws, ws_bytes, s);
         if (st != DN_OK) { cudaStreamSynchronize(pipe.in); cudaStreamSynchronize(s); cudaStreamSynchronize(pipe.out); return st; }
         DN_TRY(cudaEventRecord(pipe.computed[c], s));
@@ -312,7 +320,7 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
 int32_t dn_launches_per_call(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
     const bool t3 = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
-    return 2 + (p->nu_mode == DN_NU_KL_GAUSS ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
+    return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
 }
 
 const char* dn_path_name(const dn_problem* p) {

@@ -12,6 +12,7 @@ constexpr double kLog2e = 1.4426950408889634074;
 // Tables for the KL expansion evaluated at Gauss points (DN_NU_KL_GAUSS):
 //   ckl[b][i][j]([k]) = w * log2(e) / (1 + i^2 + j^2 (+ k^2))      so that nu = 2^(sum ckl cos cos (cos))
 //   cg[a][i-1][p]     = cos(i pi x_p),  x_p = (p/2 + (p odd ? GB : GA)) * h_a,  p < 2 (n_a - 1)
+//   cn[a][i-1][n]     = cos(i pi n h_a) at the nodes (DN_NU_KL_NODAL)
 // The cosines are evaluated in double (cospi) and rounded once.
 // ---------------------------------------------------------------------------------------
 struct TableArgs {
@@ -21,6 +22,8 @@ struct TableArgs {
     const float* kl_w;
     float* ckl;
     float* cg[3];
+    int nstride[3];
+    float* cn[3];
 };
 
 __global__ void tables_kernel(TableArgs A) {
@@ -51,6 +54,17 @@ __global__ void tables_kernel(TableArgs A) {
             if (p >= ng) p = ng - 1;                      // padding repeats the last abscissa
             const double x = ((double)(p >> 1) + ((p & 1) ? gb : ga)) / (double)(A.n[a] - 1);
             A.cg[a][idx] = (float)cospi((double)i * x);
+            return;
+        }
+        idx -= cnt;
+    }
+    for (int a = 0; a < A.dim; ++a) {
+        const long long cnt = (long long)m * A.nstride[a];
+        if (idx < cnt) {
+            const int i = (int)(idx / A.nstride[a]) + 1;
+            int n = (int)(idx % A.nstride[a]);
+            if (n >= A.n[a]) n = A.n[a] - 1;              // padding repeats the last node
+            A.cn[a][idx] = (float)cospi((double)i * (double)n / (double)(A.n[a] - 1));
             return;
         }
         idx -= cnt;
@@ -226,7 +240,8 @@ __global__ void apply_bc_kernel(long long lines, int nx, float v0, float v1, flo
 
 }  // namespace
 
-cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], cudaStream_t s) {
+cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], float* const cn[3],
+                          cudaStream_t s) {
     TableArgs A{};
     A.dim = P.dim; A.m = P.m; A.batch = P.batch;
     A.n[0] = P.nx; A.n[1] = P.ny; A.n[2] = P.nz;
@@ -234,7 +249,8 @@ cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float*
     for (int a = 0; a < P.dim; ++a) total *= P.m;
     for (int a = 0; a < 3; ++a) {
         A.gstride[a] = P.gstride[a]; A.cg[a] = cg[a];
-        if (a < P.dim) total += (long long)P.m * P.gstride[a];
+        A.nstride[a] = P.nstride[a]; A.cn[a] = cn[a];
+        if (a < P.dim) total += (long long)P.m * (P.gstride[a] + P.nstride[a]);
     }
     A.kl_w = kl_w; A.ckl = ckl;
     const int threads = 128;

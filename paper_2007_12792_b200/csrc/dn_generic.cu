@@ -40,6 +40,27 @@ __device__ __forceinline__ float kl_exponent(const Params& P, const float* c, in
     return e;
 }
 
+// KL diffusivity at the node with per-axis indices (ix, iy, iz)  (DN_NU_KL_NODAL).
+__device__ __forceinline__ float kl_node(const Params& P, const float* c, int ix, int iy, int iz) {
+    const int m = P.m;
+    float e = 0.0f;
+    for (int i = 0; i < m; ++i) {
+        float ei = 0.0f;
+        for (int j = 0; j < m; ++j) {
+            float ej;
+            if (P.dim == 3) {
+                ej = 0.0f;
+                for (int k = 0; k < m; ++k) ej = fmaf(c[(i * m + j) * m + k], P.cn[2][k * P.nstride[2] + iz], ej);
+            } else {
+                ej = c[i * m + j];
+            }
+            ei = fmaf(ej, P.cn[1][j * P.nstride[1] + iy], ei);
+        }
+        e = fmaf(ei, P.cn[0][i * P.nstride[0] + ix], e);
+    }
+    return exp2f(e);
+}
+
 // ----- 2D element: contributions to its four corners and its energy parts -------------------
 // Corner order (0,0), (1,0), (0,1), (1,1).  With e0 = u10-u00, s0 = u01-u00 and the twist
 // t = u11-u10-u01+u00, the x-derivative at the Gauss row eta is (e0 + eta t)/hx and the
@@ -54,9 +75,14 @@ __device__ __forceinline__ void element2d(const Params& P, int b, int ex, int ey
     const float u01 = load_u(P, ub, ex, i00 + nx), u11 = load_u(P, ub, ex + 1, i00 + nx + 1);
     const float ga[2] = {DN_GA, DN_GB};
     float nuq[2][2];                                   // [p: xi point][q: eta point]
-    if (P.nu_mode == DN_NU_NODAL) {
-        const float n00 = __ldg(nub + i00), n10 = __ldg(nub + i00 + 1);
-        const float n01 = __ldg(nub + i00 + nx), n11 = __ldg(nub + i00 + nx + 1);
+    if (P.nu_mode != DN_NU_KL_GAUSS) {
+        float n00, n10, n01, n11;
+        if (P.nu_mode == DN_NU_NODAL) {
+            n00 = __ldg(nub + i00); n10 = __ldg(nub + i00 + 1); n01 = __ldg(nub + i00 + nx); n11 = __ldg(nub + i00 + nx + 1);
+        } else {
+            n00 = kl_node(P, c, ex, ey, 0); n10 = kl_node(P, c, ex + 1, ey, 0);
+            n01 = kl_node(P, c, ex, ey + 1, 0); n11 = kl_node(P, c, ex + 1, ey + 1, 0);
+        }
         for (int p = 0; p < 2; ++p)
             for (int q = 0; q < 2; ++q) {
                 const float lo = n00 + ga[p] * (n10 - n00), hi = n01 + ga[p] * (n11 - n01);
@@ -116,9 +142,11 @@ __device__ __forceinline__ void element3d(const Params& P, int b, int ex, int ey
     const float ga[2] = {DN_GA, DN_GB};
     const float L[2][2] = {{1.f - DN_GA, DN_GA}, {1.f - DN_GB, DN_GB}};   // L[point][corner bit]
     float nuq[2][2][2];                                                     // [p: xi][q: eta][s: zeta]
-    if (P.nu_mode == DN_NU_NODAL) {
+    if (P.nu_mode != DN_NU_KL_GAUSS) {
         float nn[8];
-        for (int a = 0; a < 8; ++a) nn[a] = __ldg(nub + i0 + (a & 1) + ((a >> 1) & 1) * sy + ((a >> 2) & 1) * sz);
+        for (int a = 0; a < 8; ++a)
+            nn[a] = (P.nu_mode == DN_NU_NODAL) ? __ldg(nub + i0 + (a & 1) + ((a >> 1) & 1) * sy + ((a >> 2) & 1) * sz)
+                                               : kl_node(P, c, ex + (a & 1), ey + ((a >> 1) & 1), ez + ((a >> 2) & 1));
         for (int p = 0; p < 2; ++p)
             for (int q = 0; q < 2; ++q)
                 for (int s = 0; s < 2; ++s) {

@@ -26,6 +26,8 @@ struct WsLayout {
     size_t cg[3];         // float  [m][gstride[a]] cos(i pi x) at the Gauss abscissae of axis a
     size_t seam;          // float  [B][nseam][nz][nx] contributions across tile seams (tiled 3D kernel)
     int gstride[3];       // padded row length of cg[a] (multiple of 4)
+    size_t cn[3];         // float  [m][nstride[a]] cos(i pi x) at the nodes of axis a
+    int nstride[3];
     int nblk;             // energy partials per sample
     size_t total;
 };
@@ -46,6 +48,8 @@ struct Params {
     const float* ckl;
     const float* cg[3];
     int gstride[3];
+    const float* cn[3];   // cosines at the nodes (KL-at-nodes mode)
+    int nstride[3];
     int nblk;
     long long nodes;      // per sample
     float* seam;          // tiled 3D: contributions of a tile's top element row to the next tile's first node row
@@ -65,7 +69,8 @@ WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight = false);
 dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
                     size_t ws_bytes, void* stream);
 
-cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], cudaStream_t s);
+cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], float* const cn[3],
+                          cudaStream_t s);
 cudaError_t launch_generic(const Params& P, cudaStream_t s);
 cudaError_t launch_tiled2d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s);

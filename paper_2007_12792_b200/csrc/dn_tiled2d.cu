@@ -559,7 +559,7 @@ cudaError_t launch_k(const Params& P, const Geo2& g, cudaStream_t s) {
 }  // namespace
 
 bool tiled2d_applicable(const dn_problem& p) {
-    return p.grid.dim == 2 && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 128 * 2 * T2_MAX_WARPS &&
+    return p.grid.dim == 2 && p.nu_mode != DN_NU_KL_NODAL && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 128 * 2 * T2_MAX_WARPS &&
            p.grid.ny >= 2;
 }
 

@@ -635,7 +635,7 @@ cudaError_t launch_m(const Params& P, const Geo3& g, cudaStream_t s) {
 }  // namespace
 
 bool tiled3d_applicable(const dn_problem& p) {
-    return p.grid.dim == 3 && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 512 &&
+    return p.grid.dim == 3 && p.nu_mode != DN_NU_KL_NODAL && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 512 &&
            p.grid.ny >= 2 && p.grid.nz >= 2;
 }
 

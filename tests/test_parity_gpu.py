@@ -10,7 +10,7 @@ from parity_util import dev, make_problems, run_gpu, check, J_RTOL, R_RTOL
 
 pytestmark = pytest.mark.gpu
 
-MODES = [B.DN_NU_KL_GAUSS, B.DN_NU_NODAL]
+MODES = [B.DN_NU_KL_GAUSS, B.DN_NU_NODAL, B.DN_NU_KL_NODAL]
 
 
 def nodal_nu(inp):
