@@ -117,7 +117,7 @@ def oracle_sample_run(cfg: int, mode: str, target_seconds: float = 12.0):
     """Times the oracle (as it stands) on a bounded sample of the workload: whole samples of the batch."""
     import oracle
     wl = inputs.WORKLOADS[cfg]
-    nu_mode = oracle.NU_KL_GAUSS if mode == "kl" else oracle.NU_NODAL
+    nu_mode = {"kl": oracle.NU_KL_GAUSS, "nodal": oracle.NU_NODAL, "klnodal": oracle.NU_KL_NODAL}[mode]
 
     def run(samples):
         inp = inputs.make_inputs(cfg, samples=samples)
@@ -169,7 +169,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (default: 2D 2048^2, batch 16)")
-    ap.add_argument("--nu-mode", default="kl", choices=["kl", "nodal"])
+    ap.add_argument("--nu-mode", default="kl", choices=["kl", "nodal", "klnodal"],
+                    help="kl: KL at Gauss points (default); nodal: stored nodal field; klnodal: KL at nodes inside the kernel")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -198,7 +199,7 @@ def main():
     u = torch.from_numpy(inp.u).cuda()
     w = torch.from_numpy(inp.kl_w).cuda()
     nu = None
-    mode = B.DN_NU_KL_GAUSS if args.nu_mode == "kl" else B.DN_NU_NODAL
+    mode = {"kl": B.DN_NU_KL_GAUSS, "nodal": B.DN_NU_NODAL, "klnodal": B.DN_NU_KL_NODAL}[args.nu_mode]
     if mode == B.DN_NU_NODAL:
         nu = torch.empty_like(u)
         B.dn_kl_field(inp.dim, inp.nx, inp.ny, inp.nz, inp.batch, inp.kl_modes, w, nu)
@@ -329,7 +330,7 @@ def main():
         peak, peak_kind = measured_peak()
         elements = wl.elements * inp.batch
         nodes = wl.nodes * inp.batch
-        alg_bytes = nodes * (8 if mode == B.DN_NU_KL_GAUSS else 12)
+        alg_bytes = nodes * (12 if mode == B.DN_NU_NODAL else 8)
         achieved = alg_bytes / (main_ms * 1e-3) / 1e9
         path = B.dn_path_name(prob)
         key = f"{path}:{wl.name}:{args.nu_mode}"

@@ -86,14 +86,16 @@ template <int M> struct GamStride { static constexpr int value = (2 * (M + 1) + 
 
 template <int NE> struct Row { float v[NE]; float halo; };
 
-template <int K, int M, bool WANT_R, bool FULL, bool RING>
+template <int K, int M, bool WANT_R, bool FULL, bool RING, bool KN>
 __global__ void __launch_bounds__(256, 2)
 tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
     extern __shared__ __align__(16) float smem[];
-    constexpr bool KL = (M > 0);
+    constexpr bool HASM = (M > 0);                      // KL weights in play (either KL mode)
+    constexpr bool KL = HASM && !KN;                    // nu evaluated at the Gauss points
+    constexpr bool NLOAD = !HASM;                       // nu rows loaded from a nodal field
     constexpr int NE = 4 * K;
-    constexpr int GS = GamStride<KL ? M : 1>::value;
-    constexpr int MM = KL ? M : 1;
+    constexpr int GS = GamStride<HASM ? M : 1>::value;
+    constexpr int MM = HASM ? M : 1;
     const int lane = threadIdx.x & 31;
     const int wid = threadIdx.x >> 5;
     const int wx = wid % W, wy = wid / W;
@@ -105,13 +107,13 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
     const int n1 = min(n0 + R, ny);
     const int jbeg = max(n0 - 1, 0);
     const int jend = min(n1 - 1, ny - 2);          // last element row of this chunk (inclusive)
-    const int gam_rows = R + 1;
+    const int gam_rows = R + 2;                         // element rows (Gauss mode) or node rows (KL at nodes) of a chunk
     float* gam = smem + (size_t)wy * gam_rows * GS;
-    float* xch = smem + (size_t)WY * gam_rows * (KL ? GS : 0) + (size_t)wy * 2 * T2_MAX_WARPS * 2;
+    float* xch = smem + (size_t)WY * gam_rows * (HASM ? GS : 0) + (size_t)wy * 2 * T2_MAX_WARPS * 2;
     // ring of T2_STAGES node rows per warp row (u, and nu in nodal mode): per lane NE floats, then one halo per warp
-    constexpr int NARR = KL ? 1 : 2;
+    constexpr int NARR = NLOAD ? 2 : 1;
     const int ring_row = 32 * W * NE + 4 * ((W + 3) / 4);                      // floats per (stage, array)
-    float* ring = smem + (size_t)WY * gam_rows * (KL ? GS : 0) + (size_t)WY * 2 * T2_MAX_WARPS * 2 +
+    float* ring = smem + (size_t)WY * gam_rows * (HASM ? GS : 0) + (size_t)WY * 2 * T2_MAX_WARPS * 2 +
                   (size_t)wy * T2_STAGES * NARR * ring_row;
 
     // ---- prologue: polynomial coefficients of the KL exponent for the Gauss rows of the chunk
@@ -147,6 +149,38 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             for (int k = 0; k <= M; ++k) dst[2 * k] = (float)acc[k];
         }
     }
+    // KL at the nodes: the same polynomial per NODE row, stored as (g_k, g_k) pairs for two-wide evaluation
+    if constexpr (KN) if (!idle) {
+        const int count = jend - jbeg + 2;              // node rows jbeg .. jend+1
+        const float* c = P.ckl + (size_t)b * M * M;
+        for (int q = wx * 32 + lane; q < count; q += 32 * W) {
+            const int iy = jbeg + q;
+            double g[MM];
+#pragma unroll
+            for (int i = 0; i < M; ++i) {
+                double a = 0.0;
+#pragma unroll
+                for (int j = 0; j < M; ++j) a += (double)c[i * M + j] * (double)P.cn[1][j * P.nstride[1] + iy];
+                g[i] = a;
+            }
+            double acc[MM + 1], tp[MM + 1], tc[MM + 1];
+#pragma unroll
+            for (int k = 0; k <= M; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
+#pragma unroll
+            for (int i = 1; i <= M; ++i) {
+#pragma unroll
+                for (int k = 0; k <= M; ++k) acc[k] += g[i - 1] * tc[k];
+                double tn[MM + 1];
+#pragma unroll
+                for (int k = 0; k <= M; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
+#pragma unroll
+                for (int k = 0; k <= M; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
+            }
+            float* dst = gam + (size_t)q * GS;
+#pragma unroll
+            for (int k = 0; k <= M; ++k) { dst[2 * k] = (float)acc[k]; dst[2 * k + 1] = (float)acc[k]; }
+        }
+    }
     __syncthreads();
 
     float en = 0.f, ell = 0.f;
@@ -156,7 +190,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
         const int xhalo = x0 + NE;                      // node right of this lane's nodes
         const bool warp_has_halo = (wx * 32 + 32) * NE < nx;
         const float* ub = P.u + (size_t)b * P.nodes;
-        const float* nub = KL ? nullptr : P.nu + (size_t)b * P.nodes;
+        const float* nub = NLOAD ? P.nu + (size_t)b * P.nodes : nullptr;
         float* rb = WANT_R ? P.r + (size_t)b * P.nodes : nullptr;
         const bool impose = (P.flags & DN_IMPOSE_BC_ON_LOAD) != 0;
         const bool nomask = (P.flags & DN_NO_MASK) != 0;
@@ -233,6 +267,9 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
                 }
             }
         };
+        auto right_nb_nu = [&](const Row<NE>& r) {      // KL at nodes: every lane computed its own right neighbour
+            return r.halo;
+        };
         auto right_nb = [&](const Row<NE>& r) {
             const float rn = __shfl_down_sync(0xffffffffu, r.v[0], 1);
             return (lane == 31) ? r.halo : rn;
@@ -255,6 +292,40 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             }
         }
 
+        // KL at the nodes: cos(pi x) at this lane's nodes (pairs) and at the node right of them
+        u64 cnp[NE / 2];
+        float cnh = 0.f;
+        if constexpr (KN) {
+#pragma unroll
+            for (int s = 0; s < K; ++s) {
+                float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (act[s]) q = __ldg(reinterpret_cast<const float4*>(P.cn[0] + x0 + 4 * s));
+                cnp[2 * s] = pack2(q.x, q.y); cnp[2 * s + 1] = pack2(q.z, q.w);
+            }
+            if (x0 + NE < nx) cnh = __ldg(P.cn[0] + x0 + NE);
+        }
+        // nu on node row `row`, evaluated from the row's polynomial (values of this lane and of the node right of it)
+        auto nu_row = [&](Row<NE>& r, int row) {
+            const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(gam + (size_t)(row - jbeg) * GS);
+            u64 gg[GS / 2];
+#pragma unroll
+            for (int k = 0; k < GS / 4; ++k) { const ulonglong2 t = gp[k]; gg[2 * k] = t.x; gg[2 * k + 1] = t.y; }
+            float gh, dmy;
+            unpack2(gg[MM], gh, dmy);
+#pragma unroll
+            for (int i = 0; i < NE / 2; ++i) {
+                u64 e = gg[MM];
+#pragma unroll
+                for (int m = MM - 1; m >= 0; --m) e = fma2(e, cnp[i], gg[m]);
+                float e0, e1;
+                unpack2(e, e0, e1);
+                r.v[2 * i] = ex2_approx(e0); r.v[2 * i + 1] = ex2_approx(e1);
+            }
+#pragma unroll
+            for (int m = MM - 1; m >= 0; --m) { float gm; unpack2(gg[m], gm, dmy); gh = fmaf(gh, cnh, gm); }
+            r.halo = ex2_approx(gh);
+        };
+
         // ---- state of the node row below the current element row
         float ehor[NE], U[NE], hnu[NE], nlr = 0.f;
         Row<NE> A, B, C, nA, nB, nC;
@@ -276,15 +347,17 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             }
         }
         if constexpr (!KL) {
-            if constexpr (RING) read_row(nA, jbeg, 1); else load_row(nA, nub, jbeg);
-            nlr = right_nb(nA);
+            if constexpr (KN) nu_row(nA, jbeg);
+            else if constexpr (RING) read_row(nA, jbeg, 1);
+            else load_row(nA, nub, jbeg);
+            nlr = KN ? nA.halo : right_nb(nA);
 #pragma unroll
             for (int k = 0; k < NE; ++k) hnu[k] = nA.v[k] + ((k + 1 < NE) ? nA.v[(k + 1 < NE) ? k + 1 : k] : nlr);
         }
 
         if constexpr (!RING) {
             load_row(B, ub, jbeg + 1);
-            if constexpr (!KL) load_row(nB, nub, jbeg + 1);
+            if constexpr (NLOAD) load_row(nB, nub, jbeg + 1);
         }
 
         // One element row: lo holds node row j, cur node row j+1 (read from the ring, or loaded by the
@@ -294,16 +367,17 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
                 issue_row(j + T2_STAGES);               // its slot held row j, which is in registers already
                 cp_async_wait<T2_STAGES - 1>();         // row j+1 has landed
                 read_row(cur, j + 1, 0);
-                if constexpr (!KL) read_row(ncur, j + 1, 1);
+                if constexpr (NLOAD) read_row(ncur, j + 1, 1);
             } else if (j < jend) {
                 load_row(nxt, ub, j + 2);
-                if constexpr (!KL) load_row(nnxt, nub, j + 2);
+                if constexpr (NLOAD) load_row(nnxt, nub, j + 2);
             }
+            if constexpr (KN) nu_row(ncur, j + 1);
             fix_bc(cur);
             const bool own = (j >= n0);
             const float hir = right_nb(cur);
             float nhr = 0.f;
-            if constexpr (!KL) nhr = right_nb(ncur);
+            if constexpr (!KL) nhr = KN ? right_nb_nu(ncur) : right_nb(ncur);
 
             u64 g2[GS / 2];
             if constexpr (KL) {
@@ -494,10 +568,10 @@ Geo2 geometry(const dn_problem& p) {
     g.W = (nx + 128 * g.K - 1) / (128 * g.K);
     g.WY = T2_MAX_WARPS / g.W;
     g.full = (g.W * 128 * g.K == nx);
-    const int m = (p.nu_mode == DN_NU_KL_GAUSS) ? p.kl_modes : 0;
+    const int m = (p.nu_mode != DN_NU_NODAL) ? p.kl_modes : 0;
     g.GS = m ? (2 * (m + 1) + 3) / 4 * 4 : 0;
     const long long slots = 2ll * sm_count();
-    const int rmax_smem = g.GS ? (int)(32768 / ((size_t)g.WY * g.GS * 4)) - 1 : 4096;
+    const int rmax_smem = g.GS ? (int)(32768 / ((size_t)g.WY * g.GS * 4)) - 2 : 4096;
     long long best = -1;
     int bestR = 16;
     for (int R = 8; R <= 512 && R <= rmax_smem; ++R) {
@@ -512,32 +586,36 @@ Geo2 geometry(const dn_problem& p) {
     const int nch = (ny + g.R - 1) / g.R;
     g.nblkx = (nch + g.WY - 1) / g.WY;
     const size_t ring_row = (size_t)32 * g.W * 4 * g.K + 4 * ((g.W + 3) / 4);
-    g.smem = sizeof(float) * ((size_t)g.WY * (g.R + 1) * g.GS + (size_t)g.WY * 2 * T2_MAX_WARPS * 2 +
+    g.smem = sizeof(float) * ((size_t)g.WY * (g.R + 2) * g.GS + (size_t)g.WY * 2 * T2_MAX_WARPS * 2 +
                               (m ? 0 : (size_t)g.WY * T2_STAGES * 2 * ring_row));      // the ring serves the nodal variant
     return g;
 }
 
-template <int K, int M, bool FULL>
-cudaError_t launch_kmf(const Params& P, const Geo2& g, cudaStream_t s) {
+template <int K, int M, bool FULL, bool KN>
+cudaError_t launch_kmfn(const Params& P, const Geo2& g, cudaStream_t s) {
     dim3 grid((unsigned)g.nblkx, (unsigned)P.batch);
     const int threads = 32 * g.W * g.WY;
     // the energy-only kernel sums element energies; the fused kernel takes J from the residual
     cudaError_t e;
     if (P.r) {
-        e = cudaFuncSetAttribute(tiled2d_kernel<K, M, true, FULL, (M == 0)>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+        e = cudaFuncSetAttribute(tiled2d_kernel<K, M, true, FULL, (M == 0), KN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
         if (e != cudaSuccess) return e;
-        tiled2d_kernel<K, M, true, FULL, (M == 0)><<<grid, threads, g.smem, s>>>(P, g.W, g.WY, g.R);
+        tiled2d_kernel<K, M, true, FULL, (M == 0), KN><<<grid, threads, g.smem, s>>>(P, g.W, g.WY, g.R);
     } else {
-        e = cudaFuncSetAttribute(tiled2d_kernel<K, M, false, FULL, (M == 0)>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+        e = cudaFuncSetAttribute(tiled2d_kernel<K, M, false, FULL, (M == 0), KN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
         if (e != cudaSuccess) return e;
-        tiled2d_kernel<K, M, false, FULL, (M == 0)><<<grid, threads, g.smem, s>>>(P, g.W, g.WY, g.R);
+        tiled2d_kernel<K, M, false, FULL, (M == 0), KN><<<grid, threads, g.smem, s>>>(P, g.W, g.WY, g.R);
     }
     return cudaGetLastError();
 }
 
 template <int K, int M>
 cudaError_t launch_km(const Params& P, const Geo2& g, cudaStream_t s) {
-    return g.full ? launch_kmf<K, M, true>(P, g, s) : launch_kmf<K, M, false>(P, g, s);
+    if constexpr (M > 0) {
+        if (P.nu_mode == DN_NU_KL_NODAL)
+            return g.full ? launch_kmfn<K, M, true, true>(P, g, s) : launch_kmfn<K, M, false, true>(P, g, s);
+    }
+    return g.full ? launch_kmfn<K, M, true, false>(P, g, s) : launch_kmfn<K, M, false, false>(P, g, s);
 }
 
 template <int K>
@@ -559,7 +637,7 @@ cudaError_t launch_k(const Params& P, const Geo2& g, cudaStream_t s) {
 }  // namespace
 
 bool tiled2d_applicable(const dn_problem& p) {
-    return p.grid.dim == 2 && p.nu_mode != DN_NU_KL_NODAL && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 128 * 2 * T2_MAX_WARPS &&
+    return p.grid.dim == 2 && p.grid.nx % 4 == 0 && p.grid.nx >= 8 && p.grid.nx <= 128 * 2 * T2_MAX_WARPS &&
            p.grid.ny >= 2;
 }
 
