@@ -358,6 +358,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
         if constexpr (!RING) {
             load_row(B, ub, jbeg + 1);
             if constexpr (NLOAD) load_row(nB, nub, jbeg + 1);
+            if constexpr (KN) nu_row(nB, jbeg + 1);
         }
 
         // One element row: lo holds node row j, cur node row j+1 (read from the ring, or loaded by the
@@ -372,7 +373,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
                 load_row(nxt, ub, j + 2);
                 if constexpr (NLOAD) load_row(nnxt, nub, j + 2);
             }
-            if constexpr (KN) nu_row(ncur, j + 1);
+            if constexpr (KN) { if (j < jend) nu_row(nnxt, j + 2); }   // one row ahead, like the loaded rows
             fix_bc(cur);
             const bool own = (j >= n0);
             const float hir = right_nb(cur);
