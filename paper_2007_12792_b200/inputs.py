@@ -171,3 +171,35 @@ def random_positive_field(shape, seed: int, spread: float = 0.5) -> np.ndarray:
 def random_field(shape, seed: int, scale: float = 1.0) -> np.ndarray:
     rng = np.random.default_rng(np.random.SeedSequence([int(seed), 11]))
     return (scale * rng.standard_normal(shape)).astype(np.float32)
+
+
+# ---- the paper's own workload: inviscid Burgers on (x, t) in [0,1] x [0, 0.2] -------------------------
+@dataclass
+class BurgersInputs:
+    nx: int
+    nt: int
+    batch: int
+    T: float
+    lam: float
+    c: np.ndarray         # float32 [B]: parameter of the initial-condition family
+    u: np.ndarray         # float32 [B][nt][nx]: stand-in for a generator output
+    seed: int
+
+
+def burgers_inputs(nx: int, nt: int, batch: int, seed: int = BASE_SEED + 7000, noise: float = 0.01,
+                   samples: Optional[Sequence[int]] = None) -> BurgersInputs:
+    """Synthetic generator outputs for the Burgers loss: c ~ U(3, 6) (the paper's first example), the
+    initial profile transported with speed 1/2, u = (1 - cos(2 pi c (x - t/2))) / 2, plus N(0, noise^2)."""
+    if samples is None:
+        samples = range(batch)
+    samples = list(samples)
+    x = _axis(nx)
+    t = 0.2 * _axis(nt)
+    cs, us = [], []
+    for b in samples:
+        rng = _rng(seed, b)
+        c = np.float32(rng.uniform(3.0, 6.0))
+        u = 0.5 * (1.0 - np.cos(2.0 * np.pi * float(c) * (x[None, :] - 0.5 * t[:, None]))) + noise * rng.standard_normal((nt, nx))
+        cs.append(c)
+        us.append(u.astype(np.float32))
+    return BurgersInputs(nx, nt, len(samples), 0.2, 1.0, np.array(cs, dtype=np.float32), np.stack(us), seed)
