@@ -164,6 +164,48 @@ dn_status dn_energy_grad_host(const dn_problem* problem, const float* u_host, co
                               float* J_host, float* r_host, void* staging, size_t staging_bytes,
                               void* stream);
 
+/* ---- The paper's own example: finite-difference loss of the inviscid Burgers equation ------------
+ *
+ *        u_t + u u_x = 0 on (x,t) in [0,1] x [0,T],   u(x,0) = (1 - cos(2 pi c x)) / 2
+ *
+ * ("Introduction", Eq. (Inviscid_Burgers), Eq. (initial-condition)).  A generated field is scored by
+ * L = L_p + lambda L_b ("DiffNets", Eq. (diffnetloss), Eq. (pde_loss), Eq. (boundaryloss)) with the
+ * first derivatives taken by 3x3 Sobel stencils ("Implementing the forward model"):
+ *
+ *   field   u[b][j][i] at x_i = i hx, t_j = j ht,  hx = 1/(nx-1), ht = T/(nt-1)   (x fastest)
+ *   u_x     = sum Sx[dj][di] u[j+dj][i+di] / (8 hx),  Sx = [[-1,0,1],[-2,0,2],[-1,0,1]];  u_t: Sx transposed, / (8 ht)
+ *   res     = u_t + u u_x at the interior nodes (0 < i < nx-1, 0 < j < nt-1)
+ *   L_p[b]  = hx ht sum_interior res^2
+ *   L_b[b]  = hx sum_i (u[0][i] - u(x_i,0))^2 + ht sum_j u[j][0]^2      (initial row and inflow column)
+ *   L[b]    = L_p[b] + lambda L_b[b],    g = dL/du at every node.
+ *
+ * The paper names the stencils only; the 1/(8h) normalisation (exact on linear fields), the discrete
+ * norms and the inflow-only boundary term are this library's reading. */
+typedef struct {
+    int32_t nx, nt;              /* nodes in x and t, each in 3..DN_MAX_EXTENT                      */
+    int32_t batch;               /* B >= 1                                                         */
+    float T;                     /* final time (> 0); the paper's domain has T = 0.2               */
+    float lambda;                /* weight of L_b                                                  */
+    const float* c;              /* [B] wave numbers of the initial-condition family               */
+    uint32_t flags;              /* DN_FORCE_GENERIC or 0                                          */
+} dn_burgers;
+
+/* Bytes of device scratch (per-warp loss partials) dn_burgers_loss_grad needs; 0 if invalid. */
+size_t dn_burgers_workspace_bytes(const dn_burgers* problem);
+
+/* Loss and its exact gradient in one pass over u (Algorithm 1: loss, then its gradient for
+ * back-propagation).  u: [B][nt][nx];  L: [B] or NULL;  parts: [B][2] = (L_p, L_b) or NULL;
+ * g: [B][nt][nx] or NULL (loss only), multiplied by gL[b] when gL != NULL; g must not overlap u.
+ * Grids with nx % 4 == 0 and 16-byte aligned u and g take the row-marching kernel, all others an
+ * any-size kernel.  event_before / event_after: optional caller-owned CUDA events recorded on
+ * `stream` around the main kernel (a measurement aid), or NULL. */
+dn_status dn_burgers_loss_grad(const dn_burgers* problem, const float* u, const float* gL, float* L,
+                               float* parts, float* g, void* workspace, size_t workspace_bytes,
+                               void* stream, void* event_before, void* event_after);
+
+/* Name of the kernel family dn_burgers_loss_grad would use for these pointers ("march", "generic"). */
+const char* dn_burgers_path_name(const dn_burgers* problem, const float* u, const float* g);
+
 /* Number of kernel launches the last-validated path of this problem enqueues per
  * dn_energy_grad call (for launch accounting); 0 if the problem is invalid. */
 int32_t dn_launches_per_call(const dn_problem* problem);

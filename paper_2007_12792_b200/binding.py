@@ -29,7 +29,8 @@ DN_FORCE_GENERIC = 4
 DN_MAX_KL_MODES = 8
 
 EXPORTS = ("dn_workspace_bytes", "dn_host_staging_bytes", "dn_kl_field", "dn_energy", "dn_energy_grad",
-           "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced", "dn_energy_grad_static", "dn_launches_per_call", "dn_path_name", "dn_status_string")
+           "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced", "dn_energy_grad_static", "dn_launches_per_call", "dn_path_name", "dn_status_string",
+           "dn_burgers_workspace_bytes", "dn_burgers_loss_grad", "dn_burgers_path_name")
 
 
 class DnGrid(C.Structure):
@@ -42,6 +43,11 @@ class DnProblem(C.Structure):
         ("kl_modes", C.c_int32), ("kl_w", C.c_void_p), ("f_const", C.c_float), ("f", C.c_void_p),
         ("bc_x0", C.c_float), ("bc_x1", C.c_float), ("flags", C.c_uint32),
     ]
+
+
+class DnBurgers(C.Structure):
+    _fields_ = [("nx", C.c_int32), ("nt", C.c_int32), ("batch", C.c_int32), ("T", C.c_float), ("lam", C.c_float),
+                ("c", C.c_void_p), ("flags", C.c_uint32)]
 
 
 class DnError(RuntimeError):
@@ -77,6 +83,12 @@ def lib():
         L.dn_launches_per_call.argtypes = [PP]; L.dn_launches_per_call.restype = C.c_int32
         L.dn_path_name.argtypes = [PP]; L.dn_path_name.restype = C.c_char_p
         L.dn_status_string.argtypes = [C.c_int]; L.dn_status_string.restype = C.c_char_p
+        PB = C.POINTER(DnBurgers)
+        L.dn_burgers_workspace_bytes.argtypes = [PB]; L.dn_burgers_workspace_bytes.restype = C.c_size_t
+        L.dn_burgers_loss_grad.argtypes = [PB, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.dn_burgers_loss_grad.restype = C.c_int
+        L.dn_burgers_path_name.argtypes = [PB, C.c_void_p, C.c_void_p]; L.dn_burgers_path_name.restype = C.c_char_p
         for f in ("dn_kl_field", "dn_energy", "dn_energy_grad", "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced"):
             getattr(L, f).restype = C.c_int
         _lib = L
@@ -238,3 +250,52 @@ def dn_energy_grad_host(problem: Problem, u_host: torch.Tensor, gJ_host: Optiona
                                      _ptr(J_host, "J_host", "cpu"), _ptr(r_host, "r_host", "cpu"),
                                      staging.data_ptr(), staging.numel(), _stream(stream)), "dn_energy_grad_host")
     return J_host, r_host
+
+
+@dataclass
+class Burgers:
+    """Python mirror of ``dn_burgers`` (the paper's Burgers finite-difference loss)."""
+    nx: int
+    nt: int
+    batch: int
+    c: Optional[torch.Tensor] = None      # [B] float32 wave numbers of the initial-condition family
+    T: float = 0.2
+    lam: float = 1.0
+    flags: int = 0
+
+    @property
+    def shape(self):
+        return (self.batch, self.nt, self.nx)
+
+    def c_struct(self, device: str = "cuda") -> DnBurgers:
+        p = DnBurgers()
+        p.nx, p.nt, p.batch, p.T, p.lam, p.flags = self.nx, self.nt, self.batch, self.T, self.lam, self.flags
+        p.c = _ptr(self.c, "c", device)
+        return p
+
+
+def dn_burgers_workspace_bytes(problem: Burgers) -> int:
+    return int(lib().dn_burgers_workspace_bytes(C.byref(problem.c_struct(device="any"))))
+
+
+def dn_burgers_path_name(problem: Burgers, u: Optional[torch.Tensor], g: Optional[torch.Tensor]) -> str:
+    return lib().dn_burgers_path_name(C.byref(problem.c_struct(device="any")), _ptr(u, "u", "any"), _ptr(g, "g", "any")).decode()
+
+
+def new_burgers_workspace(problem: Burgers, device="cuda") -> torch.Tensor:
+    return torch.empty(max(dn_burgers_workspace_bytes(problem), 256), dtype=torch.uint8, device=device)
+
+
+def dn_burgers_loss_grad(problem: Burgers, u: torch.Tensor, gL: Optional[torch.Tensor], L: Optional[torch.Tensor],
+                         parts: Optional[torch.Tensor], g: Optional[torch.Tensor], workspace: torch.Tensor, stream=None,
+                         event_before: Optional[torch.cuda.Event] = None, event_after: Optional[torch.cuda.Event] = None,
+                         _cstruct=None):
+    """L[b] = L_p + lam L_b, parts[b] = (L_p, L_b) and g = dL/du (times gL[b]) of the Burgers loss; any of L, parts,
+    g may be None.  The two optional (created, timing-enabled) events are recorded around the main kernel."""
+    p = _cstruct if _cstruct is not None else problem.c_struct()
+    eb = None if event_before is None else event_before.cuda_event
+    ea = None if event_after is None else event_after.cuda_event
+    _check(lib().dn_burgers_loss_grad(C.byref(p), _ptr(u, "u"), _ptr(gL, "gL"), _ptr(L, "L"), _ptr(parts, "parts"),
+                                      _ptr(g, "g"), workspace.data_ptr(), workspace.numel(), _stream(stream), eb, ea),
+           "dn_burgers_loss_grad")
+    return L, parts, g
