@@ -28,10 +28,10 @@ namespace dn {
 namespace {
 
 constexpr int BG_WARPS = 8;          // warps per block
-constexpr int BG_RING = 8;           // ring slots per warp (BG_RING - 1 rows in flight)
+constexpr int BG_RING = 6;           // ring slots per warp (BG_RING - 1 rows in flight); the six step phases name them
 constexpr int BG_COLS = 120;         // columns of g per warp
 constexpr int BG_SMS = 148;
-constexpr int BG_BLOCKS_PER_SM = 3;
+constexpr int BG_BLOCKS_PER_SM = 2;
 
 struct BParams {
     int nx, nt, batch;
@@ -46,10 +46,11 @@ struct BParams {
     double* partials;                // [B][nslot][3]: sum res^2, sum (u - u0)^2 on row 0, sum u^2 on column 0
 };
 
-__device__ __forceinline__ void cp_async16_zfill(float* smem_dst, const float* gsrc, bool valid) {
-    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-    const int n = valid ? 16 : 0;    // bytes read from gsrc; the rest of the 16 is written as zero
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "r"(n) : "memory");
+// 16-byte asynchronous copy into the ring slot at byte offset OFF of smem_base; reads nothing and writes zeros when !valid.
+template <int OFF>
+__device__ __forceinline__ void cp_async16_zfill(unsigned smem_base, const float* gsrc, bool valid) {
+    const int n = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0+%3], [%1], 16, %2;" ::"r"(smem_base), "l"(gsrc), "r"(n), "n"(OFF) : "memory");
 }
 __device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -62,38 +63,42 @@ struct MarchState {
 
 struct MarchCtx {
     const float* ub;                 // this sample's field
-    float* gb;
-    float* ring;                     // this lane's slot 0 in the warp's ring
-    int nx, nt, j0, j1, xl, lane;
-    bool xvalid;                     // this lane's four columns exist
-    bool store;                      // ... and belong to this warp's range
+    const float* psrc;               // this lane's four columns of the row that is copied next
+    float* pg;                       // this lane's four columns of the row of g that is stored next
+    const float4* ring;              // this lane's entry of ring slot 0
+    unsigned ring_s;                 // the same as a shared-space address
+    int nt_lane;                     // nt, or a negative number for lanes past the field (nothing to copy)
+    int j0, j1;
+    bool store;                      // this lane's four columns exist and belong to this warp's range
     bool col0, colN;                 // this lane's first column is x = 0 / its last column is x = nx-1
+    int nx;
     float ct, cx, s, bts;            // s = 2 hx ht gL;  bts = lambda 2 ht gL
+    float ef, ebf;                   // running sums of res^2 and of u(0,t)^2 since the last flush
     double e, ebt;
 };
 
-__device__ __forceinline__ void issue_row(const MarchCtx& C, int n, int k) {
-    const bool ok = C.xvalid && n >= 0 && n < C.nt;
-    const float* src = ok ? C.ub + (size_t)n * C.nx + C.xl : C.ub;
-    cp_async16_zfill(C.ring + (size_t)(k & (BG_RING - 1)) * 128, src, ok);
-    cp_commit();
-}
-
-// One step of the march: row n of u lands (ring slot k), the residual of row n-1 is formed, row n-2 of g leaves.
-template <int PH, bool WANT_G>
-__device__ __forceinline__ void march_step(MarchState& S, MarchCtx& C, int n, int k) {
+// One step of the march: row n of u lands (ring slot PH), the residual of row n-1 is formed, row n-2 of g leaves.
+// EDGE steps test every row index against the field and the chunk; the others are known to be clear of all edges.
+template <int PH, bool EDGE, bool WANT_G>
+__device__ __forceinline__ void march_step(MarchState& S, MarchCtx& C, int n) {
     constexpr int iu = PH % 3, ic = (PH + 2) % 3, im = (PH + 1) % 3;
     constexpr int p0 = PH % 2, p1 = 1 - p0;
     cp_wait<BG_RING - 2>();
-    const float4 v = *reinterpret_cast<const float4*>(C.ring + (size_t)(k & (BG_RING - 1)) * 128);
-    issue_row(C, n + BG_RING - 1, k + BG_RING - 1);
+    const float4 v = C.ring[PH * 32];
+    {
+        const int nn = n + BG_RING - 1;                         // the slot of row n-1 is free again
+        const bool ok = EDGE ? (nn >= 0 && nn < C.nt_lane) : (nn < C.nt_lane);
+        cp_async16_zfill<((PH + BG_RING - 1) % BG_RING) * 512>(C.ring_s, ok ? C.psrc : C.ub, ok);
+        cp_commit();
+        C.psrc += C.nx;
+    }
     S.u[iu][1] = v.x; S.u[iu][2] = v.y; S.u[iu][3] = v.z; S.u[iu][4] = v.w;
     S.u[iu][0] = __shfl_up_sync(0xffffffffu, v.w, 1);
     S.u[iu][5] = __shfl_down_sync(0xffffffffu, v.x, 1);
 
     float ux[4], a[6], b[6], res[4];
     const int q = n - 1;                                        // residual row
-    const bool rowok = q >= 1 && q <= C.nt - 2 && q >= C.j0 - 1;
+    const bool rowok = !EDGE || (q >= 1 && q <= C.nt_lane - 2 && q >= C.j0 - 1);
     const float s = rowok ? C.s : 0.0f;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
@@ -109,22 +114,17 @@ __device__ __forceinline__ void march_step(MarchState& S, MarchCtx& C, int n, in
         const float dts = dt[c] + dt[c + 2] + 2.0f * dt[c + 1];
         res[c] = C.ct * dts + S.u[ic][c + 1] * ux[c];
         if (c == 0 && C.col0) res[c] = 0.0f;                // the residual lives at interior columns only (lanes past
-                                                            // the field carry s = 0)
-        if (c == 3 && C.colN) res[c] = 0.0f;
+        if (c == 3 && C.colN) res[c] = 0.0f;                // the field carry s = 0)
         a[c + 1] = res[c] * s;
         b[c + 1] = a[c + 1] * S.u[ic][c + 1];
     }
-    if (rowok && q >= C.j0 && q < C.j1 && C.store) {
-        const float e = res[0] * res[0] + res[1] * res[1] + (res[2] * res[2] + res[3] * res[3]);
-        C.e += (double)e;
-    }
+    if (!EDGE || (rowok && q >= C.j0 && q < C.j1))              // lanes that store nothing drop their sum at the end
+        C.ef += res[0] * res[0] + res[1] * res[1] + (res[2] * res[2] + res[3] * res[3]);
     a[0] = __shfl_up_sync(0xffffffffu, a[4], 1);
     a[5] = __shfl_down_sync(0xffffffffu, a[1], 1);
     b[0] = __shfl_up_sync(0xffffffffu, b[4], 1);
     b[5] = __shfl_down_sync(0xffffffffu, b[1], 1);
 
-    const int jr = n - 2;                                       // row of g that is now complete
-    const bool emit = jr >= C.j0 && jr < C.j1;
     float g[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
@@ -134,20 +134,21 @@ __device__ __forceinline__ void march_step(MarchState& S, MarchCtx& C, int n, in
         g[c] = C.ct * (S.Ax[p1][c] - axn) + C.cx * (S.Db[p1][c] + dbn + 2.0f * S.Db[p0][c]) + S.P[p0][c];
         S.Ax[p1][c] = axn; S.Db[p1][c] = dbn; S.P[p1][c] = pn;
     }
-    if (emit && C.store) {
+    const int jr = n - 2;                                       // row of g that is now complete
+    if (C.store && (!EDGE || (jr >= C.j0 && jr < C.j1))) {
         if (C.col0) {
             const float w = S.u[im][1];
             g[0] += C.bts * w;
-            C.ebt += (double)(w * w);
+            C.ebf += w * w;
         }
-        if (WANT_G)
-            __stcs(reinterpret_cast<float4*>(C.gb + (size_t)jr * C.nx + C.xl), make_float4(g[0], g[1], g[2], g[3]));
+        if (WANT_G) __stcs(reinterpret_cast<float4*>(C.pg), make_float4(g[0], g[1], g[2], g[3]));
     }
+    C.pg += C.nx;
 }
 
 template <bool WANT_G>
 __global__ void __launch_bounds__(BG_WARPS * 32, BG_BLOCKS_PER_SM) burgers_march_kernel(BParams Q) {
-    __shared__ __align__(16) float ring_all[BG_WARPS][BG_RING][128];
+    __shared__ float4 ring_all[BG_WARPS][BG_RING][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long task = (long long)blockIdx.x * BG_WARPS + warp;
     if (task >= Q.tasks) return;                                // whole warps leave; nothing below synchronises the block
@@ -156,20 +157,22 @@ __global__ void __launch_bounds__(BG_WARPS * 32, BG_BLOCKS_PER_SM) burgers_march
     const int bi = (int)(task / ((long long)Q.wx * Q.nchunk));
 
     MarchCtx C;
-    C.nx = Q.nx; C.nt = Q.nt; C.lane = lane;
+    C.nx = Q.nx;
     C.j0 = chunk * Q.R;
     C.j1 = min(C.j0 + Q.R, Q.nt);
-    C.xl = BG_COLS * w - 4 + 4 * lane;
-    C.xvalid = C.xl >= 0 && C.xl < Q.nx;
-    C.store = C.xvalid && lane >= 1 && lane <= 30;
-    C.col0 = C.xl == 0;
-    C.colN = C.xl + 4 == Q.nx;
+    const int xl = BG_COLS * w - 4 + 4 * lane;
+    const bool xvalid = xl >= 0 && xl < Q.nx;
+    C.nt_lane = xvalid ? Q.nt : -(1 << 30);
+    C.store = xvalid && lane >= 1 && lane <= 30;
+    C.col0 = xl == 0;
+    C.colN = xl + 4 == Q.nx;
     C.ub = Q.u + (size_t)bi * Q.nt * Q.nx;
-    C.gb = WANT_G ? Q.g + (size_t)bi * Q.nt * Q.nx : nullptr;
-    C.ring = &ring_all[warp][0][4 * lane];
+    float* const gb = WANT_G ? Q.g + (size_t)bi * Q.nt * Q.nx : nullptr;
+    C.ring = &ring_all[warp][0][lane];
+    C.ring_s = (unsigned)__cvta_generic_to_shared(C.ring);
     const float gl = Q.gL ? Q.gL[bi] : 1.0f;
-    C.ct = Q.ct; C.cx = Q.cx; C.s = C.xvalid ? Q.w2 * gl : 0.0f; C.bts = Q.bt * gl;
-    C.e = 0.0; C.ebt = 0.0;
+    C.ct = Q.ct; C.cx = Q.cx; C.s = xvalid ? Q.w2 * gl : 0.0f; C.bts = Q.bt * gl;
+    C.e = 0.0; C.ebt = 0.0; C.ef = 0.0f; C.ebf = 0.0f;
 
     MarchState S;
 #pragma unroll
@@ -181,37 +184,58 @@ __global__ void __launch_bounds__(BG_WARPS * 32, BG_BLOCKS_PER_SM) burgers_march
 #pragma unroll
         for (int c = 0; c < 4; ++c) { S.Dx[r][c] = 0.0f; S.Ax[r][c] = 0.0f; S.Db[r][c] = 0.0f; S.P[r][c] = 0.0f; }
 
-    const int nbeg = C.j0 - 2, nend = C.j1 + 2;                 // rows n = nbeg .. nend-1 are walked
+    // Rows n = nbeg .. nend-1 are walked.  Steps with  j0 + 2 <= n < min(j1 + 1, nt),  whose copy also stays at or
+    // after row 0, touch no edge of the field or of the chunk.
+    const int nbeg = C.j0 - 2, nend = C.j1 + 2;
+    const int nfull0 = C.j0 + 2, nfull1 = min(C.j1 + 1, Q.nt);
+    {
+        const float* p = C.ub + ((long long)nbeg * Q.nx + xl);  // not dereferenced unless the row exists
 #pragma unroll
-    for (int d = 0; d < BG_RING - 1; ++d) issue_row(C, nbeg + d, d);
-    int n = nbeg, k = 0;
-    while (true) {
-        march_step<0, WANT_G>(S, C, n, k); if (++n >= nend) break; ++k;
-        march_step<1, WANT_G>(S, C, n, k); if (++n >= nend) break; ++k;
-        march_step<2, WANT_G>(S, C, n, k); if (++n >= nend) break; ++k;
-        march_step<3, WANT_G>(S, C, n, k); if (++n >= nend) break; ++k;
-        march_step<4, WANT_G>(S, C, n, k); if (++n >= nend) break; ++k;
-        march_step<5, WANT_G>(S, C, n, k); if (++n >= nend) break; ++k;
+        for (int d = 0; d < BG_RING - 1; ++d) {
+            const int nn = nbeg + d;
+            const bool ok = nn >= 0 && nn < C.nt_lane;
+            const unsigned dst = C.ring_s + d * 512;
+            cp_async16_zfill<0>(dst, ok ? p : C.ub, ok);
+            cp_commit();
+            p += Q.nx;
+        }
+        C.psrc = p;
+        C.pg = gb + ((long long)(nbeg - 2) * Q.nx + xl);
     }
+    int n = nbeg;
+#define DN_BG_STEP(PH)                                                      \
+    if (n >= nend) break;                                                   \
+    if (n >= nfull0 && n < nfull1) march_step<PH, false, WANT_G>(S, C, n);  \
+    else march_step<PH, true, WANT_G>(S, C, n);                             \
+    ++n;
+    while (true) {
+        DN_BG_STEP(0) DN_BG_STEP(1) DN_BG_STEP(2) DN_BG_STEP(3) DN_BG_STEP(4) DN_BG_STEP(5)
+        C.e += (double)C.ef; C.ef = 0.0f;
+        C.ebt += (double)C.ebf; C.ebf = 0.0f;
+    }
+#undef DN_BG_STEP
+    C.e += (double)C.ef;
+    C.ebt += (double)C.ebf;
+    if (!C.store) C.e = 0.0;
     cp_wait<0>();                                               // copies issued past the last row (zero-fill or unused rows)
 
     // Initial-condition term of L_b on row 0 (first chunk only): this lane adds it to the row it stored itself.
     double e0 = 0.0;
     if (C.j0 == 0 && C.store) {
-        const float4 uv = *reinterpret_cast<const float4*>(C.ub + C.xl);
+        const float4 uv = *reinterpret_cast<const float4*>(C.ub + xl);
         const float uu[4] = {uv.x, uv.y, uv.z, uv.w};
         const double cc = (double)Q.c[bi];
         const float bxs = Q.bx * gl;
         float d[4], ee = 0.0f;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const float u0 = (float)(0.5 * (1.0 - cospi(2.0 * cc * ((double)(C.xl + c) / (double)(Q.nx - 1)))));
+            const float u0 = (float)(0.5 * (1.0 - cospi(2.0 * cc * ((double)(xl + c) / (double)(Q.nx - 1)))));
             d[c] = uu[c] - u0;
             ee += d[c] * d[c];
         }
         e0 = (double)ee;
         if (WANT_G) {
-            float4* gp = reinterpret_cast<float4*>(C.gb + C.xl);
+            float4* gp = reinterpret_cast<float4*>(gb + xl);
             float4 gv = *gp;
             gv.x += bxs * d[0]; gv.y += bxs * d[1]; gv.z += bxs * d[2]; gv.w += bxs * d[3];
             *gp = gv;
