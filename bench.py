@@ -3,6 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--nu-mode kl|nodal]
     python bench.py --impl reference ...      # the fp64 CPU oracle on the host cores
+    python bench.py --workload burgers ...    # second workload: the paper's finite-difference Burgers loss
 
 One "step" is one pass of the whole hot path over one synthetic batch: a single
 ``dn_energy_grad`` call (KL tables -> fused energy+residual kernel -> energy
@@ -162,6 +163,156 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+BURGERS = {"nx": 1024, "nt": 1024, "batch": 64}       # the paper's first high-resolution example: 1024 x 1024, minibatch 64
+BURGERS_METRIC = "Burgers FD loss+gradient Gnodes/s"
+BURGERS_UNIT = "Gnodes/s"
+BURGERS_NAME = "burgers_1024x1024_b64"
+
+
+def burgers_oracle_sample_run(target_seconds: float = 12.0):
+    """Times the numpy oracle of the Burgers loss on whole samples of the workload."""
+    from oracle import burgers as ob
+    nodes = BURGERS["nx"] * BURGERS["nt"]
+
+    def run(n):
+        inp = inputs.burgers_inputs(BURGERS["nx"], BURGERS["nt"], BURGERS["batch"], samples=range(n))
+        t = time.perf_counter()
+        ob.loss_grad(inp.u, inp.c.astype(np.float64), T=float(np.float32(0.2)))
+        return time.perf_counter() - t
+
+    t1 = run(1)
+    n = int(max(1, min(BURGERS["batch"], round(target_seconds / max(t1, 1e-3)))))
+    t = run(n) if n > 1 else t1
+    return {"value": nodes * n / t / 1e9, "unit": BURGERS_UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{n} of {BURGERS['batch']} samples of {BURGERS_NAME} ({nodes * n} nodes, loss + full gradient, "
+                      f"numpy fp64), {t:.2f} s wall"}, t, n
+
+
+def run_reference_burgers(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    times, base, n = [], None, 1
+    for it in range(args.warmup + args.steps):
+        base, t, n = burgers_oracle_sample_run(target_seconds=max(0.5, min(4.0, 150.0 / (args.steps + args.warmup))))
+        if it >= args.warmup:
+            times.append(t)
+    ms = 1e3 * sum(times) / len(times)
+    value = BURGERS["nx"] * BURGERS["nt"] * n / (ms * 1e-3) / 1e9
+    base["value"] = value
+    print(json.dumps({"impl": "reference", "metric": BURGERS_METRIC, "value": value, "unit": BURGERS_UNIT,
+                      "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                      "config": {"workload": BURGERS_NAME, "step": f"oracle pass over {n} sample(s)"},
+                      "cpu_baseline": base,
+                      "e2e": {"value": value, "unit": BURGERS_UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main_burgers(args):
+    """The paper's own loss (finite-difference Burgers residual) as a second workload: one step = one
+    dn_burgers_loss_grad call (marching kernel + finaliser) over a minibatch of 64 fields of 1024 x 1024."""
+    import torch
+    import torch.distributed as dist
+    from paper_2007_12792_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()
+    nx, nt, bs = BURGERS["nx"], BURGERS["nt"], BURGERS["batch"]
+    inp = inputs.burgers_inputs(nx, nt, world * bs, samples=sharding.minibatch_indices(world * bs, world * bs, world, rank, 0))
+    u = torch.from_numpy(inp.u).cuda()
+    c = torch.from_numpy(inp.c).cuda()
+    g = torch.empty_like(u)
+    L = torch.empty(bs, device="cuda")
+    gL = torch.full((bs,), 1.0 / bs, device="cuda")            # gradient of the minibatch mean
+    prob = B.Burgers(nx=nx, nt=nt, batch=bs, c=c, T=float(np.float32(0.2)), lam=1.0)
+    ws = B.new_burgers_workspace(prob)
+    cs = prob.c_struct()
+    field_bytes = u.numel() * 4                                # 256 MiB in, 256 MiB out: larger than L2
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K = args.steps
+    ev_step = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    ev_main = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b_ in ev_step + ev_main:
+        a.record(); b_.record()
+    for _ in range(args.warmup):
+        B.dn_burgers_loss_grad(prob, u, gL, L, None, g, ws, _cstruct=cs)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    t0 = time.time()
+    for k in range(K):
+        ev_step[k][0].record()
+        B.dn_burgers_loss_grad(prob, u, gL, L, None, g, ws, event_before=ev_main[k][0], event_after=ev_main[k][1], _cstruct=cs)
+        ev_step[k][1].record()
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    step_ms = sum(a.elapsed_time(b_) for a, b_ in ev_step) / K
+    main_ms = sum(a.elapsed_time(b_) for a, b_ in ev_main) / K
+    Lsum = float(L.double().sum())
+
+    u_h = torch.from_numpy(inp.u).pin_memory()
+    c_h = torch.from_numpy(inp.c).pin_memory()
+    gL_h = gL.cpu().pin_memory()
+    g_h = torch.empty(u.shape).pin_memory()
+    L_h = torch.empty(bs).pin_memory()
+    prob_h = B.Burgers(nx=nx, nt=nt, batch=bs, c=c_h, T=float(np.float32(0.2)), lam=1.0)
+    staging = B.new_burgers_host_staging(prob_h)
+    B.dn_burgers_loss_grad_host(prob_h, u_h, gL_h, L_h, None, g_h, staging)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.e2e_steps):
+        B.dn_burgers_loss_grad_host(prob_h, u_h, gL_h, L_h, None, g_h, staging)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+    step_ms, main_ms, e2e_ms = sharding.max_over_ranks([step_ms, main_ms, e2e_ms])
+    Lmean = sharding.mean_over_ranks(Lsum, bs)
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        nodes = nx * nt * bs
+        alg_bytes = 8 * nodes
+        achieved = alg_bytes / (main_ms * 1e-3) / 1e9
+        cap = ncu_capture(f"march:{BURGERS_NAME}")
+        line = {
+            "metric": BURGERS_METRIC, "value": world * nodes / (step_ms * 1e-3) / 1e9, "unit": BURGERS_UNIT, "n_gpus": world,
+            "steps": K, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": BURGERS_NAME, "kernel_path": B.dn_burgers_path_name(prob, u, g),
+                       "nodes_per_step_per_gpu": nodes, "sharding": "independent batches per rank",
+                       "l2": "inputs larger than L2"},
+            "clocks": clocks,
+            "e2e": {"value": world * nodes / (e2e_ms * 1e-3) / 1e9, "unit": BURGERS_UNIT,
+                    "h2d_bytes_per_step": field_bytes + 8 * bs, "d2h_bytes_per_step": field_bytes + 4 * bs,
+                    "ms_per_step": e2e_ms, "steps": args.e2e_steps, "entry": "dn_burgers_loss_grad_host (pinned host buffers)"},
+            "gpu_launches": 2 * K,
+            "roofline": {"bound": "hbm", "kernel": "burgers_march_kernel", "achieved": achieved, "peak": peak,
+                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                         "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": main_ms,
+                         "traffic": cap["traffic"] if cap else None},
+            "checksum_L": Lsum, "mean_L_all_ranks": Lmean,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = burgers_oracle_sample_run()[0]
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -171,12 +322,16 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (default: 2D 2048^2, batch 16)")
     ap.add_argument("--nu-mode", default="kl", choices=["kl", "nodal", "klnodal"],
                     help="kl: KL at Gauss points (default); nodal: stored nodal field; klnodal: KL at nodes inside the kernel")
+    ap.add_argument("--workload", default="fem", choices=["fem", "burgers"],
+                    help="fem: the Galerkin energy+residual path (default); burgers: the paper's finite-difference Burgers loss")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
-        return run_reference(args)
+        return run_reference_burgers(args) if args.workload == "burgers" else run_reference(args)
+    if args.workload == "burgers":
+        return main_burgers(args)
 
     import torch
     import torch.distributed as dist

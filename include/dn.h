@@ -203,6 +203,18 @@ dn_status dn_burgers_loss_grad(const dn_burgers* problem, const float* u, const 
                                float* parts, float* g, void* workspace, size_t workspace_bytes,
                                void* stream, void* event_before, void* event_after);
 
+/* Bytes of device staging dn_burgers_loss_grad_host needs (u, g, c, gL, L, parts and the workspace); 0 if invalid. */
+size_t dn_burgers_host_staging_bytes(const dn_burgers* problem);
+
+/* dn_burgers_loss_grad with HOST buffers (problem->c is a HOST pointer here): copies c, gL and u to the
+ * device staging area, runs the same kernels, copies L, parts and g back and waits for the last copy.
+ * The batch flows in chunks of whole samples over two internal copy streams, as in dn_energy_grad_host.
+ * g_host must not be NULL; L_host, parts_host, gL_host may be.  staging: device memory of
+ * dn_burgers_host_staging_bytes(problem) bytes, 256-byte aligned.  Use pinned host memory. */
+dn_status dn_burgers_loss_grad_host(const dn_burgers* problem, const float* u_host, const float* gL_host,
+                                    float* L_host, float* parts_host, float* g_host, void* staging,
+                                    size_t staging_bytes, void* stream);
+
 /* Name of the kernel family dn_burgers_loss_grad would use for these pointers ("march", "generic"). */
 const char* dn_burgers_path_name(const dn_burgers* problem, const float* u, const float* g);
 

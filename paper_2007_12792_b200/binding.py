@@ -30,7 +30,8 @@ DN_MAX_KL_MODES = 8
 
 EXPORTS = ("dn_workspace_bytes", "dn_host_staging_bytes", "dn_kl_field", "dn_energy", "dn_energy_grad",
            "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced", "dn_energy_grad_static", "dn_launches_per_call", "dn_path_name", "dn_status_string",
-           "dn_burgers_workspace_bytes", "dn_burgers_loss_grad", "dn_burgers_path_name")
+           "dn_burgers_workspace_bytes", "dn_burgers_loss_grad", "dn_burgers_path_name",
+           "dn_burgers_host_staging_bytes", "dn_burgers_loss_grad_host")
 
 
 class DnGrid(C.Structure):
@@ -88,6 +89,10 @@ def lib():
         L.dn_burgers_loss_grad.argtypes = [PB, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]
         L.dn_burgers_loss_grad.restype = C.c_int
+        L.dn_burgers_host_staging_bytes.argtypes = [PB]; L.dn_burgers_host_staging_bytes.restype = C.c_size_t
+        L.dn_burgers_loss_grad_host.argtypes = [PB, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                C.c_size_t, C.c_void_p]
+        L.dn_burgers_loss_grad_host.restype = C.c_int
         L.dn_burgers_path_name.argtypes = [PB, C.c_void_p, C.c_void_p]; L.dn_burgers_path_name.restype = C.c_char_p
         for f in ("dn_kl_field", "dn_energy", "dn_energy_grad", "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced"):
             getattr(L, f).restype = C.c_int
@@ -299,3 +304,24 @@ def dn_burgers_loss_grad(problem: Burgers, u: torch.Tensor, gL: Optional[torch.T
                                       _ptr(g, "g"), workspace.data_ptr(), workspace.numel(), _stream(stream), eb, ea),
            "dn_burgers_loss_grad")
     return L, parts, g
+
+
+def dn_burgers_host_staging_bytes(problem: Burgers) -> int:
+    return int(lib().dn_burgers_host_staging_bytes(C.byref(problem.c_struct(device="any"))))
+
+
+def new_burgers_host_staging(problem: Burgers, device="cuda") -> torch.Tensor:
+    return torch.empty(max(dn_burgers_host_staging_bytes(problem), 256), dtype=torch.uint8, device=device)
+
+
+def dn_burgers_loss_grad_host(problem: Burgers, u_host: torch.Tensor, gL_host: Optional[torch.Tensor],
+                              L_host: Optional[torch.Tensor], parts_host: Optional[torch.Tensor], g_host: torch.Tensor,
+                              staging: torch.Tensor, stream=None):
+    """Host-buffer variant: ``problem.c`` and all tensors are HOST tensors (pinned for speed); ``staging`` is a device
+    byte buffer of dn_burgers_host_staging_bytes(problem).  Returns after the results are on the host."""
+    p = problem.c_struct(device="cpu")
+    _check(lib().dn_burgers_loss_grad_host(C.byref(p), _ptr(u_host, "u_host", "cpu"), _ptr(gL_host, "gL_host", "cpu"),
+                                           _ptr(L_host, "L_host", "cpu"), _ptr(parts_host, "parts_host", "cpu"),
+                                           _ptr(g_host, "g_host", "cpu"), staging.data_ptr(), staging.numel(),
+                                           _stream(stream)), "dn_burgers_loss_grad_host")
+    return L_host, parts_host, g_host

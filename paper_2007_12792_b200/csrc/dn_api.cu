@@ -214,34 +214,6 @@ dn_status dn_apply_bc(const dn_grid* g, int32_t batch, float b0, float b1, int32
                                                                                                             : DN_ERR_CUDA;
 }
 
-namespace {
-// Streams and events of one dn_energy_grad_host call (created and destroyed inside the call).
-struct HostPipe {
-    static constexpr int kMaxChunks = 32;
-    cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, copied[kMaxChunks] = {}, computed[kMaxChunks] = {};
-    bool create(int nchunks) {
-        if (cudaStreamCreateWithFlags(&in, cudaStreamNonBlocking) != cudaSuccess) return false;
-        if (cudaStreamCreateWithFlags(&out, cudaStreamNonBlocking) != cudaSuccess) return false;
-        if (cudaEventCreateWithFlags(&start, cudaEventDisableTiming) != cudaSuccess) return false;
-        for (int c = 0; c < nchunks; ++c) {
-            if (cudaEventCreateWithFlags(&copied[c], cudaEventDisableTiming) != cudaSuccess) return false;
-            if (cudaEventCreateWithFlags(&computed[c], cudaEventDisableTiming) != cudaSuccess) return false;
-        }
-        return true;
-    }
-    ~HostPipe() {
-        for (int c = 0; c < kMaxChunks; ++c) {
-            if (copied[c]) cudaEventDestroy(copied[c]);
-            if (computed[c]) cudaEventDestroy(computed[c]);
-        }
-        if (start) cudaEventDestroy(start);
-        if (in) cudaStreamDestroy(in);
-        if (out) cudaStreamDestroy(out);
-    }
-};
-}  // namespace
-
 // The batch is cut into chunks of whole samples that flow through three stages on three streams:
 // host->device copy, kernels (on the caller's stream), device->host copy.  Chunk c+1 is copied in
 // and chunk c-1 copied out while chunk c computes, so both directions of the host link stay busy.

@@ -445,4 +445,68 @@ dn_status dn_burgers_loss_grad(const dn_burgers* p, const float* u, const float*
     return DN_OK;
 }
 
+size_t dn_burgers_host_staging_bytes(const dn_burgers* p) {
+    if (validate_burgers(p) != DN_OK) return 0;
+    const size_t field = align_up(sizeof(float) * (size_t)p->batch * p->nx * p->nt);
+    const size_t small = align_up(sizeof(float) * 2 * (size_t)p->batch);
+    return 2 * field + 4 * small + dn_burgers_workspace_bytes(p);
+}
+
+dn_status dn_burgers_loss_grad_host(const dn_burgers* p, const float* u_host, const float* gL_host, float* L_host,
+                                    float* parts_host, float* g_host, void* staging, size_t staging_bytes, void* stream) {
+    dn_status st = validate_burgers(p);
+    if (st != DN_OK) return st;
+    if (!u_host || !g_host) return DN_ERR_NULL;
+    if (!staging || (reinterpret_cast<uintptr_t>(staging) % kAlign) != 0 || staging_bytes < dn_burgers_host_staging_bytes(p))
+        return DN_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t nodes = (size_t)p->nx * p->nt;
+    const size_t field = align_up(sizeof(float) * (size_t)p->batch * nodes);
+    const size_t small = align_up(sizeof(float) * 2 * (size_t)p->batch);
+    char* base = static_cast<char*>(staging);
+    float* d_u = reinterpret_cast<float*>(base);
+    float* d_g = reinterpret_cast<float*>(base + field);
+    float* d_c = reinterpret_cast<float*>(base + 2 * field);
+    float* d_gL = reinterpret_cast<float*>(base + 2 * field + small);
+    float* d_L = reinterpret_cast<float*>(base + 2 * field + 2 * small);
+    float* d_parts = reinterpret_cast<float*>(base + 2 * field + 3 * small);
+    void* ws = base + 2 * field + 4 * small;
+    const size_t ws_bytes = staging_bytes - (2 * field + 4 * small);   // a chunk never needs more than the whole batch
+
+    const int csize = (p->batch + HostPipe::kMaxChunks - 1) / HostPipe::kMaxChunks;
+    const int nchunks = (p->batch + csize - 1) / csize;
+    HostPipe pipe;
+    if (!pipe.create(nchunks)) return DN_ERR_CUDA;
+#define DN_TRY(x) do { if ((x) != cudaSuccess) return DN_ERR_CUDA; } while (0)
+    DN_TRY(cudaEventRecord(pipe.start, s));
+    DN_TRY(cudaStreamWaitEvent(pipe.in, pipe.start, 0));
+    DN_TRY(cudaStreamWaitEvent(pipe.out, pipe.start, 0));
+    DN_TRY(cudaMemcpyAsync(d_c, p->c, sizeof(float) * p->batch, cudaMemcpyHostToDevice, pipe.in));
+    if (gL_host) DN_TRY(cudaMemcpyAsync(d_gL, gL_host, sizeof(float) * p->batch, cudaMemcpyHostToDevice, pipe.in));
+    for (int c = 0; c < nchunks; ++c) {
+        const int b0 = c * csize;
+        const int nb = (b0 + csize <= p->batch) ? csize : p->batch - b0;
+        const size_t o = (size_t)b0 * nodes, n = (size_t)nb * nodes;
+        DN_TRY(cudaMemcpyAsync(d_u + o, u_host + o, sizeof(float) * n, cudaMemcpyHostToDevice, pipe.in));
+        DN_TRY(cudaEventRecord(pipe.copied[c], pipe.in));
+        DN_TRY(cudaStreamWaitEvent(s, pipe.copied[c], 0));
+        dn_burgers q = *p;
+        q.batch = nb;
+        q.c = d_c + b0;
+        st = dn_burgers_loss_grad(&q, d_u + o, gL_host ? d_gL + b0 : nullptr, L_host ? d_L + b0 : nullptr,
+                                  parts_host ? d_parts + 2 * (size_t)b0 : nullptr, d_g + o, ws, ws_bytes, s, nullptr, nullptr);
+        if (st != DN_OK) { cudaStreamSynchronize(pipe.in); cudaStreamSynchronize(s); cudaStreamSynchronize(pipe.out); return st; }
+        DN_TRY(cudaEventRecord(pipe.computed[c], s));
+        DN_TRY(cudaStreamWaitEvent(pipe.out, pipe.computed[c], 0));
+        DN_TRY(cudaMemcpyAsync(g_host + o, d_g + o, sizeof(float) * n, cudaMemcpyDeviceToHost, pipe.out));
+    }
+    DN_TRY(cudaStreamSynchronize(pipe.in));
+    DN_TRY(cudaStreamSynchronize(s));
+    if (L_host) DN_TRY(cudaMemcpyAsync(L_host, d_L, sizeof(float) * p->batch, cudaMemcpyDeviceToHost, pipe.out));
+    if (parts_host) DN_TRY(cudaMemcpyAsync(parts_host, d_parts, sizeof(float) * 2 * p->batch, cudaMemcpyDeviceToHost, pipe.out));
+    DN_TRY(cudaStreamSynchronize(pipe.out));
+#undef DN_TRY
+    return DN_OK;
+}
+
 }  // extern "C"

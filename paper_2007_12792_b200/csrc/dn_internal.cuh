@@ -85,6 +85,32 @@ Launch tiled2d_geometry(const dn_problem& p);
 Launch tiled3d_geometry(const dn_problem& p);
 size_t tiled3d_seam_floats(const dn_problem& p);   // scratch floats the tiled 3D kernel needs for its tile seams
 
+// Streams and events of one *_host call (created and destroyed inside the call).
+struct HostPipe {
+    static constexpr int kMaxChunks = 32;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, copied[kMaxChunks] = {}, computed[kMaxChunks] = {};
+    bool create(int nchunks) {
+        if (cudaStreamCreateWithFlags(&in, cudaStreamNonBlocking) != cudaSuccess) return false;
+        if (cudaStreamCreateWithFlags(&out, cudaStreamNonBlocking) != cudaSuccess) return false;
+        if (cudaEventCreateWithFlags(&start, cudaEventDisableTiming) != cudaSuccess) return false;
+        for (int c = 0; c < nchunks; ++c) {
+            if (cudaEventCreateWithFlags(&copied[c], cudaEventDisableTiming) != cudaSuccess) return false;
+            if (cudaEventCreateWithFlags(&computed[c], cudaEventDisableTiming) != cudaSuccess) return false;
+        }
+        return true;
+    }
+    ~HostPipe() {
+        for (int c = 0; c < kMaxChunks; ++c) {
+            if (copied[c]) cudaEventDestroy(copied[c]);
+            if (computed[c]) cudaEventDestroy(computed[c]);
+        }
+        if (start) cudaEventDestroy(start);
+        if (in) cudaStreamDestroy(in);
+        if (out) cudaStreamDestroy(out);
+    }
+};
+
 #ifdef __CUDACC__
 // Sum (d, l) over the block in a fixed order and let thread 0 store the pair.
 // Every thread of the block must call this.  blockDim.x * blockDim.y <= 1024.

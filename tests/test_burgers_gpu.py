@@ -126,6 +126,20 @@ def test_validation():
     assert B.dn_burgers_workspace_bytes(B.Burgers(nx=16, nt=8, batch=0, c=dev(inp.c))) == 0
 
 
+def test_host_entry_point():
+    inp = inputs.burgers_inputs(256, 96, 5)
+    gL = np.array([1.0, 0.5, 2.0, -1.0, 0.25], dtype=np.float32)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).pin_memory()
+    p = B.Burgers(nx=256, nt=96, batch=5, c=pin(inp.c), T=T32, lam=0.7)
+    g_h = torch.full(p.shape, float("nan")).pin_memory()
+    L_h = torch.full((5,), float("nan")).pin_memory()
+    parts_h = torch.full((5, 2), float("nan")).pin_memory()
+    staging = B.new_burgers_host_staging(p)
+    B.dn_burgers_loss_grad_host(p, pin(inp.u), pin(gL), L_h, parts_h, g_h, staging)
+    f = lambda t: t.numpy().astype(np.float64)
+    check(inp, f(L_h), f(parts_h), f(g_h), lam=0.7, gL=gL)
+
+
 def test_full_size_paper_example_on_sampled_samples():
     """1024 x 1024 outputs, minibatch 64 (the paper's first high-resolution example), in the launch configuration
     the benchmark times; the oracle scores three samples of the batch."""
