@@ -28,7 +28,9 @@ namespace dn {
 namespace {
 
 constexpr int BG_WARPS = 8;          // warps per block
-constexpr int BG_RING = 6;           // ring slots per warp (BG_RING - 1 rows in flight); the six step phases name them
+constexpr int BG_RING = 6;           // ring slots per warp (BG_RING - 1 rows in flight), a multiple of 6: the step
+                                     // phases (3-row and 2-row rotations of the register state) name the slots
+static_assert(BG_RING % 6 == 0, "ring slots are named by the step phase");
 constexpr int BG_COLS = 120;         // columns of g per warp
 constexpr int BG_SMS = 148;
 constexpr int BG_BLOCKS_PER_SM = 2;
@@ -46,10 +48,10 @@ struct BParams {
     double* partials;                // [B][nslot][3]: sum res^2, sum (u - u0)^2 on row 0, sum u^2 on column 0
 };
 
-// 16-byte asynchronous copy into the ring slot at byte offset OFF of smem_base; reads nothing and writes zeros when !valid.
+// 16-byte asynchronous copy into the ring slot at byte offset OFF of smem_base: n = 16 bytes are read from gsrc, or
+// n = 0 and the slot is filled with zeros.
 template <int OFF>
-__device__ __forceinline__ void cp_async16_zfill(unsigned smem_base, const float* gsrc, bool valid) {
-    const int n = valid ? 16 : 0;
+__device__ __forceinline__ void cp_async16_zfill(unsigned smem_base, const float* gsrc, int n) {
     asm volatile("cp.async.cg.shared.global [%0+%3], [%1], 16, %2;" ::"r"(smem_base), "l"(gsrc), "r"(n), "n"(OFF) : "memory");
 }
 __device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -65,14 +67,15 @@ struct MarchCtx {
     const float* ub;                 // this sample's field
     const float* psrc;               // this lane's four columns of the row that is copied next
     float* pg;                       // this lane's four columns of the row of g that is stored next
-    const float4* ring;              // this lane's entry of ring slot 0
-    unsigned ring_s;                 // the same as a shared-space address
+    unsigned ring_s;                 // this lane's entry of ring slot 0 (shared-space address)
     int nt_lane;                     // nt, or a negative number for lanes past the field (nothing to copy)
+    int src_stride, src_bytes;       // nx and 16, or 0 and 0 for lanes past the field
     int j0, j1;
     bool store;                      // this lane's four columns exist and belong to this warp's range
     bool col0, colN;                 // this lane's first column is x = 0 / its last column is x = nx-1
     int nx;
-    float ct, cx, s, bts;            // s = 2 hx ht gL;  bts = lambda 2 ht gL
+    float ct, cx, s;                 // s = 2 hx ht gL
+    float bts0, m0;                  // lambda 2 ht gL and 1 in the lane that holds column x = 0, else 0 and 0
     float ef, ebf;                   // running sums of res^2 and of u(0,t)^2 since the last flush
     double e, ebt;
 };
@@ -84,13 +87,21 @@ __device__ __forceinline__ void march_step(MarchState& S, MarchCtx& C, int n) {
     constexpr int iu = PH % 3, ic = (PH + 2) % 3, im = (PH + 1) % 3;
     constexpr int p0 = PH % 2, p1 = 1 - p0;
     cp_wait<BG_RING - 2>();
-    const float4 v = C.ring[PH * 32];
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+%5];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(C.ring_s), "n"(PH * 512) : "memory");
     {
-        const int nn = n + BG_RING - 1;                         // the slot of row n-1 is free again
-        const bool ok = EDGE ? (nn >= 0 && nn < C.nt_lane) : (nn < C.nt_lane);
-        cp_async16_zfill<((PH + BG_RING - 1) % BG_RING) * 512>(C.ring_s, ok ? C.psrc : C.ub, ok);
+        // row n + BG_RING - 1 goes to the slot that row n-1 has just left; away from the edges that row exists
+        constexpr int off = ((PH + BG_RING - 1) % BG_RING) * 512;
+        if (EDGE) {
+            const int nn = n + BG_RING - 1;
+            const bool ok = nn >= 0 && nn < C.nt_lane;
+            cp_async16_zfill<off>(C.ring_s, ok ? C.psrc : C.ub, ok ? 16 : 0);
+        } else {
+            cp_async16_zfill<off>(C.ring_s, C.psrc, C.src_bytes);
+        }
         cp_commit();
-        C.psrc += C.nx;
+        C.psrc += C.src_stride;
     }
     S.u[iu][1] = v.x; S.u[iu][2] = v.y; S.u[iu][3] = v.z; S.u[iu][4] = v.w;
     S.u[iu][0] = __shfl_up_sync(0xffffffffu, v.w, 1);
@@ -135,16 +146,40 @@ __device__ __forceinline__ void march_step(MarchState& S, MarchCtx& C, int n) {
         S.Ax[p1][c] = axn; S.Db[p1][c] = dbn; S.P[p1][c] = pn;
     }
     const int jr = n - 2;                                       // row of g that is now complete
-    if (C.store && (!EDGE || (jr >= C.j0 && jr < C.j1))) {
-        if (C.col0) {
-            const float w = S.u[im][1];
-            g[0] += C.bts * w;
-            C.ebf += w * w;
-        }
-        if (WANT_G) __stcs(reinterpret_cast<float4*>(C.pg), make_float4(g[0], g[1], g[2], g[3]));
+    if (!EDGE || (jr >= C.j0 && jr < C.j1)) {
+        const float w = S.u[im][1];                             // inflow term of L_b: only the lane with x = 0 has m0, bts0 != 0
+        g[0] = fmaf(C.bts0, w, g[0]);
+        C.ebf = fmaf(w * C.m0, w, C.ebf);
+        if (WANT_G && C.store) __stcs(reinterpret_cast<float4*>(C.pg), make_float4(g[0], g[1], g[2], g[3]));
     }
     C.pg += C.nx;
 }
+
+__device__ __forceinline__ void flush_sums(MarchCtx& C) {
+    C.e += (double)C.ef; C.ef = 0.0f;
+    C.ebt += (double)C.ebf; C.ebf = 0.0f;
+}
+
+// COUNT consecutive steps starting in phase K (mod BG_RING) at row n, unrolled at compile time.
+template <int K, int COUNT, bool EDGE, bool WANT_G>
+struct StepSeq {
+    static __device__ __forceinline__ void run(MarchState& S, MarchCtx& C, int n) {
+        march_step<K % BG_RING, EDGE, WANT_G>(S, C, n);
+        StepSeq<K + 1, COUNT - 1, EDGE, WANT_G>::run(S, C, n + 1);
+    }
+    // the same, stopping in front of row nend; advances n; false once nend has been reached
+    static __device__ __forceinline__ bool run_until(MarchState& S, MarchCtx& C, int& n, int nend) {
+        if (n >= nend) return false;
+        march_step<K % BG_RING, EDGE, WANT_G>(S, C, n);
+        ++n;
+        return StepSeq<K + 1, COUNT - 1, EDGE, WANT_G>::run_until(S, C, n, nend);
+    }
+};
+template <int K, bool EDGE, bool WANT_G>
+struct StepSeq<K, 0, EDGE, WANT_G> {
+    static __device__ __forceinline__ void run(MarchState&, MarchCtx&, int) {}
+    static __device__ __forceinline__ bool run_until(MarchState&, MarchCtx&, int&, int) { return true; }
+};
 
 template <bool WANT_G>
 __global__ void __launch_bounds__(BG_WARPS * 32, BG_BLOCKS_PER_SM) burgers_march_kernel(BParams Q) {
@@ -168,10 +203,13 @@ __global__ void __launch_bounds__(BG_WARPS * 32, BG_BLOCKS_PER_SM) burgers_march
     C.colN = xl + 4 == Q.nx;
     C.ub = Q.u + (size_t)bi * Q.nt * Q.nx;
     float* const gb = WANT_G ? Q.g + (size_t)bi * Q.nt * Q.nx : nullptr;
-    C.ring = &ring_all[warp][0][lane];
-    C.ring_s = (unsigned)__cvta_generic_to_shared(C.ring);
+    C.ring_s = (unsigned)__cvta_generic_to_shared(&ring_all[warp][0][lane]);
     const float gl = Q.gL ? Q.gL[bi] : 1.0f;
-    C.ct = Q.ct; C.cx = Q.cx; C.s = xvalid ? Q.w2 * gl : 0.0f; C.bts = Q.bt * gl;
+    C.src_stride = xvalid ? Q.nx : 0;
+    C.src_bytes = xvalid ? 16 : 0;
+    C.ct = Q.ct; C.cx = Q.cx; C.s = xvalid ? Q.w2 * gl : 0.0f;
+    C.bts0 = C.col0 ? Q.bt * gl : 0.0f;
+    C.m0 = C.col0 ? 1.0f : 0.0f;
     C.e = 0.0; C.ebt = 0.0; C.ef = 0.0f; C.ebf = 0.0f;
 
     MarchState S;
@@ -187,7 +225,7 @@ __global__ void __launch_bounds__(BG_WARPS * 32, BG_BLOCKS_PER_SM) burgers_march
     // Rows n = nbeg .. nend-1 are walked.  Steps with  j0 + 2 <= n < min(j1 + 1, nt),  whose copy also stays at or
     // after row 0, touch no edge of the field or of the chunk.
     const int nbeg = C.j0 - 2, nend = C.j1 + 2;
-    const int nfull0 = C.j0 + 2, nfull1 = min(C.j1 + 1, Q.nt);
+    const int nfull1 = min(C.j1 + 1, Q.nt);
     {
         const float* p = C.ub + ((long long)nbeg * Q.nx + xl);  // not dereferenced unless the row exists
 #pragma unroll
@@ -195,27 +233,26 @@ __global__ void __launch_bounds__(BG_WARPS * 32, BG_BLOCKS_PER_SM) burgers_march
             const int nn = nbeg + d;
             const bool ok = nn >= 0 && nn < C.nt_lane;
             const unsigned dst = C.ring_s + d * 512;
-            cp_async16_zfill<0>(dst, ok ? p : C.ub, ok);
+            cp_async16_zfill<0>(dst, ok ? p : C.ub, ok ? 16 : 0);
             cp_commit();
             p += Q.nx;
         }
-        C.psrc = p;
+        C.psrc = xvalid ? p : C.ub;
         C.pg = gb + ((long long)(nbeg - 2) * Q.nx + xl);
     }
+    // The first four steps (two rows to fill the registers, one residual row below the chunk, one row without a
+    // complete g) and the last few take the EDGE variant; in between, groups of BG_RING edge-free steps run unchecked.
     int n = nbeg;
-#define DN_BG_STEP(PH)                                                      \
-    if (n >= nend) break;                                                   \
-    if (n >= nfull0 && n < nfull1) march_step<PH, false, WANT_G>(S, C, n);  \
-    else march_step<PH, true, WANT_G>(S, C, n);                             \
-    ++n;
-    while (true) {
-        DN_BG_STEP(0) DN_BG_STEP(1) DN_BG_STEP(2) DN_BG_STEP(3) DN_BG_STEP(4) DN_BG_STEP(5)
-        C.e += (double)C.ef; C.ef = 0.0f;
-        C.ebt += (double)C.ebf; C.ebf = 0.0f;
+    StepSeq<0, 4, true, WANT_G>::run(S, C, n);
+    n += 4;
+    const int nmain1 = min(nfull1, Q.nt - (BG_RING - 1));       // ... and their copies stay inside the field
+    while (n + BG_RING <= nmain1) {
+        StepSeq<4, BG_RING, false, WANT_G>::run(S, C, n);
+        n += BG_RING;
+        flush_sums(C);
     }
-#undef DN_BG_STEP
-    C.e += (double)C.ef;
-    C.ebt += (double)C.ebf;
+    while (StepSeq<4, BG_RING, true, WANT_G>::run_until(S, C, n, nend)) flush_sums(C);
+    flush_sums(C);
     if (!C.store) C.e = 0.0;
     cp_wait<0>();                                               // copies issued past the last row (zero-fill or unused rows)
 
