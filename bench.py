@@ -42,6 +42,8 @@ NCU_CAPTURES = {
                                           "src": "dn_tiled2d.cu", "sha": "b475340dd3ea795f"},
     "tiled3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 571209216, "fp32_ops_per_element": 155.8,
                                         "src": "dn_tiled3d.cu", "sha": "a93b60c4b75b77cd"},
+    "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
+                                    "src": "dn_burgers.cu", "sha": "baf4524ba7aede8d"},
 }
 
 
