@@ -31,3 +31,27 @@ def energy(u: torch.Tensor, problem: B.Problem, workspace: torch.Tensor = None) 
     if workspace is None:
         workspace = B.new_workspace(problem)
     return _Energy.apply(u, problem, workspace)
+
+
+class _BurgersLoss(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, u, problem, workspace):
+        u = u.contiguous()
+        L = torch.empty(problem.batch, dtype=torch.float32, device=u.device)
+        g = torch.empty_like(u)
+        B.dn_burgers_loss_grad(problem, u, None, L, None, g, workspace)
+        ctx.save_for_backward(g)
+        return L
+
+    @staticmethod
+    def backward(ctx, grad_L):
+        (g,) = ctx.saved_tensors
+        return grad_L.reshape(-1, 1, 1).to(g.dtype) * g, None, None
+
+
+def burgers_loss(u: torch.Tensor, problem: B.Burgers, workspace: torch.Tensor = None) -> torch.Tensor:
+    """L[b] = L_p + lambda L_b of the Burgers finite-difference loss for a batch of fields u [B][nt][nx]
+    (contiguous float32 CUDA tensor); differentiable with respect to u."""
+    if workspace is None:
+        workspace = B.new_burgers_workspace(problem)
+    return _BurgersLoss.apply(u, problem, workspace)
