@@ -164,6 +164,23 @@ dn_status dn_energy_grad_host(const dn_problem* problem, const float* u_host, co
                               float* J_host, float* r_host, void* staging, size_t staging_bytes,
                               void* stream);
 
+/* ---- The discrete FEM solution by matrix-free conjugate gradients ----------------------------------
+ * The conventional-solver side of the paper's comparison ("Mathematical preliminaries": the PDE is usually
+ * discretised and solved; the appendix sets the generator's fields against such solutions): solves
+ * K(nu) u = F on the free nodes with u = bc_x0 / bc_x1 on the Dirichlet faces, by Jacobi-preconditioned
+ * conjugate gradients whose operator is the fused energy+residual kernel of dn_energy_grad.  The result is
+ * the minimiser of J, i.e. the lower bound of the loss a generator can reach for this nu.
+ *  - u_inout: [B][nz][ny][nx]; its interior is the initial guess, its Dirichlet faces are overwritten.
+ *  - Exactly max_iters iterations are enqueued (nothing is read back); a sample whose residual norm has
+ *    fallen to rtol times its initial value stops changing.  relres_out: [B] floats = |r| / |r0| reached,
+ *    iters_out: [B] int32 = iterations a sample took part in; either may be NULL.
+ *  - problem->flags: DN_FORCE_GENERIC is honoured, the other flags are ignored.
+ *  - workspace: dn_cg_workspace_bytes(problem) bytes (four fields + dn_workspace_bytes), 256-byte aligned. */
+size_t dn_cg_workspace_bytes(const dn_problem* problem);
+dn_status dn_cg_solve(const dn_problem* problem, float* u_inout, int32_t max_iters, float rtol,
+                      float* relres_out, int32_t* iters_out, void* workspace, size_t workspace_bytes,
+                      void* stream);
+
 /* ---- The paper's own example: finite-difference loss of the inviscid Burgers equation ------------
  *
  *        u_t + u u_x = 0 on (x,t) in [0,1] x [0,T],   u(x,0) = (1 - cos(2 pi c x)) / 2

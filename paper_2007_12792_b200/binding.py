@@ -31,7 +31,7 @@ DN_MAX_KL_MODES = 8
 EXPORTS = ("dn_workspace_bytes", "dn_host_staging_bytes", "dn_kl_field", "dn_energy", "dn_energy_grad",
            "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced", "dn_energy_grad_static", "dn_launches_per_call", "dn_path_name", "dn_status_string",
            "dn_burgers_workspace_bytes", "dn_burgers_loss_grad", "dn_burgers_path_name",
-           "dn_burgers_host_staging_bytes", "dn_burgers_loss_grad_host")
+           "dn_burgers_host_staging_bytes", "dn_burgers_loss_grad_host", "dn_cg_workspace_bytes", "dn_cg_solve")
 
 
 class DnGrid(C.Structure):
@@ -84,6 +84,10 @@ def lib():
         L.dn_launches_per_call.argtypes = [PP]; L.dn_launches_per_call.restype = C.c_int32
         L.dn_path_name.argtypes = [PP]; L.dn_path_name.restype = C.c_char_p
         L.dn_status_string.argtypes = [C.c_int]; L.dn_status_string.restype = C.c_char_p
+        L.dn_cg_workspace_bytes.argtypes = [PP]; L.dn_cg_workspace_bytes.restype = C.c_size_t
+        L.dn_cg_solve.argtypes = [PP, C.c_void_p, C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                  C.c_void_p]
+        L.dn_cg_solve.restype = C.c_int
         PB = C.POINTER(DnBurgers)
         L.dn_burgers_workspace_bytes.argtypes = [PB]; L.dn_burgers_workspace_bytes.restype = C.c_size_t
         L.dn_burgers_loss_grad.argtypes = [PB, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -325,3 +329,24 @@ def dn_burgers_loss_grad_host(problem: Burgers, u_host: torch.Tensor, gL_host: O
                                            _ptr(g_host, "g_host", "cpu"), staging.data_ptr(), staging.numel(),
                                            _stream(stream)), "dn_burgers_loss_grad_host")
     return L_host, parts_host, g_host
+
+
+def dn_cg_workspace_bytes(problem: Problem) -> int:
+    return int(lib().dn_cg_workspace_bytes(C.byref(problem.c_struct(device="any"))))
+
+
+def new_cg_workspace(problem: Problem, device="cuda") -> torch.Tensor:
+    return torch.empty(max(dn_cg_workspace_bytes(problem), 256), dtype=torch.uint8, device=device)
+
+
+def dn_cg_solve(problem: Problem, u: torch.Tensor, max_iters: int, rtol: float, relres: Optional[torch.Tensor],
+                iters: Optional[torch.Tensor], workspace: torch.Tensor, stream=None):
+    """Solves K(nu) u = F in place (matrix-free Jacobi-preconditioned CG on the fused kernel); relres: [B] float32,
+    iters: [B] int32 device tensors or None.  Enqueues exactly max_iters iterations."""
+    if iters is not None and (iters.dtype != torch.int32 or not iters.is_cuda or not iters.is_contiguous()):
+        raise ValueError("iters: expected a contiguous int32 CUDA tensor")
+    p = problem.c_struct()
+    _check(lib().dn_cg_solve(C.byref(p), _ptr(u, "u"), int(max_iters), float(rtol), _ptr(relres, "relres"),
+                             None if iters is None else iters.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                             _stream(stream)), "dn_cg_solve")
+    return u

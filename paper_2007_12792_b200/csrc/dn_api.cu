@@ -146,6 +146,35 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
     return DN_OK;
 }
 
+dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, size_t ws_bytes, cudaStream_t s,
+                       bool build_tables, const double** partials, int* nblk, Params* P_out) {
+    dn_status st = validate(p);
+    if (st != DN_OK) return st;
+    if (!u || !r) return DN_ERR_NULL;
+    const Launch l = choose_launch(*p, u, r);
+    const WsLayout w = make_layout(*p, l, false);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign) != 0 || ws_bytes < w.total) return DN_ERR_WORKSPACE;
+    Params P = make_params(*p, w, u, nullptr, r, ws);
+    cudaError_t e = cudaSuccess;
+    if (build_tables && p->nu_mode != DN_NU_NODAL) {
+        char* base = static_cast<char*>(ws);
+        float* cg[3] = {reinterpret_cast<float*>(base + w.cg[0]), reinterpret_cast<float*>(base + w.cg[1]),
+                        reinterpret_cast<float*>(base + w.cg[2])};
+        float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
+                        reinterpret_cast<float*>(base + w.cn[2])};
+        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s);
+        if (e != cudaSuccess) return DN_ERR_CUDA;
+    }
+    if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
+    else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
+    else e = launch_generic(P, s);
+    if (e != cudaSuccess) return DN_ERR_CUDA;
+    if (partials) *partials = P.partials;
+    if (nblk) *nblk = w.nblk;
+    if (P_out) *P_out = P;
+    return DN_OK;
+}
+
 dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
                     size_t ws_bytes, void* stream) {
     if (!r) return DN_ERR_NULL;
