@@ -147,7 +147,7 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
 }
 
 dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, size_t ws_bytes, cudaStream_t s,
-                       bool build_tables, const double** partials, int* nblk, Params* P_out) {
+                       bool build_tables, const double** partials, int* nblk) {
     dn_status st = validate(p);
     if (st != DN_OK) return st;
     if (!u || !r) return DN_ERR_NULL;
@@ -171,7 +171,6 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
     if (e != cudaSuccess) return DN_ERR_CUDA;
     if (partials) *partials = P.partials;
     if (nblk) *nblk = w.nblk;
-    if (P_out) *P_out = P;
     return DN_OK;
 }
 

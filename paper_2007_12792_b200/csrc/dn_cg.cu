@@ -162,6 +162,31 @@ __global__ void __launch_bounds__(CG_THREADS) cg_direction_kernel(long long node
         p[base + i] = fmaf(beta, p[base + i], r[base + i] * dinv[base + i]);
 }
 
+// ---- diagonal of K by probing ------------------------------------------------------------------------
+// Nodes whose indices agree modulo 3 on every axis share no element, so the fused kernel applied to the
+// indicator of one such colour class returns K_ii at the nodes i of that class: 3^dim applications give the
+// whole diagonal.  One block per x-row; only the rows of the class (iy, iz congruent to the colour) do work.
+// phase 0: e = 1 on the free nodes of the class in this row, 0 elsewhere in the row (e is zero outside the class rows).
+// phase 1: dinv = 1 / (K e) on the free nodes of the class, 0 on its Dirichlet nodes; the row of e is cleared again.
+__global__ void __launch_bounds__(CG_THREADS) cg_probe_kernel(int nx, int ny, int nz, int colour, int phase,
+                                                              float* __restrict__ e, const float* __restrict__ q,
+                                                              float* __restrict__ dinv) {
+    const long long row = blockIdx.x;
+    const int iy = (int)(row % ny), iz = (int)((row / ny) % nz);
+    const int cx = colour % 3, cy = (colour / 3) % 3, cz = colour / 9;
+    if (iy % 3 != cy || iz % 3 != cz) return;
+    const long long base = row * nx;
+    for (int ix = threadIdx.x; ix < nx; ix += CG_THREADS) {
+        const bool mine = ix % 3 == cx, face = ix == 0 || ix == nx - 1;
+        if (phase == 0) {
+            e[base + ix] = (mine && !face) ? 1.0f : 0.0f;
+        } else {
+            if (mine) dinv[base + ix] = face ? 0.0f : 1.0f / q[base + ix];
+            e[base + ix] = 0.0f;
+        }
+    }
+}
+
 __global__ void cg_report_kernel(const CgScalars* __restrict__ sc, int batch, float* __restrict__ relres,
                                  int32_t* __restrict__ iters) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -231,22 +256,34 @@ dn_status dn_cg_solve(const dn_problem* p, float* u, int32_t max_iters, float rt
     if (st != DN_OK) return st;
     dn_problem p1 = *p;
     p1.flags &= ~(DN_NO_MASK | DN_IMPOSE_BC_ON_LOAD);
-    Params P{};
-    st = run_operator(&p1, u, r, op_ws, op_bytes, s, true, nullptr, nullptr, &P);
+    st = run_operator(&p1, u, r, op_ws, op_bytes, s, true, nullptr, nullptr);
     if (st != DN_OK) return st;
-    if (launch_diag_inverse(P, dinv, s) != cudaSuccess) return DN_ERR_CUDA;
-    cg_init_kernel<<<vgrid, CG_THREADS, 0, s>>>(nodes, nvb, r, dinv, pd, partials);
-    cg_start_kernel<<<p->batch, CG_THREADS, 0, s>>>(partials, nvb, sc);
-    if (cudaGetLastError() != cudaSuccess) return DN_ERR_CUDA;
 
     // the operator on directions: zero forcing, zero boundary values, same diffusivity (tables stay valid)
     dn_problem p0 = p1;
     p0.f = nullptr; p0.f_const = 0.0f; p0.bc_x0 = 0.0f; p0.bc_x1 = 0.0f;
+    {   // Jacobi preconditioner: the diagonal of K, one colour class per application (p and q serve as scratch)
+        const int nz = p->grid.dim == 3 ? p->grid.nz : 1;
+        const unsigned rows = (unsigned)((long long)p->batch * nz * p->grid.ny);
+        const int ncol = p->grid.dim == 3 ? 27 : 9;
+        if (cudaMemsetAsync(pd, 0, sizeof(float) * (size_t)nodes * p->batch, s) != cudaSuccess) return DN_ERR_CUDA;
+        for (int c = 0; c < ncol; ++c) {
+            cg_probe_kernel<<<rows, CG_THREADS, 0, s>>>(p->grid.nx, p->grid.ny, nz, c, 0, pd, nullptr, nullptr);
+            st = run_operator(&p0, pd, q, op_ws, op_bytes, s, false, nullptr, nullptr);
+            if (st != DN_OK) return st;
+            cg_probe_kernel<<<rows, CG_THREADS, 0, s>>>(p->grid.nx, p->grid.ny, nz, c, 1, pd, q, dinv);
+        }
+        if (cudaGetLastError() != cudaSuccess) return DN_ERR_CUDA;
+    }
+    cg_init_kernel<<<vgrid, CG_THREADS, 0, s>>>(nodes, nvb, r, dinv, pd, partials);
+    cg_start_kernel<<<p->batch, CG_THREADS, 0, s>>>(partials, nvb, sc);
+    if (cudaGetLastError() != cudaSuccess) return DN_ERR_CUDA;
+
     const double rtol2 = (double)rtol * (double)rtol;
     for (int it = 0; it < max_iters; ++it) {
         const double* op_partials = nullptr;
         int op_nblk = 0;
-        st = run_operator(&p0, pd, q, op_ws, op_bytes, s, false, &op_partials, &op_nblk, nullptr);
+        st = run_operator(&p0, pd, q, op_ws, op_bytes, s, false, &op_partials, &op_nblk);
         if (st != DN_OK) return st;
         cg_alpha_kernel<<<p->batch, CG_THREADS, 0, s>>>(op_partials, op_nblk, sc);
         cg_update_kernel<<<vgrid, CG_THREADS, 0, s>>>(nodes, nvb, u, r, pd, q, dinv, sc, partials);

@@ -66,14 +66,13 @@ __device__ __forceinline__ float kl_node(const Params& P, const float* c, int ix
 // t = u11-u10-u01+u00, the x-derivative at the Gauss row eta is (e0 + eta t)/hx and the
 // y-derivative at the Gauss column xi is (s0 + xi t)/hy; the energy is a function of
 // (e0, s0, t) and the chain rule distributes its three partial derivatives to the corners.
-// ub == nullptr: the corner values are taken from uc[4] instead of the field (used for the diagonal of K).
 __device__ __forceinline__ void element2d(const Params& P, int b, int ex, int ey, const float* ub,
                                           const float* nub, const float* fb, const float* c,
-                                          float rc[4], float& ed, float& el, const float* uc = nullptr) {
+                                          float rc[4], float& ed, float& el) {
     const int nx = P.nx;
     const long long i00 = (long long)ey * nx + ex;
-    const float u00 = ub ? load_u(P, ub, ex, i00) : uc[0], u10 = ub ? load_u(P, ub, ex + 1, i00 + 1) : uc[1];
-    const float u01 = ub ? load_u(P, ub, ex, i00 + nx) : uc[2], u11 = ub ? load_u(P, ub, ex + 1, i00 + nx + 1) : uc[3];
+    const float u00 = load_u(P, ub, ex, i00), u10 = load_u(P, ub, ex + 1, i00 + 1);
+    const float u01 = load_u(P, ub, ex, i00 + nx), u11 = load_u(P, ub, ex + 1, i00 + nx + 1);
     const float ga[2] = {DN_GA, DN_GB};
     float nuq[2][2];                                   // [p: xi point][q: eta point]
     if (P.nu_mode != DN_NU_KL_GAUSS) {
@@ -133,13 +132,13 @@ __device__ __forceinline__ void element2d(const Params& P, int b, int ex, int ey
 // per direction, which are distributed back to the edges with the same bilinear weights.
 __device__ __forceinline__ void element3d(const Params& P, int b, int ex, int ey, int ez, const float* ub,
                                           const float* nub, const float* fb, const float* c,
-                                          float rc[8], float& ed, float& el, const float* uc = nullptr) {
+                                          float rc[8], float& ed, float& el) {
     const int nx = P.nx;
     const long long sy = nx, sz = (long long)nx * P.ny;
     const long long i0 = ((long long)ez * P.ny + ey) * nx + ex;
     float u[8];
     for (int a = 0; a < 8; ++a)
-        u[a] = ub ? load_u(P, ub, ex + (a & 1), i0 + (a & 1) + ((a >> 1) & 1) * sy + ((a >> 2) & 1) * sz) : uc[a];
+        u[a] = load_u(P, ub, ex + (a & 1), i0 + (a & 1) + ((a >> 1) & 1) * sy + ((a >> 2) & 1) * sz);
     const float ga[2] = {DN_GA, DN_GB};
     const float L[2][2] = {{1.f - DN_GA, DN_GA}, {1.f - DN_GB, DN_GB}};   // L[point][corner bit]
     float nuq[2][2][2];                                                     // [p: xi][q: eta][s: zeta]
@@ -261,47 +260,7 @@ __global__ void __launch_bounds__(GEN_THREADS) generic_kernel(const Params P) {
     block_reduce_store(ed_acc, el_acc, P.partials + 2 * ((long long)b * P.nblk + blockIdx.x));
 }
 
-// Diagonal of K(nu): entry i is the response at node i to a unit value at node i, summed over the adjacent
-// elements (each element's own diagonal entry comes from the element routine applied to a unit corner vector).
-// Written as its reciprocal, 0 at the Dirichlet nodes: the Jacobi preconditioner of the conjugate-gradient solver.
-template <int DIM>
-__global__ void __launch_bounds__(GEN_THREADS) diag_inverse_kernel(Params P, float* __restrict__ dinv) {
-    const int b = blockIdx.y;
-    const long long node = (long long)blockIdx.x * GEN_THREADS + threadIdx.x;
-    if (node >= P.nodes) return;
-    P.f_const = 0.0f;
-    const float* nub = P.nu ? P.nu + (long long)b * P.nodes : nullptr;
-    long long mpow = 1;
-    for (int a = 0; a < DIM; ++a) mpow *= P.m;
-    const float* c = P.ckl + (long long)b * mpow;
-    const int ix = (int)(node % P.nx);
-    const int iy = (int)((node / P.nx) % P.ny);
-    const int iz = (int)(node / ((long long)P.nx * P.ny));
-    float d = 0.f;
-    for (int dz = (DIM == 3 ? -1 : 0); dz <= 0; ++dz)
-        for (int dy = -1; dy <= 0; ++dy)
-            for (int dx = -1; dx <= 0; ++dx) {
-                const int ex = ix + dx, ey = iy + dy, ez = iz + dz;
-                if (ex < 0 || ex >= P.nx - 1 || ey < 0 || ey >= P.ny - 1) continue;
-                if (DIM == 3 && (ez < 0 || ez >= P.nz - 1)) continue;
-                const int corner = (-dx) | ((-dy) << 1) | ((DIM == 3 ? -dz : 0) << 2);
-                float uc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, rc[8], ed, el;
-                uc[corner] = 1.0f;
-                if (DIM == 2) element2d(P, b, ex, ey, nullptr, nub, nullptr, c, rc, ed, el, uc);
-                else element3d(P, b, ex, ey, ez, nullptr, nub, nullptr, c, rc, ed, el, uc);
-                d += rc[corner];
-            }
-    dinv[(long long)b * P.nodes + node] = (ix == 0 || ix == P.nx - 1) ? 0.0f : 1.0f / d;
-}
-
 }  // namespace
-
-cudaError_t launch_diag_inverse(const Params& P, float* dinv, cudaStream_t s) {
-    dim3 grid((unsigned)generic_blocks_per_sample(P.nodes), (unsigned)P.batch);
-    if (P.dim == 2) diag_inverse_kernel<2><<<grid, GEN_THREADS, 0, s>>>(P, dinv);
-    else diag_inverse_kernel<3><<<grid, GEN_THREADS, 0, s>>>(P, dinv);
-    return cudaGetLastError();
-}
 
 int generic_blocks_per_sample(long long nodes) { return (int)((nodes + GEN_THREADS - 1) / GEN_THREADS); }
 

@@ -70,15 +70,13 @@ dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float*
                     size_t ws_bytes, void* stream);
 // The fused kernel alone, for callers that apply the operator repeatedly: no energy finaliser; the KL tables are
 // built only when build_tables is set (they depend on the problem, not on u); *partials / *nblk tell where the
-// kernel left its per-block energy pairs (diffusion part, load part), [batch][*nblk][2] doubles; *P_out receives
-// the kernel parameters (for launch_diag_inverse).
+// kernel left its per-block energy pairs (diffusion part, load part), [batch][*nblk][2] doubles.
 dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, size_t ws_bytes, cudaStream_t s,
-                       bool build_tables, const double** partials, int* nblk, Params* P_out);
+                       bool build_tables, const double** partials, int* nblk);
 
 cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], float* const cn[3],
                           cudaStream_t s);
 cudaError_t launch_generic(const Params& P, cudaStream_t s);
-cudaError_t launch_diag_inverse(const Params& P, float* dinv, cudaStream_t s);   // needs the KL tables of P
 cudaError_t launch_tiled2d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s);
