@@ -33,8 +33,8 @@ def test_loss_of_a_linear_field_closed_form():
     hx, ht = 1.0 / (nx - 1), T / (nt - 1)
     res = c + (a + b * x + c * t) * b                                      # u_t + u u_x typed out
     Lp = hx * ht * (res[1:-1, 1:-1] ** 2).sum()
-    cpar = np.array([2.0])
-    u0 = 0.5 * (1 - np.cos(2 * np.pi * 2.0 * x[0]))
+    cpar = np.array([2.3])                                                 # not an integer: sums over whole periods would hide a wrong frequency
+    u0 = 0.5 * (1 - np.cos(2 * np.pi * 2.3 * x[0]))
     Lb = hx * ((u[0, 0] - u0) ** 2).sum() + ht * (u[0, :, 0] ** 2).sum()
     L, Lp_o, Lb_o, g = ob.loss_grad(u, cpar, T=T, lam=0.7)
     assert Lp_o[0] == pytest.approx(Lp, rel=1e-13) and Lb_o[0] == pytest.approx(Lb, rel=1e-13)
