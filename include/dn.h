@@ -87,6 +87,8 @@ typedef struct {
     const float* f;              /* optional nodal forcing [B][nz][ny][nx], Q1-interpolated        */
     float bc_x0, bc_x1;          /* Dirichlet values on x = 0 and x = 1                            */
     uint32_t flags;              /* DN_* flags above                                               */
+    const float* bc_x0_b;        /* optional [B]: per-sample Dirichlet value on x = 0 (the paper samples the  */
+    const float* bc_x1_b;        /* boundary data b per minibatch); each overrides its scalar when non-NULL   */
 } dn_problem;
 
 /* Bytes of device scratch that dn_energy / dn_energy_grad need for this problem (per-block
@@ -154,10 +156,15 @@ dn_status dn_energy_grad_static(const dn_problem* problem, const float* u, const
 dn_status dn_apply_bc(const dn_grid* grid, int32_t batch, float bc_x0, float bc_x1, int32_t mode,
                       float* field_inout, void* stream);
 
+/* dn_apply_bc (mode 0) with one pair of values per sample: field[b] = bc_x0_b[b] at ix = 0 and bc_x1_b[b] at
+ * ix = nx-1.  bc_x0_b, bc_x1_b: [B] floats. */
+dn_status dn_apply_bc_per_sample(const dn_grid* grid, int32_t batch, const float* bc_x0_b, const float* bc_x1_b,
+                                 float* field_inout, void* stream);
+
 /* dn_energy_grad with HOST buffers: copies u (and nu / f / kl_w / gJ when present) to the
  * device staging area, runs the same kernels, copies J and r back, and waits for the last
  * copy.  The batch is pipelined in chunks of whole samples over two internal copy streams (created
- * and destroyed inside the call) so that both directions of the host link overlap with the kernels.  In `problem`, nu / kl_w / f are HOST pointers here.  u_host, r_host: [B][..] floats;
+ * and destroyed inside the call) so that both directions of the host link overlap with the kernels.  In `problem`, nu / kl_w / f / bc_x0_b / bc_x1_b are HOST pointers here.  u_host, r_host: [B][..] floats;
  * J_host: [B] floats or NULL; staging: device memory of dn_host_staging_bytes(problem) bytes,
  * 256-byte aligned.  Use pinned host memory for full copy bandwidth. */
 dn_status dn_energy_grad_host(const dn_problem* problem, const float* u_host, const float* gJ_host,

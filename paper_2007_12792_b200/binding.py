@@ -28,7 +28,7 @@ DN_NO_MASK = 2
 DN_FORCE_GENERIC = 4
 DN_MAX_KL_MODES = 8
 
-EXPORTS = ("dn_workspace_bytes", "dn_host_staging_bytes", "dn_kl_field", "dn_energy", "dn_energy_grad",
+EXPORTS = ("dn_apply_bc_per_sample", "dn_workspace_bytes", "dn_host_staging_bytes", "dn_kl_field", "dn_energy", "dn_energy_grad",
            "dn_apply_bc", "dn_energy_grad_host", "dn_energy_grad_traced", "dn_energy_grad_static", "dn_launches_per_call", "dn_path_name", "dn_status_string",
            "dn_burgers_workspace_bytes", "dn_burgers_loss_grad", "dn_burgers_path_name",
            "dn_burgers_host_staging_bytes", "dn_burgers_loss_grad_host", "dn_cg_workspace_bytes", "dn_cg_solve")
@@ -43,6 +43,7 @@ class DnProblem(C.Structure):
         ("grid", DnGrid), ("batch", C.c_int32), ("nu_mode", C.c_int32), ("nu", C.c_void_p),
         ("kl_modes", C.c_int32), ("kl_w", C.c_void_p), ("f_const", C.c_float), ("f", C.c_void_p),
         ("bc_x0", C.c_float), ("bc_x1", C.c_float), ("flags", C.c_uint32),
+        ("bc_x0_b", C.c_void_p), ("bc_x1_b", C.c_void_p),
     ]
 
 
@@ -80,6 +81,8 @@ def lib():
         L.dn_energy_grad_static.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.dn_energy_grad_static.restype = C.c_int
         L.dn_apply_bc.argtypes = [PG, C.c_int32, C.c_float, C.c_float, C.c_int32, C.c_void_p, C.c_void_p]
+        L.dn_apply_bc_per_sample.argtypes = [PG, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.dn_apply_bc_per_sample.restype = C.c_int
         L.dn_energy_grad_host.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.dn_launches_per_call.argtypes = [PP]; L.dn_launches_per_call.restype = C.c_int32
         L.dn_path_name.argtypes = [PP]; L.dn_path_name.restype = C.c_char_p
@@ -145,6 +148,8 @@ class Problem:
     bc_x0: float = 1.0
     bc_x1: float = 0.0
     flags: int = 0
+    bc_x0_b: Optional[torch.Tensor] = None      # [B] per-sample Dirichlet values; override the scalars
+    bc_x1_b: Optional[torch.Tensor] = None
 
     @property
     def shape(self):
@@ -161,6 +166,8 @@ class Problem:
         p.kl_w = _ptr(self.kl_w, "kl_w", device)
         p.f = _ptr(self.f, "f", device)
         p.f_const, p.bc_x0, p.bc_x1, p.flags = self.f_const, self.bc_x0, self.bc_x1, self.flags
+        p.bc_x0_b = _ptr(self.bc_x0_b, "bc_x0_b", device)
+        p.bc_x1_b = _ptr(self.bc_x1_b, "bc_x1_b", device)
         return p
 
 
@@ -247,6 +254,14 @@ def dn_apply_bc(dim: int, nx: int, ny: int, nz: int, batch: int, bc_x0: float, b
                 field: torch.Tensor, stream=None) -> torch.Tensor:
     g = DnGrid(dim, nx, ny, nz if dim == 3 else 1)
     _check(lib().dn_apply_bc(C.byref(g), batch, bc_x0, bc_x1, mode, _ptr(field, "field"), _stream(stream)), "dn_apply_bc")
+    return field
+
+
+def dn_apply_bc_per_sample(dim: int, nx: int, ny: int, nz: int, batch: int, bc_x0_b: torch.Tensor, bc_x1_b: torch.Tensor,
+                           field: torch.Tensor, stream=None) -> torch.Tensor:
+    g = DnGrid(dim, nx, ny, nz if dim == 3 else 1)
+    _check(lib().dn_apply_bc_per_sample(C.byref(g), batch, _ptr(bc_x0_b, "bc_x0_b"), _ptr(bc_x1_b, "bc_x1_b"),
+                                        _ptr(field, "field"), _stream(stream)), "dn_apply_bc_per_sample")
     return field
 
 

@@ -95,6 +95,7 @@ static Params make_params(const dn_problem& p, const WsLayout& w, const float* u
     P.hx = (float)(1.0 / (P.nx - 1)); P.hy = (float)(1.0 / (P.ny - 1));
     P.hz = (P.dim == 3) ? (float)(1.0 / (P.nz - 1)) : 1.0f;
     P.u = u; P.nu = p.nu; P.f = p.f; P.gJ = gJ; P.r = r;
+    P.bc0_b = p.bc_x0_b; P.bc1_b = p.bc_x1_b;
     char* base = static_cast<char*>(ws);
     P.partials = reinterpret_cast<double*>(base + w.partials);
     P.ckl = reinterpret_cast<const float*>(base + w.ckl);
@@ -197,7 +198,7 @@ size_t dn_host_staging_bytes(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
     const size_t field = align_up(sizeof(float) * (size_t)p->batch * nodes_per_sample(p->grid));
     size_t total = 2 * field;                                   // u, r
-    total += 2 * align_up(sizeof(float) * (size_t)p->batch);    // J, gJ
+    total += 4 * align_up(sizeof(float) * (size_t)p->batch);    // J, gJ, per-sample boundary values
     if (p->nu_mode == DN_NU_NODAL) total += field;
     if (p->f) total += field;
     size_t mpow = 1;
@@ -245,6 +246,16 @@ dn_status dn_apply_bc(const dn_grid* g, int32_t batch, float b0, float b1, int32
 // The batch is cut into chunks of whole samples that flow through three stages on three streams:
 // host->device copy, kernels (on the caller's stream), device->host copy.  Chunk c+1 is copied in
 // and chunk c-1 copied out while chunk c computes, so both directions of the host link stay busy.
+dn_status dn_apply_bc_per_sample(const dn_grid* g, int32_t batch, const float* b0, const float* b1, float* field,
+                                 void* stream) {
+    if (!g || !field || !b0 || !b1) return DN_ERR_NULL;
+    dn_status st = DN_OK;
+    if (!valid_grid(*g, st)) return st;
+    if (batch < 1 || batch > 65535) return DN_ERR_SIZE;
+    return launch_apply_bc(*g, batch, 0.f, 0.f, 0, field, static_cast<cudaStream_t>(stream), b0, b1) == cudaSuccess
+               ? DN_OK : DN_ERR_CUDA;
+}
+
 dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const float* gJ_host, float* J_host,
                               float* r_host, void* staging, size_t staging_bytes, void* stream) {
     dn_status st = validate(p);
@@ -265,6 +276,8 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
     float* d_r = reinterpret_cast<float*>(base + off); off += field;
     float* d_J = reinterpret_cast<float*>(base + off); off += small;
     float* d_g = reinterpret_cast<float*>(base + off); off += small;
+    float* d_b0 = reinterpret_cast<float*>(base + off); off += small;
+    float* d_b1 = reinterpret_cast<float*>(base + off); off += small;
     float* d_nu = nullptr; float* d_f = nullptr;
     if (p->nu_mode == DN_NU_NODAL) { d_nu = reinterpret_cast<float*>(base + off); off += field; }
     if (p->f) { d_f = reinterpret_cast<float*>(base + off); off += field; }
@@ -289,6 +302,8 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
     if (p->nu_mode != DN_NU_NODAL)
         DN_TRY(cudaMemcpyAsync(d_w, p->kl_w, sizeof(float) * (size_t)p->batch * mpow, cudaMemcpyHostToDevice, pipe.in));
     if (gJ_host) DN_TRY(cudaMemcpyAsync(d_g, gJ_host, sizeof(float) * p->batch, cudaMemcpyHostToDevice, pipe.in));
+    if (p->bc_x0_b) DN_TRY(cudaMemcpyAsync(d_b0, p->bc_x0_b, sizeof(float) * p->batch, cudaMemcpyHostToDevice, pipe.in));
+    if (p->bc_x1_b) DN_TRY(cudaMemcpyAsync(d_b1, p->bc_x1_b, sizeof(float) * p->batch, cudaMemcpyHostToDevice, pipe.in));
     for (int c = 0; c < nchunks; ++c) {
         const int b0 = c * csize;
         const int nb = (b0 + csize <= p->batch) ? csize : p->batch - b0;
@@ -303,6 +318,8 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
         q.nu = d_nu ? d_nu + o : nullptr;
         q.f = d_f ? d_f + o : nullptr;
         q.kl_w = (p->nu_mode != DN_NU_NODAL) ? d_w + (size_t)b0 * mpow : nullptr;
+        q.bc_x0_b = p->bc_x0_b ? d_b0 + b0 : nullptr;
+        q.bc_x1_b = p->bc_x1_b ? d_b1 + b0 : nullptr;
         st = run(&q, d_u + o, gJ_host ? d_g + b0 : nullptr, J_host ? d_J + b0 : nullptr, d_r + o, ws, ws_bytes, s);
         if (st != DN_OK) { cudaStreamSynchronize(pipe.in); cudaStreamSynchronize(s); cudaStreamSynchronize(pipe.out); return st; }
         DN_TRY(cudaEventRecord(pipe.computed[c], s));

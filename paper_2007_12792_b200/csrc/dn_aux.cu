@@ -231,9 +231,13 @@ cudaError_t launch_kl_field_vec(const dn_grid& g, int nz, int batch, int m, cons
     return cudaGetLastError();
 }
 
-__global__ void apply_bc_kernel(long long lines, int nx, float v0, float v1, float* __restrict__ field) {
+__global__ void apply_bc_kernel(long long lines, long long lines_per_sample, int nx, float v0, float v1,
+                                const float* __restrict__ v0_b, const float* __restrict__ v1_b,
+                                float* __restrict__ field) {
     const long long line = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (line >= lines) return;
+    if (v0_b) v0 = v0_b[line / lines_per_sample];
+    if (v1_b) v1 = v1_b[line / lines_per_sample];
     field[line * nx] = v0;
     field[line * nx + nx - 1] = v1;
 }
@@ -269,11 +273,14 @@ cudaError_t launch_kl_field(const dn_grid& g, int batch, int m, const float* kl_
     return vec ? launch_kl_field_vec<4>(g, nz, batch, m, kl_w, nu, s) : launch_kl_field_vec<1>(g, nz, batch, m, kl_w, nu, s);
 }
 
-cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int mode, float* field, cudaStream_t s) {
-    const long long lines = (long long)batch * g.ny * ((g.dim == 3) ? g.nz : 1);
+cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int mode, float* field, cudaStream_t s,
+                            const float* b0_b, const float* b1_b) {
+    const long long per_sample = (long long)g.ny * ((g.dim == 3) ? g.nz : 1);
+    const long long lines = (long long)batch * per_sample;
     const int threads = 256;
     apply_bc_kernel<<<(unsigned)((lines + threads - 1) / threads), threads, 0, s>>>(
-        lines, g.nx, mode == 0 ? b0 : 0.0f, mode == 0 ? b1 : 0.0f, field);
+        lines, per_sample, g.nx, mode == 0 ? b0 : 0.0f, mode == 0 ? b1 : 0.0f, mode == 0 ? b0_b : nullptr,
+        mode == 0 ? b1_b : nullptr, field);
     return cudaGetLastError();
 }
 

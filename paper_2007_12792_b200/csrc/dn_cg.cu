@@ -252,8 +252,9 @@ dn_status dn_cg_solve(const dn_problem* p, float* u, int32_t max_iters, float rt
     const dim3 vgrid((unsigned)nvb, (unsigned)p->batch);
 
     // Dirichlet faces of u take their values; r = K u - F (masked) with the caller's forcing
-    dn_status st = dn_apply_bc(&p->grid, p->batch, p->bc_x0, p->bc_x1, 0, u, stream);
-    if (st != DN_OK) return st;
+    if (launch_apply_bc(p->grid, p->batch, p->bc_x0, p->bc_x1, 0, u, s, p->bc_x0_b, p->bc_x1_b) != cudaSuccess)
+        return DN_ERR_CUDA;
+    dn_status st = DN_OK;
     dn_problem p1 = *p;
     p1.flags &= ~(DN_NO_MASK | DN_IMPOSE_BC_ON_LOAD);
     st = run_operator(&p1, u, r, op_ws, op_bytes, s, true, nullptr, nullptr);
@@ -261,7 +262,7 @@ dn_status dn_cg_solve(const dn_problem* p, float* u, int32_t max_iters, float rt
 
     // the operator on directions: zero forcing, zero boundary values, same diffusivity (tables stay valid)
     dn_problem p0 = p1;
-    p0.f = nullptr; p0.f_const = 0.0f; p0.bc_x0 = 0.0f; p0.bc_x1 = 0.0f;
+    p0.f = nullptr; p0.f_const = 0.0f; p0.bc_x0 = 0.0f; p0.bc_x1 = 0.0f; p0.bc_x0_b = nullptr; p0.bc_x1_b = nullptr;
     {   // Jacobi preconditioner: the diagonal of K, one colour class per application (p and q serve as scratch)
         const int nz = p->grid.dim == 3 ? p->grid.nz : 1;
         const unsigned rows = (unsigned)((long long)p->batch * nz * p->grid.ny);

@@ -11,10 +11,10 @@ namespace {
 
 constexpr int GEN_THREADS = 128;
 
-__device__ __forceinline__ float load_u(const Params& P, const float* ub, int ix, long long idx) {
+__device__ __forceinline__ float load_u(const Params& P, int b, const float* ub, int ix, long long idx) {
     if (P.flags & DN_IMPOSE_BC_ON_LOAD) {
-        if (ix == 0) return P.bc_x0;
-        if (ix == P.nx - 1) return P.bc_x1;
+        if (ix == 0) return P.bc0_b ? __ldg(P.bc0_b + b) : P.bc_x0;
+        if (ix == P.nx - 1) return P.bc1_b ? __ldg(P.bc1_b + b) : P.bc_x1;
     }
     return __ldg(ub + idx);
 }
@@ -71,8 +71,8 @@ __device__ __forceinline__ void element2d(const Params& P, int b, int ex, int ey
                                           float rc[4], float& ed, float& el) {
     const int nx = P.nx;
     const long long i00 = (long long)ey * nx + ex;
-    const float u00 = load_u(P, ub, ex, i00), u10 = load_u(P, ub, ex + 1, i00 + 1);
-    const float u01 = load_u(P, ub, ex, i00 + nx), u11 = load_u(P, ub, ex + 1, i00 + nx + 1);
+    const float u00 = load_u(P, b, ub, ex, i00), u10 = load_u(P, b, ub, ex + 1, i00 + 1);
+    const float u01 = load_u(P, b, ub, ex, i00 + nx), u11 = load_u(P, b, ub, ex + 1, i00 + nx + 1);
     const float ga[2] = {DN_GA, DN_GB};
     float nuq[2][2];                                   // [p: xi point][q: eta point]
     if (P.nu_mode != DN_NU_KL_GAUSS) {
@@ -138,7 +138,7 @@ __device__ __forceinline__ void element3d(const Params& P, int b, int ex, int ey
     const long long i0 = ((long long)ez * P.ny + ey) * nx + ex;
     float u[8];
     for (int a = 0; a < 8; ++a)
-        u[a] = load_u(P, ub, ex + (a & 1), i0 + (a & 1) + ((a >> 1) & 1) * sy + ((a >> 2) & 1) * sz);
+        u[a] = load_u(P, b, ub, ex + (a & 1), i0 + (a & 1) + ((a >> 1) & 1) * sy + ((a >> 2) & 1) * sz);
     const float ga[2] = {DN_GA, DN_GB};
     const float L[2][2] = {{1.f - DN_GA, DN_GA}, {1.f - DN_GB, DN_GB}};   // L[point][corner bit]
     float nuq[2][2][2];                                                     // [p: xi][q: eta][s: zeta]

@@ -43,6 +43,8 @@ struct Params {
     const float* nu;
     const float* f;
     const float* gJ;
+    const float* bc0_b;   // per-sample boundary values or NULL (then bc_x0 / bc_x1 hold for every sample)
+    const float* bc1_b;
     float* r;             // may be NULL (energy only)
     double* partials;
     const float* ckl;
@@ -81,7 +83,8 @@ cudaError_t launch_tiled2d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s);
 cudaError_t launch_kl_field(const dn_grid& g, int batch, int m, const float* kl_w, float* nu, cudaStream_t s);
-cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int mode, float* field, cudaStream_t s);
+cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int mode, float* field, cudaStream_t s,
+                            const float* b0_b = nullptr, const float* b1_b = nullptr);
 
 int generic_blocks_per_sample(long long nodes);
 bool tiled2d_applicable(const dn_problem& p);

@@ -194,7 +194,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
         float* rb = WANT_R ? P.r + (size_t)b * P.nodes : nullptr;
         const bool impose = (P.flags & DN_IMPOSE_BC_ON_LOAD) != 0;
         const bool nomask = (P.flags & DN_NO_MASK) != 0;
-        const float bc0 = P.bc_x0, bc1 = P.bc_x1;
+        const float bc0 = P.bc0_b ? __ldg(P.bc0_b + b) : P.bc_x0, bc1 = P.bc1_b ? __ldg(P.bc1_b + b) : P.bc_x1;
         const float kx = 0.25f * P.hy / P.hx, ky = 0.25f * P.hx / P.hy;
         const float kxa = kx * DN_GA, kxb = kx * DN_GB, kya = ky * DN_GA, kyb = ky * DN_GB;
         const float fw = P.f_const * P.hx * P.hy;       // nodal load of an interior node

@@ -148,7 +148,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     const float kap = iso ? kx : 1.f;                  // isotropic cells: one scale applied at the end
     const bool nomask = (P.flags & DN_NO_MASK) != 0;
     const bool impose = (P.flags & DN_IMPOSE_BC_ON_LOAD) != 0;
-    const float bc0 = P.bc_x0, bc1 = P.bc_x1;
+    const float bc0 = P.bc0_b ? __ldg(P.bc0_b + b) : P.bc_x0, bc1 = P.bc1_b ? __ldg(P.bc1_b + b) : P.bc_x1;
     const float gs = (WANT_R && P.gJ) ? __ldg(P.gJ + b) : 1.f;
     const float fw = P.f_const * P.hx * P.hy * P.hz;  // nodal load of an interior node
     const bool hasf = (P.f_const != 0.f);
