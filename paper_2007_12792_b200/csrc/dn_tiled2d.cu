@@ -12,8 +12,13 @@
 // times), so nothing is copied.  The x+1 neighbour comes from the next lane by shuffle, across
 // warps from global memory (one scalar per row).  Every
 // element is computed exactly once per block: its contributions to its two left nodes stay in the
-// thread, those to its right nodes go to the owner of the next element (shuffle; shared memory
-// between warps, one named barrier per row), those to the upper row are carried to the next step.
+// thread, those to its right nodes go to the owner of the next element (shuffle), those to the
+// upper row are carried to the next step.  Between the warps of a row the two right-hand values of
+// a warp's last element travel through shared memory one row late: the warp publishes them and
+// arrives on a split-phase barrier (mbarrier), and one row later takes its left neighbour's values
+// of the previous row, completing the one output it had stored without them.  The warps of a row
+// therefore never meet at a barrier (a full barrier per row cost 12 % in nodal mode).  Waits are
+// bounded; should one run out, the energy of that sample is returned as NaN.
 // The first element row of a chunk is recomputed by the chunk below (1/R redundancy).  No atomics.
 //
 // Arithmetic of one element (corners u00 u10 / u01 u11, e0 = u10-u00, s0 = u01-u00,
@@ -46,11 +51,27 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-__device__ __forceinline__ void named_barrier(int id, int nthreads) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-
 typedef unsigned long long u64;
+
+// Split-phase barrier among the warps of one row group (mbarrier in shared memory): a warp arrives when its seam
+// values of a row are written and waits, one row later, for the arrivals of that row.
+__device__ __forceinline__ void mbar_init(u64* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(u64* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"((unsigned)__cvta_generic_to_shared(bar)) : "memory");
+}
+// Bounded wait for the phase of the given parity; false if it did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(u64* bar, int parity) {
+    const unsigned a = (unsigned)__cvta_generic_to_shared(bar);
+    for (int it = 0; it < (1 << 16); ++it) {
+        unsigned ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
 
 // Asynchronous global -> shared copies (each thread later reads back only what it copied itself,
 // so completion of its own copy groups is all the synchronisation the ring needs).
@@ -90,6 +111,12 @@ template <int K, int M, bool WANT_R, bool FULL, bool RING, bool KN>
 __global__ void __launch_bounds__(256, 2)
 tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
     extern __shared__ __align__(16) float smem[];
+    __shared__ __align__(8) u64 seam_bar[T2_MAX_WARPS][2];
+    __shared__ float sbc[2];                            // Dirichlet values of this sample (read only when imposed on load)
+    if (threadIdx.x == 0) {
+        sbc[0] = P.bc0_b ? __ldg(P.bc0_b + blockIdx.y) : P.bc_x0;
+        sbc[1] = P.bc1_b ? __ldg(P.bc1_b + blockIdx.y) : P.bc_x1;
+    }
     constexpr bool HASM = (M > 0);                      // KL weights in play (either KL mode)
     constexpr bool KL = HASM && !KN;                    // nu evaluated at the Gauss points
     constexpr bool NLOAD = !HASM;                       // nu rows loaded from a nodal field
@@ -181,6 +208,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             for (int k = 0; k <= M; ++k) { dst[2 * k] = (float)acc[k]; dst[2 * k + 1] = (float)acc[k]; }
         }
     }
+    if (lane == 0 && wx == 0) { mbar_init(&seam_bar[wy][0], W); mbar_init(&seam_bar[wy][1], W); }
     __syncthreads();
 
     float en = 0.f, ell = 0.f;
@@ -194,7 +222,6 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
         float* rb = WANT_R ? P.r + (size_t)b * P.nodes : nullptr;
         const bool impose = (P.flags & DN_IMPOSE_BC_ON_LOAD) != 0;
         const bool nomask = (P.flags & DN_NO_MASK) != 0;
-        const float bc0 = P.bc0_b ? __ldg(P.bc0_b + b) : P.bc_x0, bc1 = P.bc1_b ? __ldg(P.bc1_b + b) : P.bc_x1;
         const float kx = 0.25f * P.hy / P.hx, ky = 0.25f * P.hx / P.hy;
         const float kxa = kx * DN_GA, kxb = kx * DN_GB, kya = ky * DN_GA, kyb = ky * DN_GB;
         const float fw = P.f_const * P.hx * P.hy;       // nodal load of an interior node
@@ -260,10 +287,10 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
         };
         auto fix_bc = [&](Row<NE>& r) {
             if (impose) {
-                if (x0 == 0) r.v[0] = bc0;
+                if (x0 == 0) r.v[0] = sbc[0];
                 if (has_last) {
 #pragma unroll
-                    for (int k = 0; k < NE; ++k) if (k == klast) r.v[k] = bc1;
+                    for (int k = 0; k < NE; ++k) if (k == klast) r.v[k] = sbc[1];
                 }
             }
         };
@@ -360,6 +387,25 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             if constexpr (NLOAD) load_row(nB, nub, jbeg + 1);
             if constexpr (KN) nu_row(nB, jbeg + 1);
         }
+
+        // Values the left neighbour warp published for step ip (node row jp): its last element's contribution to
+        // this lane's first node on row jp (that row's output is already stored without it: store it again,
+        // completed) and on row jp + 1 (still pending in U[0]).
+        float pend0 = 0.f, uprev0 = 0.f;
+        bool seam_ok = true;
+        auto seam_take = [&](const int ip, const int jp) {
+            if (!mbar_wait(&seam_bar[wy][ip & 1], (ip >> 1) & 1)) seam_ok = false;
+            if (lane == 0 && wx > 0) {
+                const float* slot = xch + (size_t)(ip & 1) * T2_MAX_WARPS * 2;
+                const float qx = slot[2 * (wx - 1)], tx = slot[2 * (wx - 1) + 1];
+                U[0] += tx;
+                if (jp >= n0) {
+                    en = fmaf(uprev0, qx, en);
+                    rb[(size_t)jp * nx + x0] = fmaf(gs, qx, pend0);
+                }
+            }
+            __syncwarp();                               // lane 31 publishes only after lane 0 has read
+        };
 
         // One element row: lo holds node row j, cur node row j+1 (read from the ring, or loaded by the
         // previous step); the direct variant loads row j+2 into nxt.
@@ -463,17 +509,23 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
 
             if (WANT_R) {
                 // contributions of the element left of this lane's first node
-                float* slot = xch + (size_t)(j & 1) * T2_MAX_WARPS * 2;
+                // Across warps the two values travel through shared memory one row late: the warp publishes
+                // them and arrives, and takes its left neighbour's values of the previous row (which every warp
+                // of the group has published by then) - so the warps of a row never meet at a barrier.
+                const int i = j - jbeg;
                 if (W > 1) {
-                    if (lane == 31) { slot[2 * wx] = Qp; slot[2 * wx + 1] = Tp; }
-                    named_barrier(1 + wy, 32 * W);
+                    // take before publishing: once every warp has arrived for the previous row, every warp has
+                    // also read the row before that, whose slot this row's values overwrite
+                    if (i > 0) seam_take(i - 1, j - 1);
+                    if (lane == 31) {
+                        float* slot = xch + (size_t)(i & 1) * T2_MAX_WARPS * 2;
+                        slot[2 * wx] = Qp; slot[2 * wx + 1] = Tp;
+                        mbar_arrive(&seam_bar[wy][i & 1]);
+                    }
                 }
                 float ql = __shfl_up_sync(0xffffffffu, Qp, 1);
                 float tl = __shfl_up_sync(0xffffffffu, Tp, 1);
-                if (lane == 0) {
-                    ql = 0.f; tl = 0.f;
-                    if (W > 1 && wx > 0) { ql = slot[2 * (wx - 1)]; tl = slot[2 * (wx - 1) + 1]; }
-                }
+                if (lane == 0) { ql = 0.f; tl = 0.f; }
                 rout[0] = fmaf(-ky, SY0, ql - Q0) + U[0];
                 U[0] = R0 + tl;
                 if (own) {
@@ -500,6 +552,7 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
                     for (int s = 0; s < K; ++s)
                         if (act[s])
                             *reinterpret_cast<float4*>(rrow + 4 * s) = make_float4(o[4 * s], o[4 * s + 1], o[4 * s + 2], o[4 * s + 3]);
+                    pend0 = o[0]; uprev0 = lo.v[0];
                 }
             }
             if constexpr (!KL) nlr = nhr;
@@ -517,6 +570,8 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
             if (++j > jend) { fin = A; break; }
         }
         if constexpr (RING) cp_async_wait<0>();
+        if constexpr (WANT_R) { if (W > 1) seam_take(jend - jbeg, jend); }
+        if (!seam_ok) en = __int_as_float(0x7fc00000);   // a wait ran out: the energy of this sample reads NaN
 
         // ---- the top node row of the domain has no element row above it
         if (n1 == ny) {
