@@ -41,6 +41,7 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 Launch choose_launch(const dn_problem& p, const float* u, const float* r) {
     const bool vec_ok = aligned16(u) && aligned16(r) && (p.nu_mode != DN_NU_NODAL || aligned16(p.nu));
     if (!(p.flags & DN_FORCE_GENERIC) && vec_ok && p.f == nullptr) {
+        if (r && strip2d_applicable(p)) return strip2d_geometry(p);
         if (tiled2d_applicable(p)) return tiled2d_geometry(p);
         if (tiled3d_applicable(p)) return tiled3d_geometry(p);
     }
@@ -55,6 +56,7 @@ Launch choose_launch(const dn_problem& p, const float* u, const float* r) {
 static int max_nblk(const dn_problem& p) {
     int n = generic_blocks_per_sample(nodes_per_sample(p.grid));
     if (tiled2d_applicable(p)) { int t = tiled2d_geometry(p).nblk; if (t > n) n = t; }
+    if (strip2d_applicable(p)) { int t = strip2d_geometry(p).nblk; if (t > n) n = t; }
     if (tiled3d_applicable(p)) { int t = tiled3d_geometry(p).nblk; if (t > n) n = t; }
     return n;
 }
@@ -83,6 +85,8 @@ WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
     }
     w.seam = off;
     if ((tight ? l.path == PATH_TILED3D : tiled3d_applicable(p))) off += align_up(sizeof(float) * tiled3d_seam_floats(p) + 16);
+    w.rowpoly = off;
+    if ((tight ? l.path == PATH_STRIP2D : strip2d_applicable(p))) off += align_up(sizeof(float) * strip2d_rowpoly_floats(p) + 16);
     w.total = off;
     return w;
 }
@@ -119,8 +123,12 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
         const char* b = reinterpret_cast<const char*>(r);
         if (a < b + bytes && b < a + bytes) return DN_ERR_ALIAS;
     }
-    const Launch l = choose_launch(*p, u, r);
-    const WsLayout w = make_layout(*p, l, tight);
+    Launch l = choose_launch(*p, u, r);
+    WsLayout w = make_layout(*p, l, tight);
+    if (tight && l.path == PATH_STRIP2D && ws_bytes < w.total) {       // its coefficient table does not fit: tiled kernel
+        l = tiled2d_geometry(*p);
+        w = make_layout(*p, l, tight);
+    }
     if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign) != 0 || ws_bytes < w.total) return DN_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Params P = make_params(*p, w, u, gJ, r, ws);
@@ -133,9 +141,11 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
                         reinterpret_cast<float*>(base + w.cn[2])};
         e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s);
         if (e != cudaSuccess) return DN_ERR_CUDA;
+        if (l.path == PATH_STRIP2D && launch_rowpoly(P, reinterpret_cast<float*>(base + w.rowpoly), s) != cudaSuccess) return DN_ERR_CUDA;
     }
     if (ev_before && cudaEventRecord(static_cast<cudaEvent_t>(ev_before), s) != cudaSuccess) return DN_ERR_CUDA;
-    if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
+    if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
+    else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
     else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
     else e = launch_generic(P, s);
     if (e != cudaSuccess) return DN_ERR_CUDA;
@@ -165,8 +175,10 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
                         reinterpret_cast<float*>(base + w.cn[2])};
         e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s);
         if (e != cudaSuccess) return DN_ERR_CUDA;
+        if (l.path == PATH_STRIP2D && launch_rowpoly(P, reinterpret_cast<float*>(base + w.rowpoly), s) != cudaSuccess) return DN_ERR_CUDA;
     }
-    if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
+    if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
+    else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
     else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
     else e = launch_generic(P, s);
     if (e != cudaSuccess) return DN_ERR_CUDA;
@@ -337,12 +349,14 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
 int32_t dn_launches_per_call(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
     const bool t3 = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
-    return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
+    const bool s2 = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && strip2d_applicable(*p);   // fused call: one more table kernel
+    return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0) + (s2 ? 1 : 0);
 }
 
 const char* dn_path_name(const dn_problem* p) {
     if (validate(p) != DN_OK) return "invalid";
     if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr) {
+        if (strip2d_applicable(*p)) return "strip2d";      // the fused call; the energy-only call of such a problem runs tiled2d
         if (tiled2d_applicable(*p)) return "tiled2d";
         if (tiled3d_applicable(*p)) return "tiled3d";
     }

@@ -17,7 +17,7 @@ constexpr int kAlign = 256;
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
-enum Path { PATH_GENERIC = 0, PATH_TILED2D = 1, PATH_TILED3D = 2 };
+enum Path { PATH_GENERIC = 0, PATH_TILED2D = 1, PATH_TILED3D = 2, PATH_STRIP2D = 3 };
 
 // Where things live inside the caller's workspace (byte offsets, all 256-B aligned).
 struct WsLayout {
@@ -28,6 +28,7 @@ struct WsLayout {
     int gstride[3];       // padded row length of cg[a] (multiple of 4)
     size_t cn[3];         // float  [m][nstride[a]] cos(i pi x) at the nodes of axis a
     int nstride[3];
+    size_t rowpoly;       // float  [B][ny-1][GS] polynomial of the KL exponent along every Gauss row (strip 2D kernel)
     int nblk;             // energy partials per sample
     size_t total;
 };
@@ -81,6 +82,8 @@ cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float*
 cudaError_t launch_generic(const Params& P, cudaStream_t s);
 cudaError_t launch_tiled2d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s);
+cudaError_t launch_rowpoly(const Params& P, float* rowpoly, cudaStream_t s);      // needs the tables of launch_tables
+cudaError_t launch_strip2d(const Params& P, const float* rowpoly, cudaStream_t s);
 cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s);
 cudaError_t launch_kl_field(const dn_grid& g, int batch, int m, const float* kl_w, float* nu, cudaStream_t s);
 cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int mode, float* field, cudaStream_t s,
@@ -89,6 +92,9 @@ cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int
 int generic_blocks_per_sample(long long nodes);
 bool tiled2d_applicable(const dn_problem& p);
 bool tiled3d_applicable(const dn_problem& p);
+bool strip2d_applicable(const dn_problem& p);     // fused energy+residual, KL at the Gauss points, wide 2D grids
+Launch strip2d_geometry(const dn_problem& p);
+size_t strip2d_rowpoly_floats(const dn_problem& p);
 Launch tiled2d_geometry(const dn_problem& p);
 Launch tiled3d_geometry(const dn_problem& p);
 size_t tiled3d_seam_floats(const dn_problem& p);   // scratch floats the tiled 3D kernel needs for its tile seams

@@ -1,0 +1,88 @@
+"""GPU parity of the strip kernel (2D, KL diffusivity at the Gauss points, energy and residual fused) against the
+fp64 oracle: strips that end exactly at the grid, ragged last strips, one and many chunks, every option it serves."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2007_12792_b200 import binding as B
+from paper_2007_12792_b200 import inputs
+from parity_util import dev, make_problems, run_gpu, check
+
+pytestmark = pytest.mark.gpu
+
+# (nx, ny, batch, m): 256 = first width the kernel takes; 252 + 128 = 380 ends a strip exactly at the grid; 376/384 are
+# one lane short / one lane beyond; 2048 is the bench width; ny = 16 is the shortest grid, 700 spans several chunks
+SIZES = [(256, 40, 2, 4), (260, 17, 3, 1), (376, 33, 2, 6), (380, 16, 2, 2), (384, 21, 1, 3), (504, 50, 2, 5),
+         (508, 20, 2, 8), (1028, 37, 1, 7), (2048, 24, 2, 6), (256, 700, 40, 2)]
+
+
+@pytest.mark.parametrize("nx,ny,batch,m", SIZES)
+def test_strip2d_parity(nx, ny, batch, m):
+    inp = inputs.random_inputs(2, nx, ny, 1, batch, m, seed=7 + nx + ny, f_const=0.6)
+    po, pg = make_problems(inp, B.DN_NU_KL_GAUSS)
+    assert B.dn_path_name(pg) == "strip2d"
+    Jo, _, _, ro = oracle.energy_grad(po, inp.u)
+    Jg, rg = run_gpu(pg, inp.u)
+    check(Jg, rg, Jo, ro, f"strip2d {nx}x{ny} b{batch} m{m}")
+    assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
+    # the any-size kernels on the same problem: two independent CUDA paths agree with the oracle
+    _, pgen = make_problems(inp, B.DN_NU_KL_GAUSS, flags=B.DN_FORCE_GENERIC)
+    Jg2, rg2 = run_gpu(pgen, inp.u)
+    check(Jg2, rg2, Jo, ro, "generic")
+
+
+@pytest.mark.parametrize("nx,ny", [(256, 37), (380, 19), (520, 23)])
+def test_strip2d_options(nx, ny):
+    inp = inputs.random_inputs(2, nx, ny, 1, 3, 3, seed=42, f_const=-0.4)
+    u = inputs.random_field(inp.u.shape, 8)           # boundary values NOT satisfied
+    gJ = np.array([1.5, -2.0, 0.25], dtype=np.float32)
+    for flags in (0, B.DN_NO_MASK, B.DN_IMPOSE_BC_ON_LOAD, B.DN_IMPOSE_BC_ON_LOAD | B.DN_NO_MASK):
+        po, pg = make_problems(inp, B.DN_NU_KL_GAUSS, flags=flags, bc=(0.8, -0.3))
+        assert B.dn_path_name(pg) == "strip2d"
+        Jo, _, _, ro = oracle.energy_grad(po, u, gJ=gJ.astype(np.float64))
+        Jg, rg = run_gpu(pg, u, gJ=gJ)
+        check(Jg, rg, Jo, ro, f"flags={flags}")
+        if not (flags & B.DN_NO_MASK):
+            assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
+    # energy-only call (tiled kernel) against the fused call (strip kernel); residual-only call gives the same residual
+    po, pg = make_problems(inp, B.DN_NU_KL_GAUSS)
+    ws = B.new_workspace(pg)
+    J1 = torch.empty(3, device="cuda"); J2 = torch.empty(3, device="cuda"); r = torch.empty(pg.shape, device="cuda")
+    B.dn_energy(pg, dev(u), J1, ws)
+    B.dn_energy_grad(pg, dev(u), None, J2, r, ws)
+    r2 = torch.empty_like(r)
+    B.dn_energy_grad(pg, dev(u), None, None, r2, ws)
+    torch.cuda.synchronize()
+    assert torch.allclose(J1, J2, rtol=1e-5, atol=0) and torch.equal(r, r2)
+
+
+def test_strip2d_per_sample_boundary_values():
+    inp = inputs.random_inputs(2, 508, 18, 1, 3, 2, seed=5, f_const=0.3)
+    u = inputs.random_field(inp.u.shape, 3)
+    b0 = np.array([0.9, -0.2, 0.4], dtype=np.float32); b1 = np.array([0.1, 0.7, -0.6], dtype=np.float32)
+    _, pg = make_problems(inp, B.DN_NU_KL_GAUSS, flags=B.DN_IMPOSE_BC_ON_LOAD)
+    pg.bc_x0_b = dev(b0); pg.bc_x1_b = dev(b1)
+    Jg, rg = run_gpu(pg, u)
+    for s in range(3):                                 # the oracle, sample by sample with that sample's values
+        one = inputs.random_inputs(2, 508, 18, 1, 3, 2, seed=5, f_const=0.3)
+        po = oracle.Problem(dim=2, nx=508, ny=18, nz=1, batch=1, nu_mode=B.DN_NU_KL_GAUSS, nu=None, kl_modes=2,
+                            kl_w=one.kl_w[s:s + 1], f_const=0.3, f=None, bc_x0=float(b0[s]), bc_x1=float(b1[s]),
+                            flags=B.DN_IMPOSE_BC_ON_LOAD)
+        Jo, _, _, ro = oracle.energy_grad(po, u[s:s + 1])
+        check(Jg[s:s + 1], rg[s:s + 1], Jo, ro, f"sample {s}")
+
+
+def test_strip2d_determinism_and_stale_workspace():
+    inp = inputs.random_inputs(2, 1028, 300, 1, 2, 6, seed=11)
+    _, pg = make_problems(inp, B.DN_NU_KL_GAUSS)
+    ws = B.new_workspace(pg)
+    ud = dev(inp.u)
+    outs = []
+    for it in range(3):
+        ws.fill_(255 if it == 1 else 0)
+        r = torch.empty(pg.shape, device="cuda"); J = torch.empty(pg.batch, device="cuda")
+        B.dn_energy_grad(pg, ud, None, J, r, ws)
+        outs.append((J.cpu().numpy().copy(), r.cpu().numpy().copy()))
+    for J, r in outs[1:]:
+        assert J.tobytes() == outs[0][0].tobytes() and r.tobytes() == outs[0][1].tobytes()
