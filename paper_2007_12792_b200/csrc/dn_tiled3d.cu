@@ -168,15 +168,17 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     float* pseam = seam_row ? P.seam + (((size_t)b * (ntile_y - 1) + tile) * nz) * nx + x0 : nullptr;
     float* pr = WANT_R ? P.r + (size_t)b * P.nodes + (size_t)yl * nx + x0 : nullptr;
 
-    u64 cda[4], cdb[4];                                // cos(pi x) at the two Gauss columns, duplicated
+    // cos(pi x) at the two Gauss columns of each element as duplicated pairs (ca, ca, cb, cb), kept in shared memory
+    float4* cps = reinterpret_cast<float4*>(gam + (size_t)(Z + 1) * TY * 2 * GS) + threadIdx.x;
+    const int cstr = blockDim.x;
     if constexpr (KL) {
         float4 q0 = make_float4(0.f, 0.f, 0.f, 0.f), q1 = q0;
         if (col_ok) {
             q0 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0));
             q1 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0 + 4));
         }
-        cda[0] = pack2_3(q0.x, q0.x); cdb[0] = pack2_3(q0.y, q0.y); cda[1] = pack2_3(q0.z, q0.z); cdb[1] = pack2_3(q0.w, q0.w);
-        cda[2] = pack2_3(q1.x, q1.x); cdb[2] = pack2_3(q1.y, q1.y); cda[3] = pack2_3(q1.z, q1.z); cdb[3] = pack2_3(q1.w, q1.w);
+        cps[0] = make_float4(q0.x, q0.x, q0.y, q0.y); cps[cstr] = make_float4(q0.z, q0.z, q0.w, q0.w);
+        cps[2 * cstr] = make_float4(q1.x, q1.x, q1.y, q1.y); cps[3 * cstr] = make_float4(q1.z, q1.z, q1.w, q1.w);
     }
 
     PlaneState S0, S1;
@@ -398,10 +400,11 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                         if constexpr (KL) {
                             // nu[p][q][s] at the 8 Gauss points: 4 packed Horner chains (column p, row q) x (s = a, b)
                             u64 h_aa = gq_a[MM], h_ab = gq_b[MM], h_ba = gq_a[MM], h_bb = gq_b[MM];   // h_{p q}
+                            const ulonglong2 cc = *reinterpret_cast<const ulonglong2*>(cps + c * cstr);
 #pragma unroll
                             for (int i = MM - 1; i >= 0; --i) {
-                                h_aa = fma2_3(h_aa, cda[c], gq_a[i]); h_ab = fma2_3(h_ab, cda[c], gq_b[i]);
-                                h_ba = fma2_3(h_ba, cdb[c], gq_a[i]); h_bb = fma2_3(h_bb, cdb[c], gq_b[i]);
+                                h_aa = fma2_3(h_aa, cc.x, gq_a[i]); h_ab = fma2_3(h_ab, cc.x, gq_b[i]);
+                                h_ba = fma2_3(h_ba, cc.y, gq_a[i]); h_bb = fma2_3(h_bb, cc.y, gq_b[i]);
                             }
                             unpack2_3(h_aa, n000, n001); unpack2_3(h_ab, n010, n011);
                             unpack2_3(h_ba, n100, n101); unpack2_3(h_bb, n110, n111);
@@ -586,7 +589,7 @@ Geo3 geometry3(const dn_problem& p) {
         const size_t fixed = sizeof(float) * 2 * ((size_t)(m ? 4 : 5) * TY * WX * 128 + (size_t)TY * WX * 4);
         for (int Z = 4; Z <= 256; ++Z) {
             if (Z > nz && Z > 4) break;
-            const size_t sm = fixed + sizeof(float) * (size_t)(Z + 1) * TY * 2 * GS;
+            const size_t sm = fixed + sizeof(float) * (size_t)(Z + 1) * TY * 2 * GS + (m ? (size_t)16 * 4 * 32 * WX * TY : 0);
             if (sm * bps > 200 * 1024) break;
             const long long nch = (nz + Z - 1) / Z;
             const long long blocks = (long long)p.batch * ntile * nch;
