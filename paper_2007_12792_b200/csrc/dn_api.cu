@@ -139,9 +139,10 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
                         reinterpret_cast<float*>(base + w.cg[2])};
         float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
                         reinterpret_cast<float*>(base + w.cn[2])};
-        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s);
+        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
+                          (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
+                          strip2d_rowpoly_stride(p->kl_modes));
         if (e != cudaSuccess) return DN_ERR_CUDA;
-        if (l.path == PATH_STRIP2D && launch_rowpoly(P, reinterpret_cast<float*>(base + w.rowpoly), s) != cudaSuccess) return DN_ERR_CUDA;
     }
     if (ev_before && cudaEventRecord(static_cast<cudaEvent_t>(ev_before), s) != cudaSuccess) return DN_ERR_CUDA;
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
@@ -173,9 +174,10 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
                         reinterpret_cast<float*>(base + w.cg[2])};
         float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
                         reinterpret_cast<float*>(base + w.cn[2])};
-        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s);
+        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
+                          (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
+                          strip2d_rowpoly_stride(p->kl_modes));
         if (e != cudaSuccess) return DN_ERR_CUDA;
-        if (l.path == PATH_STRIP2D && launch_rowpoly(P, reinterpret_cast<float*>(base + w.rowpoly), s) != cudaSuccess) return DN_ERR_CUDA;
     }
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
     else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
@@ -349,8 +351,7 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
 int32_t dn_launches_per_call(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
     const bool t3 = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
-    const bool s2 = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && strip2d_applicable(*p);   // fused call: one more table kernel
-    return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0) + (s2 ? 1 : 0);
+    return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
 }
 
 const char* dn_path_name(const dn_problem* p) {

@@ -24,7 +24,61 @@ struct TableArgs {
     float* cg[3];
     int nstride[3];
     float* cn[3];
+    float* rowpoly;       // 2D, optional: polynomial of the KL exponent along every Gauss row, [B][ny-1][rp_gs]
+    int rp_gs;
 };
+
+// exponent(x, y_q) = sum_k poly[k] c^k with c = cos(pi x), for the Gauss row q of element row j of sample b:
+// g_i = sum_j ckl[i][j] cos(j pi y_q) are the coefficients in the Chebyshev basis (cos(i pi x) = T_i(c)), converted
+// to monomials in double.  The scaled weights and the cosines are rounded to float first, exactly as the tables
+// hold them, so every kernel family sees the same numbers.  Entry 2k + q of the row; the two Gauss rows of an
+// element row interleave so that they can be evaluated together with two-wide FMAs.  Loops run to the compiled
+// maximum with zero coefficients beyond m, which keeps the small arrays in registers.
+__device__ void rowpoly_entry(const TableArgs& A, long long idx) {
+    constexpr int MX = DN_MAX_KL_MODES;
+    const int m = A.m, ny = A.n[1];
+    const int q = (int)(idx & 1);
+    const long long row = idx >> 1;                    // b * (ny - 1) + j
+    const int j = (int)(row % (ny - 1));
+    const long long b = row / (ny - 1);
+    const double ga = 0.5 * (1.0 - 0.57735026918962576451);
+    const double gb = 0.5 * (1.0 + 0.57735026918962576451);
+    const double y = ((double)j + (q ? gb : ga)) / (double)(ny - 1);
+    double cy[MX], g[MX];
+#pragma unroll
+    for (int jj = 0; jj < MX; ++jj) cy[jj] = (jj < m) ? (double)(float)cospi((double)(jj + 1) * y) : 0.0;
+    const float* w = A.kl_w + b * m * m;
+#pragma unroll
+    for (int i = 0; i < MX; ++i) {
+        double a = 0.0;
+#pragma unroll
+        for (int jj = 0; jj < MX; ++jj) {
+            if (i < m && jj < m) {
+                const double den = 1.0 + (double)((i + 1) * (i + 1)) + (double)((jj + 1) * (jj + 1));
+                a += (double)(float)((double)w[i * m + jj] * kLog2e / den) * cy[jj];
+            }
+        }
+        g[i] = a;
+    }
+    // sum_i g_i T_i(c) in the monomial basis, T_{i+1} = 2 c T_i - T_{i-1}
+    double acc[MX + 1], tp[MX + 1], tc[MX + 1];
+#pragma unroll
+    for (int k = 0; k <= MX; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
+#pragma unroll
+    for (int i = 1; i <= MX; ++i) {
+#pragma unroll
+        for (int k = 0; k <= MX; ++k) acc[k] += g[i - 1] * tc[k];
+        double tn[MX + 1];
+#pragma unroll
+        for (int k = 0; k <= MX; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
+#pragma unroll
+        for (int k = 0; k <= MX; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
+    }
+    float* dst = A.rowpoly + row * A.rp_gs + q;
+#pragma unroll
+    for (int k = 0; k <= MX; ++k)
+        if (2 * k + q < A.rp_gs) dst[2 * k] = (k <= m) ? (float)acc[k] : 0.f;
+}
 
 __global__ void tables_kernel(TableArgs A) {
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -69,6 +123,7 @@ __global__ void tables_kernel(TableArgs A) {
         }
         idx -= cnt;
     }
+    if (A.rowpoly && idx < 2ll * A.batch * (A.n[1] - 1)) rowpoly_entry(A, idx);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -245,7 +300,7 @@ __global__ void apply_bc_kernel(long long lines, long long lines_per_sample, int
 }  // namespace
 
 cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], float* const cn[3],
-                          cudaStream_t s) {
+                          cudaStream_t s, float* rowpoly, int rowpoly_stride) {
     TableArgs A{};
     A.dim = P.dim; A.m = P.m; A.batch = P.batch;
     A.n[0] = P.nx; A.n[1] = P.ny; A.n[2] = P.nz;
@@ -257,6 +312,8 @@ cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float*
         if (a < P.dim) total += (long long)P.m * (P.gstride[a] + P.nstride[a]);
     }
     A.kl_w = kl_w; A.ckl = ckl;
+    A.rowpoly = (P.dim == 2) ? rowpoly : nullptr; A.rp_gs = rowpoly_stride;
+    if (A.rowpoly) total += 2ll * P.batch * (P.ny - 1);
     const int threads = 128;
     tables_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, s>>>(A);
     return cudaGetLastError();

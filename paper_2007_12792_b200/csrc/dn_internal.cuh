@@ -77,12 +77,12 @@ dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float*
 dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, size_t ws_bytes, cudaStream_t s,
                        bool build_tables, const double** partials, int* nblk);
 
+// rowpoly (optional, 2D): also writes the per-Gauss-row polynomials the strip kernel reads, rows of rowpoly_stride floats
 cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], float* const cn[3],
-                          cudaStream_t s);
+                          cudaStream_t s, float* rowpoly = nullptr, int rowpoly_stride = 0);
 cudaError_t launch_generic(const Params& P, cudaStream_t s);
 cudaError_t launch_tiled2d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s);
-cudaError_t launch_rowpoly(const Params& P, float* rowpoly, cudaStream_t s);      // needs the tables of launch_tables
 cudaError_t launch_strip2d(const Params& P, const float* rowpoly, cudaStream_t s);
 cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s);
 cudaError_t launch_kl_field(const dn_grid& g, int batch, int m, const float* kl_w, float* nu, cudaStream_t s);
@@ -95,6 +95,7 @@ bool tiled3d_applicable(const dn_problem& p);
 bool strip2d_applicable(const dn_problem& p);     // fused energy+residual, KL at the Gauss points, wide 2D grids
 Launch strip2d_geometry(const dn_problem& p);
 size_t strip2d_rowpoly_floats(const dn_problem& p);
+int strip2d_rowpoly_stride(int kl_modes);          // floats per element row of that table
 Launch tiled2d_geometry(const dn_problem& p);
 Launch tiled3d_geometry(const dn_problem& p);
 size_t tiled3d_seam_floats(const dn_problem& p);   // scratch floats the tiled 3D kernel needs for its tile seams

@@ -21,7 +21,7 @@
 // the residual by Euler's identity for quadratic forms: 1/2 sum_i u_i (K u)_i.
 //
 // KL diffusivity: for a fixed Gauss row the exponent is a polynomial of degree m in c = cos(pi x).
-// rowpoly_kernel prepares its coefficients in double once per call (they do not depend on u), for
+// The table kernel prepares its coefficients in double once per call (they do not depend on u), for
 // both Gauss rows of every element row, interleaved so that the two rows are evaluated together
 // with packed two-wide FMAs.
 #include "dn_internal.cuh"
@@ -71,54 +71,6 @@ template <int N> __device__ __forceinline__ void s2_wait() { asm volatile("cp.as
 
 // Floats per element row in the coefficient table: (row a, row b) pairs for k = 0..M, padded to a multiple of 4.
 __host__ __device__ constexpr int s2_gs(int m) { return (2 * (m + 1) + 3) / 4 * 4; }
-
-// Coefficients of the KL exponent along the Gauss rows: exponent(x, y_q) = sum_k poly[k] c^k with c = cos(pi x).
-// One thread per (sample, element row, Gauss row of it); table [B][ny-1][GS], entry 2k + q.  All loops have
-// compile-time bounds so that the small arrays stay in registers.
-template <int M>
-__global__ void __launch_bounds__(128)
-rowpoly_kernel(const float* __restrict__ ckl, const float* __restrict__ cgy, int gstride, int ny, int batch,
-               float* __restrict__ poly) {
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long total = 2ll * batch * (ny - 1);
-    if (idx >= total) return;
-    const int q = (int)(idx & 1);
-    const long long row = idx >> 1;                    // b * (ny - 1) + j
-    const int j = (int)(row % (ny - 1));
-    const int b = (int)(row / (ny - 1));
-    const int gy = 2 * j + q;
-    const float* c = ckl + (size_t)b * M * M;
-    double cy[M], g[M];
-#pragma unroll
-    for (int jj = 0; jj < M; ++jj) cy[jj] = (double)__ldg(cgy + jj * gstride + gy);
-#pragma unroll
-    for (int i = 0; i < M; ++i) {
-        double a = 0.0;
-#pragma unroll
-        for (int jj = 0; jj < M; ++jj) a += (double)__ldg(c + i * M + jj) * cy[jj];
-        g[i] = a;
-    }
-    // sum_i g_i T_i(c) in the monomial basis, T_{i+1} = 2 c T_i - T_{i-1}
-    double acc[M + 1], tp[M + 1], tc[M + 1];
-#pragma unroll
-    for (int k = 0; k <= M; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
-#pragma unroll
-    for (int i = 1; i <= M; ++i) {
-#pragma unroll
-        for (int k = 0; k <= M; ++k) acc[k] += g[i - 1] * tc[k];
-        double tn[M + 1];
-#pragma unroll
-        for (int k = 0; k <= M; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
-#pragma unroll
-        for (int k = 0; k <= M; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
-    }
-    constexpr int GS = s2_gs(M);
-    float* dst = poly + (size_t)row * GS + q;
-#pragma unroll
-    for (int k = 0; k <= M; ++k) dst[2 * k] = (float)acc[k];
-#pragma unroll
-    for (int k = 2 * (M + 1); k < GS; k += 2) dst[k] = 0.f;
-}
 
 template <int M, int BPS>
 __global__ void __launch_bounds__(S2_WARPS * 32, BPS)
@@ -418,26 +370,7 @@ size_t strip2d_rowpoly_floats(const dn_problem& p) {
     return (size_t)p.batch * (p.grid.ny - 1) * s2_gs(p.kl_modes);
 }
 
-template <int M>
-static cudaError_t launch_rowpoly_m(const Params& P, float* rowpoly, cudaStream_t s) {
-    const long long total = 2ll * P.batch * (P.ny - 1);
-    rowpoly_kernel<M><<<(unsigned)((total + 127) / 128), 128, 0, s>>>(P.ckl, P.cg[1], P.gstride[1], P.ny, P.batch, rowpoly);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_rowpoly(const Params& P, float* rowpoly, cudaStream_t s) {
-    switch (P.m) {
-        case 1: return launch_rowpoly_m<1>(P, rowpoly, s);
-        case 2: return launch_rowpoly_m<2>(P, rowpoly, s);
-        case 3: return launch_rowpoly_m<3>(P, rowpoly, s);
-        case 4: return launch_rowpoly_m<4>(P, rowpoly, s);
-        case 5: return launch_rowpoly_m<5>(P, rowpoly, s);
-        case 6: return launch_rowpoly_m<6>(P, rowpoly, s);
-        case 7: return launch_rowpoly_m<7>(P, rowpoly, s);
-        case 8: return launch_rowpoly_m<8>(P, rowpoly, s);
-    }
-    return cudaErrorInvalidValue;
-}
+int strip2d_rowpoly_stride(int kl_modes) { return s2_gs(kl_modes); }
 
 cudaError_t launch_strip2d(const Params& P, const float* rowpoly, cudaStream_t s) {
     dn_problem p{};
