@@ -38,10 +38,12 @@ FP32_PEAK_LANE_OPS = 148 * 128 * 1.965e9     # SMs x FP32 lanes x max SM clock: 
 # (FADD + FMUL + FFMA + 2 FFMA2).  Each entry names the kernel source it was taken from and the first 16
 # hex digits of its sha256: once that file changes the entry no longer applies and null is reported.
 NCU_CAPTURES = {
-    "tiled2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 501561856, "fp32_ops_per_element": 55.2,
-                                          "src": "dn_tiled2d.cu", "sha": "b475340dd3ea795f"},
-    "tiled3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 571209216, "fp32_ops_per_element": 155.8,
-                                        "src": "dn_tiled3d.cu", "sha": "a93b60c4b75b77cd"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 500476416, "fp32_ops_per_element": 57.6,
+                                          "src": "dn_strip2d.cu", "sha": "347aaf04d621542c"},
+    "tiled2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 794709760, "fp32_ops_per_element": 35.5,
+                                             "src": "dn_tiled2d.cu", "sha": "9a937cc1666dc18f"},
+    "tiled3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 565580800, "fp32_ops_per_element": 155.8,
+                                        "src": "dn_tiled3d.cu", "sha": "a86d3246ea5ce110"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
                                     "src": "dn_burgers.cu", "sha": "baf4524ba7aede8d"},
 }

@@ -300,7 +300,12 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
     const size_t ws_bytes = staging_bytes - off;
 
     // chunks of whole samples; one chunk if a chunk's workspace would not fit (its kernels may tile differently)
+    // ... of at least 8 MiB each, so that small problems are not cut into launches that cost more than they hide
+    const size_t sample_bytes = sizeof(float) * nodes;
     int csize = (p->batch + HostPipe::kMaxChunks - 1) / HostPipe::kMaxChunks;
+    const size_t min_chunk = (size_t)8 << 20;
+    if ((size_t)csize * sample_bytes < min_chunk) csize = (int)((min_chunk + sample_bytes - 1) / sample_bytes);
+    if (csize > p->batch) csize = p->batch;
     int nchunks = (p->batch + csize - 1) / csize;
     {
         dn_problem q = *p;

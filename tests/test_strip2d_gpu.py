@@ -11,10 +11,12 @@ from parity_util import dev, make_problems, run_gpu, check
 
 pytestmark = pytest.mark.gpu
 
-# (nx, ny, batch, m): 256 = first width the kernel takes; 252 + 128 = 380 ends a strip exactly at the grid; 376/384 are
-# one lane short / one lane beyond; 2048 is the bench width; ny = 16 is the shortest grid, 700 spans several chunks
-SIZES = [(256, 40, 2, 4), (260, 17, 3, 1), (376, 33, 2, 6), (380, 16, 2, 2), (384, 21, 1, 3), (504, 50, 2, 5),
-         (508, 20, 2, 8), (1028, 37, 1, 7), (2048, 24, 2, 6), (256, 700, 40, 2)]
+# (nx, ny, batch, m): the kernel takes rows from about 1000 nodes on (narrower ones waste too many lanes) and every
+# width beyond the tiled kernel's 2048.  124 k + 128 = 1120 ends a strip exactly at the grid; 1116 / 1124 are one lane
+# short / one lane beyond; 2048 is the bench width; 2052 and 4096 only this kernel and the any-size kernels can run;
+# ny = 16 is the shortest grid, 700 rows span several chunks
+SIZES = [(1024, 40, 2, 4), (1028, 17, 3, 1), (1116, 33, 2, 6), (1120, 16, 2, 2), (1124, 21, 1, 3), (1500, 50, 2, 5),
+         (2048, 24, 2, 8), (2052, 37, 1, 7), (4096, 19, 2, 6), (1024, 700, 10, 2)]
 
 
 @pytest.mark.parametrize("nx,ny,batch,m", SIZES)
@@ -32,7 +34,7 @@ def test_strip2d_parity(nx, ny, batch, m):
     check(Jg2, rg2, Jo, ro, "generic")
 
 
-@pytest.mark.parametrize("nx,ny", [(256, 37), (380, 19), (520, 23)])
+@pytest.mark.parametrize("nx,ny", [(1024, 37), (1120, 19), (2500, 23)])
 def test_strip2d_options(nx, ny):
     inp = inputs.random_inputs(2, nx, ny, 1, 3, 3, seed=42, f_const=-0.4)
     u = inputs.random_field(inp.u.shape, 8)           # boundary values NOT satisfied
@@ -58,15 +60,15 @@ def test_strip2d_options(nx, ny):
 
 
 def test_strip2d_per_sample_boundary_values():
-    inp = inputs.random_inputs(2, 508, 18, 1, 3, 2, seed=5, f_const=0.3)
+    inp = inputs.random_inputs(2, 1100, 18, 1, 3, 2, seed=5, f_const=0.3)
     u = inputs.random_field(inp.u.shape, 3)
     b0 = np.array([0.9, -0.2, 0.4], dtype=np.float32); b1 = np.array([0.1, 0.7, -0.6], dtype=np.float32)
     _, pg = make_problems(inp, B.DN_NU_KL_GAUSS, flags=B.DN_IMPOSE_BC_ON_LOAD)
     pg.bc_x0_b = dev(b0); pg.bc_x1_b = dev(b1)
     Jg, rg = run_gpu(pg, u)
     for s in range(3):                                 # the oracle, sample by sample with that sample's values
-        one = inputs.random_inputs(2, 508, 18, 1, 3, 2, seed=5, f_const=0.3)
-        po = oracle.Problem(dim=2, nx=508, ny=18, nz=1, batch=1, nu_mode=B.DN_NU_KL_GAUSS, nu=None, kl_modes=2,
+        one = inputs.random_inputs(2, 1100, 18, 1, 3, 2, seed=5, f_const=0.3)
+        po = oracle.Problem(dim=2, nx=1100, ny=18, nz=1, batch=1, nu_mode=B.DN_NU_KL_GAUSS, nu=None, kl_modes=2,
                             kl_w=one.kl_w[s:s + 1], f_const=0.3, f=None, bc_x0=float(b0[s]), bc_x1=float(b1[s]),
                             flags=B.DN_IMPOSE_BC_ON_LOAD)
         Jo, _, _, ro = oracle.energy_grad(po, u[s:s + 1])
