@@ -67,9 +67,9 @@ struct PlaneState {
 // Floats per Gauss row pair (q fixed, s = a and b interleaved) in the coefficient table.
 template <int M> struct Gs3p { static constexpr int value = (2 * (M + 1) + 3) / 4 * 4; };
 
-template <int M, bool WANT_R, bool FULL>
+template <int M, bool WANT_R, bool FULL, bool NARROW>
 __global__ void __launch_bounds__(T3_THREADS, 1)
-tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const int ntile_y) {
+tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const int ntile_y, const int LWarg) {
     extern __shared__ __align__(16) float smem[];
     constexpr bool KL = (M > 0);
     constexpr int MM = KL ? M : 1;
@@ -77,20 +77,25 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     constexpr int NARR = KL ? 4 : 5;                    // exchange arrays: u, e, L1, U1 (, nu)
     const int lane = threadIdx.x & 31;
     const int wid = threadIdx.x >> 5;
-    const int wx = wid % WX, ty = wid / WX;
+    // A node row takes LW lanes: 32, or (NARROW) 16 / 8 on grids with nx <= 64 / 32, where a warp then holds 2 / 4 rows
+    const int LW = NARROW ? LWarg : 32;
+    const int lx = lane & (LW - 1), sub = lane / LW;
+    const bool firstl = (lx == 0), lastl = (lx == LW - 1);
+    const int wx = wid % WX, ty = (wid / WX) * (32 / LW) + sub;
     const int b = blockIdx.y;
     const int tile = blockIdx.x % ntile_y, zc = blockIdx.x / ntile_y;
     const int nx = P.nx, ny = P.ny, nz = P.nz;
     const int NXP = WX * 128;
     const int y0 = tile * TY;
     const int y = y0 + ty;                             // node row and element row of this thread
-    const int x0 = wx * 128 + 4 * lane;
+    const int x0 = wx * 128 + 4 * lx;
     const int p0 = zc * Z, p1 = min(p0 + Z, nz);
     const int kbeg = max(p0 - 1, 0), kend = min(p1 - 1, nz - 2);
     const bool col_ok = FULL || (x0 < nx);
     const bool elem_row_ok = (y < ny - 1);
     const bool out_row = (y < ny);
     const bool top_row = (ty == TY - 1);
+    const bool warp_top = ((wid / WX + 1) * (32 / LW) == TY);       // this warp holds the tile's top row (uniform per warp)
     // the top element row of a tile also feeds the first node row of the next tile: through global scratch
     const bool seam_row = WANT_R && top_row && (tile + 1 < ntile_y) && (y + 1 < ny);
 
@@ -155,7 +160,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
     const float wy = (y == 0 || y == ny - 1) ? 0.5f : 1.f;
     const bool first_col = (x0 == 0), last_col = (x0 + 3 == nx - 1);
     const bool last_elem_missing = (x0 + 3 >= nx - 1);  // element right of node x0+3 does not exist
-    const bool halo_ok = (lane == 31) && (x0 + 4 < nx);
+    const bool halo_ok = lastl && (x0 + 4 < nx);
     const float mfirst = first_col ? 0.f : 1.f, mlast = last_col ? 0.f : 1.f;
 
     const int yl = min(y, ny - 1);                     // rows beyond the grid load a valid address; unused
@@ -222,8 +227,8 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
         }
     };
     auto xdiffs = [&](const float (&v)[4], float halo, float (&e)[4]) {
-        float rn = __shfl_down_sync(0xffffffffu, v[0], 1);
-        if (lane == 31) rn = halo;
+        float rn = __shfl_down_sync(0xffffffffu, v[0], 1, LW);
+        if (lastl) rn = halo;
         e[0] = v[1] - v[0]; e[1] = v[2] - v[1]; e[2] = v[3] - v[2]; e[3] = rn - v[3];
     };
 
@@ -279,7 +284,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 l1[0] = a.x; l1[1] = a.y; l1[2] = a.z; l1[3] = a.w;
                 u1[0] = c4.x; u1[1] = c4.y; u1[2] = c4.z; u1[3] = c4.w;
             }
-            if (lane == 0 && wx > 0) {                 // left warp's last element: (r100, r110, r101, r111)
+            if (firstl && wx > 0) {                 // left warp's last element: (r100, r110, r101, r111)
                 const float4 me = *reinterpret_cast<const float4*>(sX - 4);
                 l1[0] += me.x; u1[0] += me.z;          // to this row: r100 (lower plane), r101 (upper plane)
                 if (ty > 0) {
@@ -296,7 +301,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                     l1v[0] = a.x; l1v[1] = a.y; l1v[2] = a.z; l1v[3] = a.w;
                     u1v[0] = c4.x; u1v[1] = c4.y; u1v[2] = c4.z; u1v[3] = c4.w;
                 }
-                if (lane == 0 && wx > 0) {
+                if (firstl && wx > 0) {
                     const float4 me = *reinterpret_cast<const float4*>(sX - 4);
                     l1v[0] += me.y; u1v[0] += me.w;
                 }
@@ -331,6 +336,9 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
         // ---- finish staging plane p (needs row y+1) and compute element plane p-1
         if (stage) {
             float uab[4], eab[4];
+            // a warp that holds several rows has lanes on both sides of `top_row`: its shuffles run for the whole warp
+            float eab_top[4] = {0.f, 0.f, 0.f, 0.f};
+            if constexpr (NARROW) { if (warp_top) xdiffs(ua, uah, eab_top); }
             if (!top_row) {
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f), c4 = a;
                 if (col_ok) {
@@ -342,7 +350,12 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
             } else {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) uab[c] = ua[c];
-                xdiffs(ua, uah, eab);
+                if constexpr (NARROW) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) eab[c] = eab_top[c];
+                } else {
+                    xdiffs(ua, uah, eab);               // top_row is uniform in the warp
+                }
                 if (p <= kend) load4(pa + (size_t)(p + 1) * plane, ua, uah);
             }
 #pragma unroll
@@ -350,6 +363,8 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
             if constexpr (!KL) {
                 // nu of the staged plane at the 4 (xi, eta) points of each element: x lerp on rows y and y+1, then y lerp
                 float nab[5];
+                float rn_top = 0.f;
+                if (NARROW ? warp_top : top_row) rn_top = __shfl_down_sync(0xffffffffu, na[0], 1, LW);
                 if (!top_row) {
                     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
                     float a4 = 0.f;
@@ -359,13 +374,12 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                     }
                     nab[0] = a.x; nab[1] = a.y; nab[2] = a.z; nab[3] = a.w; nab[4] = a4;
                 } else {
-                    float rn = __shfl_down_sync(0xffffffffu, na[0], 1);
-                    if (lane == 31) rn = nah;
+                    const float rn = lastl ? nah : rn_top;
                     nab[0] = na[0]; nab[1] = na[1]; nab[2] = na[2]; nab[3] = na[3]; nab[4] = rn;
                     if (p <= kend) load4n(pna + (size_t)(p + 1) * plane, na, nah);
                 }
-                float nrn = __shfl_down_sync(0xffffffffu, up.n[0], 1);
-                if (lane == 31) nrn = up.nh;
+                float nrn = __shfl_down_sync(0xffffffffu, up.n[0], 1, LW);
+                if (lastl) nrn = up.nh;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const float n0 = up.n[c], n1 = (c < 3) ? up.n[c < 3 ? c + 1 : c] : nrn;
@@ -479,9 +493,9 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                 }
                 if (WANT_R) {
                     // the left neighbour's last element feeds this thread's first node column
-                    const float a100 = __shfl_up_sync(0xffffffffu, L0p[4], 1), a110 = __shfl_up_sync(0xffffffffu, L1[4], 1);
-                    const float a101 = __shfl_up_sync(0xffffffffu, U0p[4], 1), a111 = __shfl_up_sync(0xffffffffu, U1[4], 1);
-                    if (lane > 0) { L0p[0] += a100; L1[0] += a110; U0p[0] += a101; U1[0] += a111; }
+                    const float a100 = __shfl_up_sync(0xffffffffu, L0p[4], 1, LW), a110 = __shfl_up_sync(0xffffffffu, L1[4], 1, LW);
+                    const float a101 = __shfl_up_sync(0xffffffffu, U0p[4], 1, LW), a111 = __shfl_up_sync(0xffffffffu, U1[4], 1, LW);
+                    if (!firstl) { L0p[0] += a100; L1[0] += a110; U0p[0] += a101; U1[0] += a111; }
                     // what goes to row y+1 and to the warp on the right is published by the next step's
                     // barrier: write it into the other exchange buffer now (its readers finished before
                     // this step's barrier)
@@ -490,7 +504,7 @@ tiled3d_kernel(const Params P, const int WX, const int TY, const int Z, const in
                         *reinterpret_cast<float4*>(so + 2 * TYNXP) = make_float4(L1[0], L1[1], L1[2], L1[3]);
                         *reinterpret_cast<float4*>(so + 3 * TYNXP) = make_float4(U1[0], U1[1], U1[2], U1[3]);
                     }
-                    if (lane == 31)
+                    if (lastl)
                         *reinterpret_cast<float4*>(smem + (PAR ^ 1) * BUF + XOFF + (ty * WX + wx) * 4) =
                             make_float4(L0p[4], L1[4], U0p[4], U1[4]);
                 }
@@ -555,7 +569,7 @@ __global__ void seam_fixup_kernel(float* __restrict__ r, const float* __restrict
     *dst = v;
 }
 
-struct Geo3 { int WX, TY, Z, ntile_y, nchunk_z, GS, bps; size_t smem; };
+struct Geo3 { int WX, TY, Z, ntile_y, nchunk_z, GS, bps, LW; size_t smem; };
 
 int sm_count3() {
     int dev = 0, n = 0;
@@ -574,65 +588,69 @@ Geo3 geometry3(const dn_problem& p) {
     const int GS = m ? (2 * (m + 1) + 3) / 4 * 4 : 0;               // floats per Gauss-row line pair
     const int sms = sm_count3();
     double best_cost = -1.0;
-    const int ty_max = (T3_THREADS / 32) / WX;
+    const int LW = (nx <= 32) ? 8 : (nx <= 64) ? 16 : 32;          // lanes per node row
+    const int RPW = 32 / LW;                                         // node rows per warp
+    const int ty_max = (T3_THREADS / 32) / WX * RPW;
     // Tiles do not overlap, so any tile height works.  Pick (TY, Z) by a cost model fitted to sweeps on
     // B200: work grows with the warm-up plane of every z chunk, blocks should fill whole waves, an SM
     // wants 16 resident warps (128 registers each) in more than one block (barriers), and very flat tiles
     // pay more seam traffic.
-    for (int TY = 2; TY <= ty_max; ++TY) {
-        if (TY > ny && TY > 2) break;
-        int bps = 16 / (WX * TY);                                    // blocks per SM by registers
+    for (int TY = (RPW > 2 ? RPW : 2); TY <= ty_max; TY += (RPW > 1 ? RPW : 1)) {
+        if (TY > ny && TY > 2 * RPW) break;
+        const int TYW = TY / RPW;                                    // warp rows of a block
+        int bps = 16 / (WX * TYW);                                   // blocks per SM by registers
         if (bps < 1) bps = 1;
         if (bps > 4) bps = 4;
-        const int warps = bps * WX * TY;
+        const int warps = bps * WX * TYW;
         const long long ntile = (ny + TY - 1) / TY;
         const size_t fixed = sizeof(float) * 2 * ((size_t)(m ? 4 : 5) * TY * WX * 128 + (size_t)TY * WX * 4);
         for (int Z = 4; Z <= 256; ++Z) {
             if (Z > nz && Z > 4) break;
-            const size_t sm = fixed + sizeof(float) * (size_t)(Z + 1) * TY * 2 * GS + (m ? (size_t)16 * 4 * 32 * WX * TY : 0);
+            const size_t sm = fixed + sizeof(float) * (size_t)(Z + 1) * TY * 2 * GS + (m ? (size_t)16 * 4 * 32 * WX * TYW : 0);
             if (sm * bps > 200 * 1024) break;
             const long long nch = (nz + Z - 1) / Z;
             const long long blocks = (long long)p.batch * ntile * nch;
             const long long slots = (long long)sms * bps;
             const long long waves = (blocks + slots - 1) / slots;
-            const double work = (double)blocks * (Z + 3) * TY;
+            const double work = (double)blocks * (Z + 3) * TYW;
             const double imbalance = (double)waves * slots / (double)blocks;
             const double cost = work * imbalance * (16.0 / warps) * (1.0 + 0.1 / TY) * (1.0 + 0.05 / bps);
             if (best_cost < 0 || cost < best_cost) {
                 best_cost = cost;
                 best.WX = WX; best.TY = TY; best.Z = Z; best.ntile_y = (int)ntile; best.nchunk_z = (int)nch;
-                best.GS = GS; best.bps = bps; best.smem = sm;
+                best.GS = GS; best.bps = bps; best.smem = sm; best.LW = LW;
             }
         }
     }
     return best;
 }
 
-template <int M, bool FULL>
+template <int M, bool FULL, bool NARROW>
 cudaError_t launch_mf(const Params& P, const Geo3& g, cudaStream_t s) {
     dim3 grid((unsigned)(g.ntile_y * g.nchunk_z), (unsigned)P.batch);
-    const int threads = 32 * g.WX * g.TY;
+    const int threads = 32 * g.WX * g.TY / (32 / g.LW);
     cudaError_t e;
     if (P.r) {
-        e = cudaFuncSetAttribute(tiled3d_kernel<M, true, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+        e = cudaFuncSetAttribute(tiled3d_kernel<M, true, FULL, NARROW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
         if (e != cudaSuccess) return e;
-        tiled3d_kernel<M, true, FULL><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y);
+        tiled3d_kernel<M, true, FULL, NARROW><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y, g.LW);
         if (g.ntile_y > 1) {
             const long long total4 = (long long)P.batch * (g.ntile_y - 1) * P.nz * (P.nx / 4);
             seam_fixup_kernel<<<(unsigned)((total4 + 255) / 256), 256, 0, s>>>(P.r, P.seam, P.nx, P.ny, P.nz, g.TY,
                                                                               g.ntile_y - 1, total4);
         }
     } else {
-        e = cudaFuncSetAttribute(tiled3d_kernel<M, false, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
+        e = cudaFuncSetAttribute(tiled3d_kernel<M, false, FULL, NARROW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
         if (e != cudaSuccess) return e;
-        tiled3d_kernel<M, false, FULL><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y);
+        tiled3d_kernel<M, false, FULL, NARROW><<<grid, threads, g.smem, s>>>(P, g.WX, g.TY, g.Z, g.ntile_y, g.LW);
     }
     return cudaGetLastError();
 }
 
 template <int M>
 cudaError_t launch_m(const Params& P, const Geo3& g, cudaStream_t s) {
-    return (g.WX * 128 == P.nx) ? launch_mf<M, true>(P, g, s) : launch_mf<M, false>(P, g, s);
+    if (g.LW < 32) return launch_mf<M, false, true>(P, g, s);
+    return (g.WX * 128 == P.nx) ? launch_mf<M, true, false>(P, g, s) : launch_mf<M, false, false>(P, g, s);
 }
 
 }  // namespace

@@ -36,7 +36,9 @@ def test_workload_parity_full(cfg, mode, force_generic):
 ODD = [(2, 2, 2, 1, 1, 1), (2, 3, 2, 1, 2, 2), (2, 5, 9, 1, 3, 3), (2, 64, 7, 1, 2, 4), (2, 130, 67, 1, 2, 6),
        (2, 257, 33, 1, 1, 8), (2, 516, 40, 1, 2, 5), (2, 1028, 19, 1, 1, 2),
        (3, 2, 2, 2, 1, 1), (3, 3, 4, 5, 2, 2), (3, 9, 5, 7, 2, 3), (3, 36, 10, 6, 2, 2), (3, 132, 9, 5, 1, 3),
-       (3, 64, 20, 3, 1, 2), (3, 260, 6, 4, 1, 2)]
+       (3, 64, 20, 3, 1, 2), (3, 260, 6, 4, 1, 2),
+       # narrow 3D grids: a warp holds 4 rows (nx <= 32) or 2 rows (nx <= 64) of the tile; several tiles with seams
+       (3, 12, 11, 6, 2, 2), (3, 32, 9, 7, 3, 3), (3, 28, 45, 5, 1, 2), (3, 60, 37, 6, 2, 3)]
 
 
 @pytest.mark.parametrize("mode", MODES)
