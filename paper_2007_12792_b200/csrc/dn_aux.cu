@@ -66,6 +66,7 @@ __device__ void rowpoly_entry(const TableArgs& A, long long idx) {
     for (int k = 0; k <= MX; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
 #pragma unroll
     for (int i = 1; i <= MX; ++i) {
+        if (i > m) break;                              // uniform; the rest of the terms are zero
 #pragma unroll
         for (int k = 0; k <= MX; ++k) acc[k] += g[i - 1] * tc[k];
         double tn[MX + 1];

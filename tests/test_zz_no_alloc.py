@@ -29,7 +29,11 @@ def test_static_scratch_matches_workspace_entry_point_on_consecutive_calls():
     # two calls in a row with different problems (2D KL, then 3D nodal, then 2D again): the array
     # still holds the previous call's tables and partials each time
     cases = [(inputs.make_inputs(0), B.DN_NU_KL_GAUSS), (inputs.make_inputs(3, samples=range(2)), B.DN_NU_NODAL),
-             (inputs.make_inputs(1, samples=range(4)), B.DN_NU_KL_GAUSS), (inputs.make_inputs(0), B.DN_NU_KL_GAUSS)]
+             (inputs.make_inputs(1, samples=range(4)), B.DN_NU_KL_GAUSS), (inputs.make_inputs(0), B.DN_NU_KL_GAUSS),
+             # wide 2D rows: the strip kernel when its coefficient table fits the array, else the tiled kernel
+             (inputs.random_inputs(2, 1024, 64, 1, 2, 4, seed=9, f_const=0.5), B.DN_NU_KL_GAUSS),
+             (inputs.random_inputs(2, 1024, 4000, 1, 6, 6, seed=10), B.DN_NU_KL_GAUSS),
+             (inputs.make_inputs(0), B.DN_NU_KL_GAUSS)]
     for inp, mode in cases:
         nu = None
         if mode == B.DN_NU_NODAL:
