@@ -40,10 +40,10 @@ FP32_PEAK_LANE_OPS = 148 * 128 * 1.965e9     # SMs x FP32 lanes x max SM clock: 
 NCU_CAPTURES = {
     "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 500476416, "fp32_ops_per_element": 57.6,
                                           "src": "dn_strip2d.cu", "sha": "347aaf04d621542c"},
-    "tiled2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 794709760, "fp32_ops_per_element": 35.5,
-                                             "src": "dn_tiled2d.cu", "sha": "9a937cc1666dc18f"},
-    "tiled3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 565811968, "fp32_ops_per_element": 155.8,
-                                        "src": "dn_tiled3d.cu", "sha": "7c131b2c3c48a28c"},
+    "tiled2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 792350208, "fp32_ops_per_element": 35.5,
+                                             "src": "dn_tiled2d.cu", "sha": "83d5769163988ff7"},
+    "tiled3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 565575168, "fp32_ops_per_element": 155.8,
+                                        "src": "dn_tiled3d.cu", "sha": "44f694b4e7cf5939"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
                                     "src": "dn_burgers.cu", "sha": "baf4524ba7aede8d"},
 }
@@ -483,16 +483,30 @@ def main():
         sampler.start()
         time.sleep(0.15)
     t0 = time.time()
+    # the K timed steps: the plain call a user makes (no events inside it).  Inputs larger than L2: one event pair
+    # around all K steps; otherwise one pair per step, so that the L2 flush between steps stays outside the timing.
+    if flush is None:
+        ev_step[0][0].record()
+        for k in range(K):
+            B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
+        ev_step[0][1].record()
+    else:
+        for k in range(K):
+            flush.zero_()
+            ev_step[k][0].record()
+            B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
+            ev_step[k][1].record()
+    barrier()
+    step_ms = (ev_step[0][0].elapsed_time(ev_step[0][1]) if flush is None
+               else sum(a.elapsed_time(b_) for a, b_ in ev_step)) / K
+    # K more steps with events around the fused kernel alone (the roofline's kernel time)
     for k in range(K):
         if flush is not None:
-            flush.zero_()                      # evict L2 between timed steps (outside the per-step events)
-        ev_step[k][0].record()
+            flush.zero_()
         B.dn_energy_grad_traced(prob, u, None, J, r, ws, ev_main[k][0], ev_main[k][1], _cstruct=cs)
-        ev_step[k][1].record()
     barrier()
     t1 = time.time()
     clocks = sampler.stop(t0, t1) if rank == 0 else None
-    step_ms = sum(a.elapsed_time(b_) for a, b_ in ev_step) / K
     main_ms = sum(a.elapsed_time(b_) for a, b_ in ev_main) / K
     Jsum = float(J.double().sum())
 

@@ -139,7 +139,6 @@ __device__ __forceinline__ void element3d(const Params& P, int b, int ex, int ey
     float u[8];
     for (int a = 0; a < 8; ++a)
         u[a] = load_u(P, b, ub, ex + (a & 1), i0 + (a & 1) + ((a >> 1) & 1) * sy + ((a >> 2) & 1) * sz);
-    const float ga[2] = {DN_GA, DN_GB};
     const float L[2][2] = {{1.f - DN_GA, DN_GA}, {1.f - DN_GB, DN_GB}};   // L[point][corner bit]
     float nuq[2][2][2];                                                     // [p: xi][q: eta][s: zeta]
     if (P.nu_mode != DN_NU_KL_GAUSS) {

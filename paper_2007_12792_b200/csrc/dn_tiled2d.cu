@@ -215,7 +215,6 @@ tiled2d_kernel(const Params P, const int W, const int WY, const int R) {
 
     if (!idle) {
         const int x0 = (wx * 32 + lane) * NE;
-        const int xhalo = x0 + NE;                      // node right of this lane's nodes
         const bool warp_has_halo = (wx * 32 + 32) * NE < nx;
         const float* ub = P.u + (size_t)b * P.nodes;
         const float* nub = NLOAD ? P.nu + (size_t)b * P.nodes : nullptr;

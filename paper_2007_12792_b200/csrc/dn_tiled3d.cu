@@ -43,11 +43,6 @@ __device__ __forceinline__ float ex2_approx3(float x) {
 
 typedef unsigned long long u64;
 
-__device__ __forceinline__ u64 pack2_3(float lo, float hi) {
-    u64 v;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
-    return v;
-}
 __device__ __forceinline__ void unpack2_3(u64 v, float& lo, float& hi) {
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
