@@ -118,7 +118,11 @@ dn_status dn_energy(const dn_problem* problem, const float* u, float* J, void* w
 /* Energy and its exact gradient in one pass over u (Algorithm 1: loss, then its gradient
  * for back-propagation):  r = K(nu) u - F, zeroed at Dirichlet nodes unless DN_NO_MASK,
  * multiplied by gJ[b] when gJ != NULL (the upstream dLoss/dJ_b).
- * J may be NULL (residual only).  r must not overlap u.  gJ: [B] floats or NULL. */
+ * J may be NULL (residual only).  r must not overlap u.  gJ: [B] floats or NULL.
+ * Errors found before anything is enqueued come back as a status and leave the outputs untouched.
+ * The kernels contain no unbounded wait: where warps of the tiled 2D kernel hand values to one
+ * another, the wait has an iteration limit, and should it ever run out the energy J[b] of that
+ * sample is returned as NaN (its residual is then not to be trusted either). */
 dn_status dn_energy_grad(const dn_problem* problem, const float* u, const float* gJ, float* J, float* r,
                          void* workspace, size_t workspace_bytes, void* stream);
 
@@ -246,7 +250,7 @@ const char* dn_burgers_path_name(const dn_burgers* problem, const float* u, cons
  * dn_energy_grad call (for launch accounting); 0 if the problem is invalid. */
 int32_t dn_launches_per_call(const dn_problem* problem);
 
-/* Name of the kernel family that dn_energy_grad would use ("tiled2d", "tiled3d", "generic"). */
+/* Name of the kernel family that dn_energy_grad would use ("strip2d", "tiled2d", "tiled3d", "generic"). */
 const char* dn_path_name(const dn_problem* problem);
 
 const char* dn_status_string(dn_status status);
