@@ -39,7 +39,9 @@ def test_fullsize_sampled(cfg, mode):
     idx = rng.integers(0, inp.batch * nodes, size=30000)
     n = wl.n
     special = []
-    coords = [0, 1, 2, 3, 4, 123, 124, 127, 128, 129, 251, 252, 255, 256, n // 2 - 1, n // 2, n - 5, n - 4, n - 3, n - 2, n - 1]
+    # 124 k .. 124 k + 4: where neighbouring strips of the 2D strip kernel overlap; 128 / 256: warp seams of the tiled kernels
+    coords = [0, 1, 2, 3, 4, 123, 124, 127, 128, 129, 247, 248, 251, 252, 255, 256, 371, 372, 375, 376, 1983, 1984, 1987, 1988,
+              n // 2 - 1, n // 2, n - 5, n - 4, n - 3, n - 2, n - 1]
     coords = sorted({c for c in coords if 0 <= c < n})
     for b in (0, inp.batch - 1):
         for iy in coords:
