@@ -141,7 +141,7 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
                         reinterpret_cast<float*>(base + w.cn[2])};
         e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
                           (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
-                          strip2d_rowpoly_stride(p->kl_modes));
+                          strip2d_rowpoly_stride(p->kl_modes), p->nu_mode == DN_NU_KL_NODAL);
         if (e != cudaSuccess) return DN_ERR_CUDA;
     }
     if (ev_before && cudaEventRecord(static_cast<cudaEvent_t>(ev_before), s) != cudaSuccess) return DN_ERR_CUDA;
@@ -176,7 +176,7 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
                         reinterpret_cast<float*>(base + w.cn[2])};
         e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
                           (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
-                          strip2d_rowpoly_stride(p->kl_modes));
+                          strip2d_rowpoly_stride(p->kl_modes), p->nu_mode == DN_NU_KL_NODAL);
         if (e != cudaSuccess) return DN_ERR_CUDA;
     }
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);

@@ -26,6 +26,7 @@ struct TableArgs {
     float* cn[3];
     float* rowpoly;       // 2D, optional: polynomial of the KL exponent along every Gauss row, [B][ny-1][rp_gs]
     int rp_gs;
+    int rp_nodes;         // 0: the two Gauss rows of every element row, interleaved; 1: every node row, each coefficient twice
 };
 
 // exponent(x, y_q) = sum_k poly[k] c^k with c = cos(pi x), for the Gauss row q of element row j of sample b:
@@ -38,15 +39,19 @@ __device__ void rowpoly_entry(const TableArgs& A, long long idx) {
     constexpr int MX = DN_MAX_KL_MODES;
     const int m = A.m, ny = A.n[1];
     const int q = (int)(idx & 1);
-    const long long row = idx >> 1;                    // b * (ny - 1) + j
-    const int j = (int)(row % (ny - 1));
-    const long long b = row / (ny - 1);
+    const int rows = A.rp_nodes ? ny : ny - 1;
+    const long long row = idx >> 1;                    // b * rows + j
+    const int j = (int)(row % rows);
+    const long long b = row / rows;
     const double ga = 0.5 * (1.0 - 0.57735026918962576451);
     const double gb = 0.5 * (1.0 + 0.57735026918962576451);
     const double y = ((double)j + (q ? gb : ga)) / (double)(ny - 1);
     double cy[MX], g[MX];
 #pragma unroll
-    for (int jj = 0; jj < MX; ++jj) cy[jj] = (jj < m) ? (double)(float)cospi((double)(jj + 1) * y) : 0.0;
+    for (int jj = 0; jj < MX; ++jj) {
+        const double arg = A.rp_nodes ? (double)(jj + 1) * (double)j / (double)(ny - 1) : (double)(jj + 1) * y;   // as the tables
+        cy[jj] = (jj < m) ? (double)(float)cospi(arg) : 0.0;
+    }
     const float* w = A.kl_w + b * m * m;
 #pragma unroll
     for (int i = 0; i < MX; ++i) {
@@ -124,7 +129,7 @@ __global__ void tables_kernel(TableArgs A) {
         }
         idx -= cnt;
     }
-    if (A.rowpoly && idx < 2ll * A.batch * (A.n[1] - 1)) rowpoly_entry(A, idx);
+    if (A.rowpoly && idx < 2ll * A.batch * (A.n[1] - (A.rp_nodes ? 0 : 1))) rowpoly_entry(A, idx);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -301,7 +306,7 @@ __global__ void apply_bc_kernel(long long lines, long long lines_per_sample, int
 }  // namespace
 
 cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], float* const cn[3],
-                          cudaStream_t s, float* rowpoly, int rowpoly_stride) {
+                          cudaStream_t s, float* rowpoly, int rowpoly_stride, bool rowpoly_nodes) {
     TableArgs A{};
     A.dim = P.dim; A.m = P.m; A.batch = P.batch;
     A.n[0] = P.nx; A.n[1] = P.ny; A.n[2] = P.nz;
@@ -313,8 +318,8 @@ cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float*
         if (a < P.dim) total += (long long)P.m * (P.gstride[a] + P.nstride[a]);
     }
     A.kl_w = kl_w; A.ckl = ckl;
-    A.rowpoly = (P.dim == 2) ? rowpoly : nullptr; A.rp_gs = rowpoly_stride;
-    if (A.rowpoly) total += 2ll * P.batch * (P.ny - 1);
+    A.rowpoly = (P.dim == 2) ? rowpoly : nullptr; A.rp_gs = rowpoly_stride; A.rp_nodes = rowpoly_nodes ? 1 : 0;
+    if (A.rowpoly) total += 2ll * P.batch * (P.ny - (rowpoly_nodes ? 0 : 1));
     const int threads = 128;
     tables_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, s>>>(A);
     return cudaGetLastError();

@@ -79,7 +79,8 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
 
 // rowpoly (optional, 2D): also writes the per-Gauss-row polynomials the strip kernel reads, rows of rowpoly_stride floats
 cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], float* const cn[3],
-                          cudaStream_t s, float* rowpoly = nullptr, int rowpoly_stride = 0);
+                          cudaStream_t s, float* rowpoly = nullptr, int rowpoly_stride = 0,
+                          bool rowpoly_nodes = false);   // rowpoly_nodes: one polynomial per node row (KL at the nodes)
 cudaError_t launch_generic(const Params& P, cudaStream_t s);
 cudaError_t launch_tiled2d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s);

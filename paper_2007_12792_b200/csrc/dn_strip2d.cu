@@ -1,4 +1,5 @@
-// Strip kernel for 2D grids, KL diffusivity at the Gauss points, energy and residual fused.
+// Strip kernel for 2D grids, KL diffusivity evaluated in the kernel (at the Gauss points, or at the nodes and then
+// interpolated), energy and residual fused.
 //
 // Layout of the work.  A warp is a work unit of its own: one sample, one chunk of R node rows, one
 // strip of 128 node columns (4 consecutive nodes per lane).  Strips overlap by one lane: lane 0 of
@@ -20,7 +21,7 @@
 // each derivative's own axis; chain rule to the four corners).  The diffusion energy is taken from
 // the residual by Euler's identity for quadratic forms: 1/2 sum_i u_i (K u)_i.
 //
-// KL diffusivity: for a fixed Gauss row the exponent is a polynomial of degree m in c = cos(pi x).
+// KL diffusivity: for a fixed Gauss row (or, with KN, node row) the exponent is a polynomial of degree m in c = cos(pi x).
 // The table kernel prepares its coefficients in double once per call (they do not depend on u), for
 // both Gauss rows of every element row, interleaved so that the two rows are evaluated together
 // with packed two-wide FMAs.
@@ -72,7 +73,7 @@ template <int N> __device__ __forceinline__ void s2_wait() { asm volatile("cp.as
 // Floats per element row in the coefficient table: (row a, row b) pairs for k = 0..M, padded to a multiple of 4.
 __host__ __device__ constexpr int s2_gs(int m) { return (2 * (m + 1) + 3) / 4 * 4; }
 
-template <int M, int BPS>
+template <int M, int BPS, bool KN>
 __global__ void __launch_bounds__(S2_WARPS * 32, BPS)
 strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, const int nchunk, const int nstrip) {
     extern __shared__ __align__(16) float smem[];
@@ -131,7 +132,13 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
 
     // cos(pi x) at the two Gauss columns of each element, duplicated into both halves of a pair
     u64 cda[NE], cdb[NE];
-    {
+    u64 cnp[NE / 2];                                    // KN: cos(pi x) at this lane's nodes (pairs) and at the node right of them
+    float cnh = 0.f;
+    if constexpr (KN) {
+        const float4 q = __ldg(reinterpret_cast<const float4*>(P.cn[0] + x0c));
+        cnp[0] = s2_pack(q.x, q.y); cnp[1] = s2_pack(q.z, q.w);
+        cnh = __ldg(P.cn[0] + x0c + NE);
+    } else {
         const float4 q0 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0c));
         const float4 q1 = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0c + 4));
         cda[0] = s2_pack(q0.x, q0.x); cdb[0] = s2_pack(q0.y, q0.y);
@@ -146,7 +153,9 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
     const float* usrc = ub + (size_t)(jbeg + 1) * nx;
     const bool xcoef = (lane < GS / 4), xhalo = (lane == 31) && has_halo;
     const int xp = (xcoef || xhalo) ? 1 : 0;            // this lane makes a second copy per row
-    const float* xsrc = xcoef ? rowpoly + ((size_t)b * (ny - 1) + jbeg) * GS + 4 * lane : usrc + NE;
+    // coefficient rows: per element row (its two Gauss rows), or with KN per node row (the row that arrives with it)
+    const float* polyb = rowpoly + (size_t)b * (KN ? ny : ny - 1) * GS;
+    const float* xsrc = xcoef ? polyb + (size_t)(KN ? jbeg + 1 : jbeg) * GS + 4 * lane : usrc + NE;
     const int xstep = xcoef ? GS : nx;
     const int xdst = xcoef ? S2_COLS + 4 + 4 * lane : S2_COLS;
     auto issue = [&](float* slot) {
@@ -178,6 +187,34 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         for (int k = 0; k < NE; ++k) U[k] = 0.f;
     }
 
+    // KN: nu at this lane's 4 nodes and at the node right of them, from the polynomial of that node row
+    auto nu_row = [&](const u64 (&gg)[GS / 2], float (&nn)[NE + 1]) {
+#pragma unroll
+        for (int h = 0; h < NE / 2; ++h) {
+            u64 e = gg[M];
+#pragma unroll
+            for (int i = M - 1; i >= 0; --i) e = s2_fma2(e, cnp[h], gg[i]);
+            float e0, e1;
+            s2_unpack(e, e0, e1);
+            nn[2 * h] = s2_ex2(e0); nn[2 * h + 1] = s2_ex2(e1);
+        }
+        float gh, dmy;
+        s2_unpack(gg[M], gh, dmy);
+#pragma unroll
+        for (int i = M - 1; i >= 0; --i) { float gi; s2_unpack(gg[i], gi, dmy); gh = fmaf(gh, cnh, gi); }
+        nn[NE] = s2_ex2(gh);
+    };
+    float nlo[NE + 1], hnu[NE];                         // KN: nu on the node row below and its sums over x-neighbours
+    if constexpr (KN) {
+        u64 gg[GS / 2];
+        const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(polyb + (size_t)jbeg * GS);
+#pragma unroll
+        for (int k = 0; k < GS / 4; ++k) { const ulonglong2 t = __ldg(gp + k); gg[2 * k] = t.x; gg[2 * k + 1] = t.y; }
+        nu_row(gg, nlo);
+#pragma unroll
+        for (int k = 0; k < NE; ++k) hnu[k] = nlo[k] + nlo[k + 1];
+    }
+
     float en = 0.f, ell = 0.f;                          // sum u (K u) and sum w u of the rows this lane went over
     float* rrow = rb + (size_t)jbeg * nx;
     int rd = 0;                                         // float offset of the slot to read; the one before it is refilled
@@ -204,6 +241,8 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             if (has_first) c[0] = bc0;
             if (has_last) c[NE - 1] = bc1;
         }
+        float ncur[NE + 1];
+        if constexpr (KN) nu_row(g2, ncur);
         float hir = __shfl_down_sync(0xffffffffu, c[0], 1);
         if (lane == 31) hir = has_halo ? halo : 0.f;
 
@@ -219,14 +258,25 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             const float t = e1 - e0;
             const float Dxa = fmaf(DN_GA, t, e0), Dxb = fmaf(DN_GB, t, e0);
             const float Dya = fmaf(DN_GA, t, s0), Dyb = fmaf(DN_GB, t, s0);
-            u64 ea = g2[M], eb = g2[M];                 // (row a, row b) pairs at column a / column b
+            float Na, Nb, Ma, Mb;
+            if constexpr (KN) {
+                // Q1 interpolation of the nodal values to the Gauss points, summed along each derivative's own axis
+                const float h0 = hnu[k], h1 = ncur[k] + ncur[k + 1];
+                hnu[k] = h1;
+                const float v0 = nlo[k] + ncur[k], v1 = nlo[k + 1] + ncur[k + 1];
+                const float dh = h1 - h0, dv = v1 - v0;
+                Na = fmaf(DN_GA, dh, h0); Nb = fmaf(DN_GB, dh, h0);
+                Ma = fmaf(DN_GA, dv, v0); Mb = fmaf(DN_GB, dv, v0);
+            } else {
+                u64 ea = g2[M], eb = g2[M];             // (row a, row b) pairs at column a / column b
 #pragma unroll
-            for (int i = M - 1; i >= 0; --i) { ea = s2_fma2(ea, cda[k], g2[i]); eb = s2_fma2(eb, cdb[k], g2[i]); }
-            float xaa, xab, xba, xbb;
-            s2_unpack(ea, xaa, xab);
-            s2_unpack(eb, xba, xbb);
-            const float naa = s2_ex2(xaa), nab = s2_ex2(xab), nba = s2_ex2(xba), nbb = s2_ex2(xbb);
-            const float Na = naa + nba, Nb = nab + nbb, Ma = naa + nab, Mb = nba + nbb;
+                for (int i = M - 1; i >= 0; --i) { ea = s2_fma2(ea, cda[k], g2[i]); eb = s2_fma2(eb, cdb[k], g2[i]); }
+                float xaa, xab, xba, xbb;
+                s2_unpack(ea, xaa, xab);
+                s2_unpack(eb, xba, xbb);
+                const float naa = s2_ex2(xaa), nab = s2_ex2(xab), nba = s2_ex2(xba), nbb = s2_ex2(xbb);
+                Na = naa + nba; Nb = nab + nbb; Ma = naa + nab; Mb = nba + nbb;
+            }
             const float Gxa = Na * Dxa, Gxb = Nb * Dxb, Gya = Ma * Dya, Gyb = Mb * Dyb;
             const float SXu = Gxa + Gxb, SYu = Gya + Gyb;
             float T = kxa * Gxa;
@@ -265,6 +315,10 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             if (owner) *reinterpret_cast<float4*>(rrow) = o;
         }
         rrow += nx;
+        if constexpr (KN) {
+#pragma unroll
+            for (int k = 0; k <= NE; ++k) nlo[k] = ncur[k];
+        }
     };
 
     {
@@ -338,15 +392,20 @@ GeoS geometry_s(const dn_problem& p) {
     return g;
 }
 
-template <int M>
-cudaError_t launch_m(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
+template <int M, bool KN>
+cudaError_t launch_mk(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
     const size_t smem = sizeof(float) * S2_WARPS * S2_DEPTH * S2_SLOT;
     const long long units = (long long)P.batch * g.nchunk * g.nstrip;
     const unsigned blocks = (unsigned)((units + S2_WARPS - 1) / S2_WARPS);
-    const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2, KN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    strip2d_kernel<M, 2><<<blocks, S2_WARPS * 32, smem, s>>>(P, rowpoly, g.R, g.nchunk, g.nstrip);
+    strip2d_kernel<M, 2, KN><<<blocks, S2_WARPS * 32, smem, s>>>(P, rowpoly, g.R, g.nchunk, g.nstrip);
     return cudaGetLastError();
+}
+
+template <int M>
+cudaError_t launch_m(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
+    return (P.nu_mode == DN_NU_KL_NODAL) ? launch_mk<M, true>(P, rowpoly, g, s) : launch_mk<M, false>(P, rowpoly, g, s);
 }
 
 }  // namespace
@@ -355,7 +414,7 @@ cudaError_t launch_m(const Params& P, const float* rowpoly, const GeoS& g, cudaS
 // row takes 3 strips of 128).  The tiled kernel is about 1.16 times slower per element in this mode: the strip
 // kernel takes over where its lanes are at most 15 % more than the row, and wherever the tiled kernel cannot run.
 bool strip2d_applicable(const dn_problem& p) {
-    if (!(p.grid.dim == 2 && p.nu_mode == DN_NU_KL_GAUSS && p.f == nullptr && p.grid.nx % 4 == 0 &&
+    if (!(p.grid.dim == 2 && (p.nu_mode == DN_NU_KL_GAUSS || p.nu_mode == DN_NU_KL_NODAL) && p.f == nullptr && p.grid.nx % 4 == 0 &&
           p.grid.nx >= 2 * S2_COLS && p.grid.ny >= 16))
         return false;
     const long long lanes = (long long)((p.grid.nx - S2_COLS + S2_STRIDE - 1) / S2_STRIDE + 1) * S2_COLS;
@@ -373,7 +432,7 @@ Launch strip2d_geometry(const dn_problem& p) {
 }
 
 size_t strip2d_rowpoly_floats(const dn_problem& p) {
-    return (size_t)p.batch * (p.grid.ny - 1) * s2_gs(p.kl_modes);
+    return (size_t)p.batch * p.grid.ny * s2_gs(p.kl_modes);      // ny - 1 element rows, or ny node rows (KL at the nodes)
 }
 
 int strip2d_rowpoly_stride(int kl_modes) { return s2_gs(kl_modes); }
