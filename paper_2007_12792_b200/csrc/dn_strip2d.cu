@@ -1,5 +1,5 @@
-// Strip kernel for 2D grids, KL diffusivity evaluated in the kernel (at the Gauss points, or at the nodes and then
-// interpolated), energy and residual fused.
+// Strip kernel for wide 2D grids, energy and residual fused, in all three diffusivity modes: KL evaluated in the
+// kernel at the Gauss points, KL evaluated at the nodes and then interpolated, or a stored nodal field.
 //
 // Layout of the work.  A warp is a work unit of its own: one sample, one chunk of R node rows, one
 // strip of 128 node columns (4 consecutive nodes per lane).  Strips overlap by one lane: lane 0 of
@@ -35,8 +35,8 @@ constexpr int S2_WARPS = 8;                       // warps (work units) per bloc
 constexpr int S2_NE = 4;                          // nodes per lane
 constexpr int S2_COLS = 32 * S2_NE;               // node columns a warp holds
 constexpr int S2_STRIDE = S2_COLS - S2_NE;        // distance of neighbouring strips
-constexpr int S2_DEPTH = 8;                       // ring slots per warp (DEPTH - 1 rows in flight); a power of two
-constexpr int S2_SLOT = 256;                      // floats per ring slot (node row, 4 nodes right of it, coefficient row); a power of two
+constexpr int S2_DEPTH0 = 8;                      // ring slots per warp (DEPTH - 1 rows in flight); a power of two
+constexpr int S2_SLOT0 = 256;                     // floats per ring slot (node row, 4 nodes right of it, coefficient row); a power of two
 
 typedef unsigned long long u64;
 
@@ -73,13 +73,18 @@ template <int N> __device__ __forceinline__ void s2_wait() { asm volatile("cp.as
 // Floats per element row in the coefficient table: (row a, row b) pairs for k = 0..M, padded to a multiple of 4.
 __host__ __device__ constexpr int s2_gs(int m) { return (2 * (m + 1) + 3) / 4 * 4; }
 
-template <int M, int BPS, bool KN>
+template <int M, int BPS, int MODE>
 __global__ void __launch_bounds__(S2_WARPS * 32, BPS)
 strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, const int nchunk, const int nstrip) {
     extern __shared__ __align__(16) float smem[];
     constexpr int NE = S2_NE;
     constexpr int GS = s2_gs(M);
-    static_assert(S2_COLS + 4 + GS <= S2_SLOT, "ring slot too small");
+    // MODE 0: KL at the Gauss points; 1 (KN): KL at the nodes, then Q1 interpolation; 2 (ND): stored nodal field
+    constexpr bool KN = (MODE == 1), ND = (MODE == 2);
+    // ring slot: node row of u, the 4 nodes right of it, then the coefficient row - or (ND) the same two pieces of nu
+    constexpr int S2_SLOT = ND ? 2 * S2_SLOT0 : S2_SLOT0, S2_DEPTH = ND ? S2_DEPTH0 / 2 : S2_DEPTH0;
+    constexpr int NUOFF = S2_COLS + 4;                  // ND: where the nu row starts inside a slot
+    static_assert(S2_COLS + 4 + GS <= S2_SLOT && 2 * (S2_COLS + 4) <= 2 * S2_SLOT0, "ring slot too small");
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     float* ring = smem + (size_t)warp * S2_DEPTH * S2_SLOT;
@@ -134,7 +139,8 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
     u64 cda[NE], cdb[NE];
     u64 cnp[NE / 2];                                    // KN: cos(pi x) at this lane's nodes (pairs) and at the node right of them
     float cnh = 0.f;
-    if constexpr (KN) {
+    if constexpr (ND) {
+    } else if constexpr (KN) {
         const float4 q = __ldg(reinterpret_cast<const float4*>(P.cn[0] + x0c));
         cnp[0] = s2_pack(q.x, q.y); cnp[1] = s2_pack(q.z, q.w);
         cnh = __ldg(P.cn[0] + x0c + NE);
@@ -151,7 +157,8 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
     // 16 bytes), the 4 nodes right of the strip (lane 31) and the coefficients of element row j (lanes 0 .. GS/4-1)
     int fetch = jbeg;                                   // next element row to fetch
     const float* usrc = ub + (size_t)(jbeg + 1) * nx;
-    const bool xcoef = (lane < GS / 4), xhalo = (lane == 31) && has_halo;
+    const bool xcoef = !ND && (lane < GS / 4), xhalo = (lane == 31) && has_halo;
+    const float* nsrc = ND ? P.nu + (size_t)b * P.nodes + x0c + (size_t)(jbeg + 1) * nx : nullptr;
     const int xp = (xcoef || xhalo) ? 1 : 0;            // this lane makes a second copy per row
     // coefficient rows: per element row (its two Gauss rows), or with KN per node row (the row that arrives with it)
     const float* polyb = rowpoly + (size_t)b * (KN ? ny : ny - 1) * GS;
@@ -162,9 +169,14 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         if (fetch <= jend) {                            // uniform
             s2_cp16(slot + NE * lane, usrc);
             s2_cp16_if(slot + xdst, xsrc, xp);
+            if constexpr (ND) {
+                s2_cp16(slot + NUOFF + NE * lane, nsrc);
+                s2_cp16_if(slot + NUOFF + S2_COLS, nsrc + NE, xp);
+            }
         }
         s2_commit();                                    // one group per step, possibly empty
         ++fetch; usrc += nx; xsrc += xstep;
+        if constexpr (ND) nsrc += nx;
     };
 #pragma unroll
     for (int d = 0; d < S2_DEPTH - 1; ++d) issue(ring + d * S2_SLOT);
@@ -204,7 +216,18 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         for (int i = M - 1; i >= 0; --i) { float gi; s2_unpack(gg[i], gi, dmy); gh = fmaf(gh, cnh, gi); }
         nn[NE] = s2_ex2(gh);
     };
-    float nlo[NE + 1], hnu[NE];                         // KN: nu on the node row below and its sums over x-neighbours
+    float nlo[NE + 1], hnu[NE];                         // KN, ND: nu on the node row below and its sums over x-neighbours
+    if constexpr (ND) {
+        const float* np = P.nu + (size_t)b * P.nodes + x0c + (size_t)jbeg * nx;
+        const float4 q = __ldg(reinterpret_cast<const float4*>(np));
+        nlo[0] = q.x; nlo[1] = q.y; nlo[2] = q.z; nlo[3] = q.w;
+        float halo = 0.f;
+        if (xhalo) halo = __ldg(np + NE);
+        const float rn = __shfl_down_sync(0xffffffffu, nlo[0], 1);
+        nlo[NE] = (lane == 31) ? halo : rn;
+#pragma unroll
+        for (int k = 0; k < NE; ++k) hnu[k] = nlo[k] + nlo[k + 1];
+    }
     if constexpr (KN) {
         u64 gg[GS / 2];
         const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(polyb + (size_t)jbeg * GS);
@@ -232,7 +255,7 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         }
         const float halo = slot[S2_COLS];
         u64 g2[GS / 2];
-        {
+        if constexpr (!ND) {
             const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(slot + S2_COLS + 4);
 #pragma unroll
             for (int k = 0; k < GS / 4; ++k) { const ulonglong2 t = gp[k]; g2[2 * k] = t.x; g2[2 * k + 1] = t.y; }
@@ -243,6 +266,13 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         }
         float ncur[NE + 1];
         if constexpr (KN) nu_row(g2, ncur);
+        if constexpr (ND) {
+            const float4 q = *reinterpret_cast<const float4*>(slot + NUOFF + NE * lane);
+            ncur[0] = q.x; ncur[1] = q.y; ncur[2] = q.z; ncur[3] = q.w;
+            const float nh = slot[NUOFF + S2_COLS];
+            const float rn = __shfl_down_sync(0xffffffffu, ncur[0], 1);
+            ncur[NE] = (lane == 31) ? (has_halo ? nh : 0.f) : rn;
+        }
         float hir = __shfl_down_sync(0xffffffffu, c[0], 1);
         if (lane == 31) hir = has_halo ? halo : 0.f;
 
@@ -259,7 +289,7 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             const float Dxa = fmaf(DN_GA, t, e0), Dxb = fmaf(DN_GB, t, e0);
             const float Dya = fmaf(DN_GA, t, s0), Dyb = fmaf(DN_GB, t, s0);
             float Na, Nb, Ma, Mb;
-            if constexpr (KN) {
+            if constexpr (KN || ND) {
                 // Q1 interpolation of the nodal values to the Gauss points, summed along each derivative's own axis
                 const float h0 = hnu[k], h1 = ncur[k] + ncur[k + 1];
                 hnu[k] = h1;
@@ -315,7 +345,7 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             if (owner) *reinterpret_cast<float4*>(rrow) = o;
         }
         rrow += nx;
-        if constexpr (KN) {
+        if constexpr (KN || ND) {
 #pragma unroll
             for (int k = 0; k <= NE; ++k) nlo[k] = ncur[k];
         }
@@ -392,20 +422,20 @@ GeoS geometry_s(const dn_problem& p) {
     return g;
 }
 
-template <int M, bool KN>
+template <int M, int MODE>
 cudaError_t launch_mk(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
-    const size_t smem = sizeof(float) * S2_WARPS * S2_DEPTH * S2_SLOT;
+    const size_t smem = sizeof(float) * S2_WARPS * S2_DEPTH0 * S2_SLOT0;
     const long long units = (long long)P.batch * g.nchunk * g.nstrip;
     const unsigned blocks = (unsigned)((units + S2_WARPS - 1) / S2_WARPS);
-    const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2, KN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    strip2d_kernel<M, 2, KN><<<blocks, S2_WARPS * 32, smem, s>>>(P, rowpoly, g.R, g.nchunk, g.nstrip);
+    strip2d_kernel<M, 2, MODE><<<blocks, S2_WARPS * 32, smem, s>>>(P, rowpoly, g.R, g.nchunk, g.nstrip);
     return cudaGetLastError();
 }
 
 template <int M>
 cudaError_t launch_m(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
-    return (P.nu_mode == DN_NU_KL_NODAL) ? launch_mk<M, true>(P, rowpoly, g, s) : launch_mk<M, false>(P, rowpoly, g, s);
+    return (P.nu_mode == DN_NU_KL_NODAL) ? launch_mk<M, 1>(P, rowpoly, g, s) : launch_mk<M, 0>(P, rowpoly, g, s);
 }
 
 }  // namespace
@@ -414,7 +444,7 @@ cudaError_t launch_m(const Params& P, const float* rowpoly, const GeoS& g, cudaS
 // row takes 3 strips of 128).  The tiled kernel is about 1.16 times slower per element in this mode: the strip
 // kernel takes over where its lanes are at most 15 % more than the row, and wherever the tiled kernel cannot run.
 bool strip2d_applicable(const dn_problem& p) {
-    if (!(p.grid.dim == 2 && (p.nu_mode == DN_NU_KL_GAUSS || p.nu_mode == DN_NU_KL_NODAL) && p.f == nullptr && p.grid.nx % 4 == 0 &&
+    if (!(p.grid.dim == 2 && p.f == nullptr && p.grid.nx % 4 == 0 &&
           p.grid.nx >= 2 * S2_COLS && p.grid.ny >= 16))
         return false;
     const long long lanes = (long long)((p.grid.nx - S2_COLS + S2_STRIDE - 1) / S2_STRIDE + 1) * S2_COLS;
@@ -432,6 +462,7 @@ Launch strip2d_geometry(const dn_problem& p) {
 }
 
 size_t strip2d_rowpoly_floats(const dn_problem& p) {
+    if (p.nu_mode == DN_NU_NODAL) return 0;                      // the stored field needs no table
     return (size_t)p.batch * p.grid.ny * s2_gs(p.kl_modes);      // ny - 1 element rows, or ny node rows (KL at the nodes)
 }
 
@@ -442,6 +473,7 @@ cudaError_t launch_strip2d(const Params& P, const float* rowpoly, cudaStream_t s
     p.grid.dim = 2; p.grid.nx = P.nx; p.grid.ny = P.ny; p.grid.nz = 1; p.batch = P.batch;
     p.nu_mode = P.nu_mode; p.kl_modes = P.m;
     const GeoS g = geometry_s(p);
+    if (P.nu_mode == DN_NU_NODAL) return launch_mk<1, 2>(P, rowpoly, g, s);
     switch (P.m) {
         case 1: return launch_m<1>(P, rowpoly, g, s);
         case 2: return launch_m<2>(P, rowpoly, g, s);

@@ -19,21 +19,22 @@ SIZES = [(1024, 40, 2, 4), (1028, 17, 3, 1), (1116, 33, 2, 6), (1120, 16, 2, 2),
          (2048, 24, 2, 8), (2052, 37, 1, 7), (4096, 19, 2, 6), (1024, 700, 10, 2)]
 
 
-KL_MODES = [B.DN_NU_KL_GAUSS, B.DN_NU_KL_NODAL]        # KL evaluated at the Gauss points / at the nodes, both inside the kernel
+KL_MODES = [B.DN_NU_KL_GAUSS, B.DN_NU_KL_NODAL, B.DN_NU_NODAL]   # KL at the Gauss points / at the nodes (in the kernel), stored nodal field
 
 
 @pytest.mark.parametrize("mode", KL_MODES)
 @pytest.mark.parametrize("nx,ny,batch,m", SIZES)
 def test_strip2d_parity(nx, ny, batch, m, mode):
     inp = inputs.random_inputs(2, nx, ny, 1, batch, m, seed=7 + nx + ny, f_const=0.6)
-    po, pg = make_problems(inp, mode)
+    nu = inputs.random_positive_field(inp.u.shape, 5) if mode == B.DN_NU_NODAL else None
+    po, pg = make_problems(inp, mode, nu=nu)
     assert B.dn_path_name(pg) == "strip2d"
     Jo, _, _, ro = oracle.energy_grad(po, inp.u)
     Jg, rg = run_gpu(pg, inp.u)
     check(Jg, rg, Jo, ro, f"strip2d {nx}x{ny} b{batch} m{m}")
     assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
     # the any-size kernels on the same problem: two independent CUDA paths agree with the oracle
-    _, pgen = make_problems(inp, mode, flags=B.DN_FORCE_GENERIC)
+    _, pgen = make_problems(inp, mode, nu=nu, flags=B.DN_FORCE_GENERIC)
     Jg2, rg2 = run_gpu(pgen, inp.u)
     check(Jg2, rg2, Jo, ro, "generic")
 
@@ -43,9 +44,10 @@ def test_strip2d_parity(nx, ny, batch, m, mode):
 def test_strip2d_options(nx, ny, mode):
     inp = inputs.random_inputs(2, nx, ny, 1, 3, 3, seed=42, f_const=-0.4)
     u = inputs.random_field(inp.u.shape, 8)           # boundary values NOT satisfied
+    nu = inputs.random_positive_field(inp.u.shape, 6) if mode == B.DN_NU_NODAL else None
     gJ = np.array([1.5, -2.0, 0.25], dtype=np.float32)
     for flags in (0, B.DN_NO_MASK, B.DN_IMPOSE_BC_ON_LOAD, B.DN_IMPOSE_BC_ON_LOAD | B.DN_NO_MASK):
-        po, pg = make_problems(inp, mode, flags=flags, bc=(0.8, -0.3))
+        po, pg = make_problems(inp, mode, nu=nu, flags=flags, bc=(0.8, -0.3))
         assert B.dn_path_name(pg) == "strip2d"
         Jo, _, _, ro = oracle.energy_grad(po, u, gJ=gJ.astype(np.float64))
         Jg, rg = run_gpu(pg, u, gJ=gJ)
@@ -53,7 +55,7 @@ def test_strip2d_options(nx, ny, mode):
         if not (flags & B.DN_NO_MASK):
             assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
     # energy-only call (tiled kernel) against the fused call (strip kernel); residual-only call gives the same residual
-    po, pg = make_problems(inp, mode)
+    po, pg = make_problems(inp, mode, nu=nu)
     ws = B.new_workspace(pg)
     J1 = torch.empty(3, device="cuda"); J2 = torch.empty(3, device="cuda"); r = torch.empty(pg.shape, device="cuda")
     B.dn_energy(pg, dev(u), J1, ws)
