@@ -38,12 +38,12 @@ FP32_PEAK_LANE_OPS = 148 * 128 * 1.965e9     # SMs x FP32 lanes x max SM clock: 
 # (FADD + FMUL + FFMA + 2 FFMA2).  Each entry names the kernel source it was taken from and the first 16
 # hex digits of its sha256: once that file changes the entry no longer applies and null is reported.
 NCU_CAPTURES = {
-    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 499963392, "fp32_ops_per_element": 57.7,
-                                          "src": "dn_strip2d.cu", "sha": "1fa15b0e386c409b"},
-    "strip2d:cfg2_2d_2048^2_b16_m6:klnodal": {"traffic": 499885056, "fp32_ops_per_element": 44.0,
-                                               "src": "dn_strip2d.cu", "sha": "1fa15b0e386c409b"},
-    "tiled2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 792350208, "fp32_ops_per_element": 35.5,
-                                             "src": "dn_tiled2d.cu", "sha": "83d5769163988ff7"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 500134912, "fp32_ops_per_element": 57.7,
+                                          "src": "dn_strip2d.cu", "sha": "b247dd0062e2187e"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:klnodal": {"traffic": 501000704, "fp32_ops_per_element": 44.0,
+                                               "src": "dn_strip2d.cu", "sha": "b247dd0062e2187e"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 789447680, "fp32_ops_per_element": 35.9,
+                                             "src": "dn_strip2d.cu", "sha": "b247dd0062e2187e"},
     "tiled3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 565575168, "fp32_ops_per_element": 155.8,
                                         "src": "dn_tiled3d.cu", "sha": "44f694b4e7cf5939"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
