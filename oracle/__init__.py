@@ -8,10 +8,9 @@ All arrays are numpy, C-ordered ``[B][nz][ny][nx]`` (x fastest).  Inputs that
 the GPU path also receives (``u``, ``nu``, ``kl_w``, ``f``) are float32 and are
 promoted to double inside the oracle; results are float64.
 
-Parity pins live in ``tests/test_oracle_pins.py``.  The KL-at-Gauss energy of a
-general field has no closed form and is pinned only through invariants
-(quadratic-in-t, finite differences, Euler identity, constant-exponent closed
-form): beyond those it is "parity unpinned".
+Parity pins live in ``tests/test_oracle_pins.py``; every function is pinned (the
+KL-at-Gauss mode by Gauss sums typed out point by point on Q1 fields whose
+gradient varies inside an element).
 """
 from __future__ import annotations
 

@@ -34,8 +34,9 @@
 // Pins (tests/test_oracle_pins.py): closed-form energies, textbook element
 // matrices, partition of unity, Euler identity, quadratic-in-t, finite
 // differences, 3-point-rule cross-check, dense direct solve.  The KL-at-Gauss
-// energy of a general field has no closed form; it is pinned through those
-// invariants and the closed forms for constant exponent only.
+// mode is pinned by Gauss sums typed out point by point: for u = 1 - x, and for
+// the Q1 fields u = 2x + xy and u = x + xyz, whose gradient differs at every Gauss
+// point of an element (energy, and the residual at one node).
 
 #include <cmath>
 #include <cstddef>

@@ -31,6 +31,12 @@ MUTATIONS = {
     "corner_index_swapped": ("const int ix = ex + (a & 1), iy = ey + ((a >> 1) & 1), iz = ez + ((a >> 2) & 1);\n        const long idx = node_index(g, ix, iy, iz);\n        uc[a]",
                              "const int ix = ex + ((a >> 1) & 1), iy = ey + (a & 1), iz = ez + ((a >> 2) & 1);\n        const long idx = node_index(g, ix, iy, iz);\n        uc[a]"),
     "mask_wrong_face": ("rb[node_index(g, g.nx - 1, iy, iz)] = 0.0;", "rb[node_index(g, g.nx - 2, iy, iz)] = 0.0;"),
+    "kl_gauss_abscissae_swapped_between_axes": (
+        "const double x = (ex + 0.5 * (1.0 + ref[0])) * g.h[0];\n                    const double y = (ey + 0.5 * (1.0 + ref[1])) * g.h[1];",
+        "const double x = (ex + 0.5 * (1.0 + ref[1])) * g.h[0];\n                    const double y = (ey + 0.5 * (1.0 + ref[0])) * g.h[1];"),
+    "kl_gauss_abscissae_shifted_cyclically_3d": (
+        "const double y = (ey + 0.5 * (1.0 + ref[1])) * g.h[1];\n                    const double z = (g.dim == 3) ? (ez + 0.5 * (1.0 + ref[2])) * g.h[2] : 0.0;",
+        "const double y = (ey + 0.5 * (1.0 + ref[g.dim == 3 ? 2 : 1])) * g.h[1];\n                    const double z = (g.dim == 3) ? (ez + 0.5 * (1.0 + ref[1])) * g.h[2] : 0.0;"),
     "nodal_nu_not_interpolated": ("nuq += N[a] * nuc[a];", "nuq += 0.125 * nuc[a] * (g.dim == 3 ? 1.0 : 2.0);"),
 }
 
@@ -124,6 +130,41 @@ def pins_hold(o) -> bool:
     p = Problem(dim=2, nx=nx, ny=ny, batch=1, nu_mode=NU_KL_GAUSS, kl_modes=2, kl_w=wk)
     lin = np.broadcast_to(1.0 - np.arange(nx) / (nx - 1), (1, ny, nx)).copy()
     if abs(o.energy_grad(p, lin)[0][0] - ref) > 1e-13:
+        return False
+    # typed-out Gauss sums for KL at Gauss points on Q1 fields whose gradient varies inside an element:
+    # u = 2x + xy on 3 x 4 nodes, grad u = (2 + y, x);  u = x + xyz on 2 x 3 x 2 nodes, grad u = (1 + yz, xz, xy)
+    nx, ny = 3, 4
+    hx, hy = 1 / 2, 1 / 3
+    X = np.arange(nx) * hx; Y = np.arange(ny) * hy
+    ref = 0.0
+    for ex in range(nx - 1):
+        for ey in range(ny - 1):
+            for sx in (-g, g):
+                for sy in (-g, g):
+                    xq, yq = (ex + 0.5 + 0.5 * sx) * hx, (ey + 0.5 + 0.5 * sy) * hy
+                    nuq = np.exp(sum(wd[i - 1, j - 1] * np.cos(i * np.pi * xq) * np.cos(j * np.pi * yq) / (1 + i * i + j * j)
+                                     for i in (1, 2) for j in (1, 2)))
+                    ref += 0.5 * (hx * hy / 4) * nuq * ((2 + yq) ** 2 + xq ** 2)
+    p = Problem(dim=2, nx=nx, ny=ny, batch=1, nu_mode=NU_KL_GAUSS, kl_modes=2, kl_w=wk)
+    if abs(o.energy_grad(p, (2 * X[None, :] + X[None, :] * Y[:, None])[None])[0][0] - ref) > 1e-12 * ref:
+        return False
+    w3 = rng.uniform(-1.7, 1.7, (1, 2, 2, 2)).astype(np.float32)
+    w3d = w3[0].astype(np.float64)
+    nx, ny, nz = 2, 3, 2
+    hx, hy, hz = 1.0, 0.5, 1.0
+    X = np.arange(nx) * hx; Y = np.arange(ny) * hy; Z = np.arange(nz) * hz
+    ref = 0.0
+    for ey in range(ny - 1):
+        for sx in (-g, g):
+            for sy in (-g, g):
+                for sz in (-g, g):
+                    xq, yq, zq = (0.5 + 0.5 * sx) * hx, (ey + 0.5 + 0.5 * sy) * hy, (0.5 + 0.5 * sz) * hz
+                    nuq = np.exp(sum(w3d[i - 1, j - 1, k - 1] * np.cos(i * np.pi * xq) * np.cos(j * np.pi * yq) * np.cos(k * np.pi * zq)
+                                     / (1 + i * i + j * j + k * k) for i in (1, 2) for j in (1, 2) for k in (1, 2)))
+                    ref += 0.5 * (hx * hy * hz / 8) * nuq * ((1 + yq * zq) ** 2 + (xq * zq) ** 2 + (xq * yq) ** 2)
+    p = Problem(dim=3, nx=nx, ny=ny, nz=nz, batch=1, nu_mode=NU_KL_GAUSS, kl_modes=2, kl_w=w3)
+    u3 = (X[None, None, :] + X[None, None, :] * Y[None, :, None] * Z[:, None, None])[None]
+    if abs(o.energy_grad(p, u3)[0][0] - ref) > 1e-12 * ref:
         return False
     return True
 

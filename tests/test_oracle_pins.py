@@ -388,6 +388,88 @@ def test_kl_gauss_points_written_out_on_one_and_two_elements():
     assert oracle.energy_grad(p, lin_profile(p.shape), want_r=False)[0][0] == pytest.approx(ref, rel=1e-14)
 
 
+def _kl_nu_point(wd, *xyz):
+    """The KL formula at one physical point, typed out (wd: float64 weights [m]^d)."""
+    m = wd.shape[0]
+    rng_ = range(1, m + 1)
+    if len(xyz) == 2:
+        x, y = xyz
+        return np.exp(sum(wd[i - 1, j - 1] * np.cos(i * np.pi * x) * np.cos(j * np.pi * y) / (1 + i * i + j * j)
+                          for i in rng_ for j in rng_))
+    x, y, z = xyz
+    return np.exp(sum(wd[i - 1, j - 1, k - 1] * np.cos(i * np.pi * x) * np.cos(j * np.pi * y) * np.cos(k * np.pi * z)
+                      / (1 + i * i + j * j + k * k) for i in rng_ for j in rng_ for k in rng_))
+
+
+def test_kl_gauss_energy_and_residual_of_fields_with_varying_gradient_written_out():
+    """Which Gauss point's nu multiplies which gradient.  u = 2x + xy (2D) and u = x + xyz (3D) are Q1
+    fields, so the interpolant is the field itself and grad u at a Gauss point is (2 + y, x) resp.
+    (1 + yz, xz, xy) exactly, different at every point of an element; the energy is then the typed-out sum
+    J = sum_e sum_q W 1/2 nu(x_q) |grad u(x_q)|^2 on non-square meshes with random weights.  The residual at
+    one interior node is typed out the same way from the hat function's gradient."""
+    g = 1.0 / np.sqrt(3.0)
+    # ---- 2D, 3 x 4 nodes
+    w = inputs.draw_weights(np.random.default_rng(21), 2, 2)[None]
+    wd = w[0].astype(np.float64)
+    nx, ny = 3, 4
+    hx, hy = 1.0 / (nx - 1), 1.0 / (ny - 1)
+    X = np.arange(nx) * hx; Y = np.arange(ny) * hy
+    u = (2 * X[None, :] + X[None, :] * Y[:, None])[None]
+    ref = 0.0
+    # residual at the interior node (1, 2): its hat function is (1 - |x - X1|/hx)(1 - |y - Y2|/hy)
+    ix, iy = 1, 2
+    rref = 0.0
+    for ex in range(nx - 1):
+        for ey in range(ny - 1):
+            for sx in (-g, g):
+                for sy in (-g, g):
+                    xq, yq = (ex + 0.5 + 0.5 * sx) * hx, (ey + 0.5 + 0.5 * sy) * hy
+                    nuq = _kl_nu_point(wd, xq, yq)
+                    gx, gy = 2.0 + yq, xq
+                    W = hx * hy / 4.0
+                    ref += W * 0.5 * nuq * (gx * gx + gy * gy)
+                    if abs(xq - X[ix]) < hx and abs(yq - Y[iy]) < hy:
+                        hxv, hyv = 1 - abs(xq - X[ix]) / hx, 1 - abs(yq - Y[iy]) / hy
+                        dhx, dhy = -np.sign(xq - X[ix]) / hx, -np.sign(yq - Y[iy]) / hy
+                        rref += W * nuq * (gx * dhx * hyv + gy * hxv * dhy)
+    p = Problem(dim=2, nx=nx, ny=ny, batch=1, nu_mode=NU_KL_GAUSS, kl_modes=2, kl_w=w, flags=NO_MASK)
+    J, Jd, Jl, r = oracle.energy_grad(p, u)
+    assert J[0] == pytest.approx(ref, rel=1e-13)
+    assert r[0, iy, ix] == pytest.approx(rref, rel=1e-12)
+    # ---- 3D, 2 x 3 x 2 nodes
+    w3 = inputs.draw_weights(np.random.default_rng(22), 3, 2)[None]
+    w3d = w3[0].astype(np.float64)
+    nx, ny, nz = 2, 3, 2
+    hx, hy, hz = 1.0 / (nx - 1), 1.0 / (ny - 1), 1.0 / (nz - 1)
+    X = np.arange(nx) * hx; Y = np.arange(ny) * hy; Z = np.arange(nz) * hz
+    u = (X[None, None, :] + X[None, None, :] * Y[None, :, None] * Z[:, None, None])[None]
+    ref = 0.0
+    ix, iy, iz = 1, 1, 0                                  # node on the x = 1 and z = 0 faces, interior in y
+    rref = 0.0
+    for ex in range(nx - 1):
+        for ey in range(ny - 1):
+            for ez in range(nz - 1):
+                for sx in (-g, g):
+                    for sy in (-g, g):
+                        for sz in (-g, g):
+                            xq, yq, zq = (ex + 0.5 + 0.5 * sx) * hx, (ey + 0.5 + 0.5 * sy) * hy, (ez + 0.5 + 0.5 * sz) * hz
+                            nuq = _kl_nu_point(w3d, xq, yq, zq)
+                            gr = (1.0 + yq * zq, xq * zq, xq * yq)
+                            W = hx * hy * hz / 8.0
+                            ref += W * 0.5 * nuq * (gr[0] ** 2 + gr[1] ** 2 + gr[2] ** 2)
+                            d = (xq - X[ix], yq - Y[iy], zq - Z[iz])
+                            hh = (hx, hy, hz)
+                            if all(abs(d[a]) < hh[a] for a in range(3)):
+                                v = [1 - abs(d[a]) / hh[a] for a in range(3)]
+                                dv = [-np.sign(d[a]) / hh[a] for a in range(3)]
+                                rref += W * nuq * (gr[0] * dv[0] * v[1] * v[2] + gr[1] * v[0] * dv[1] * v[2]
+                                                   + gr[2] * v[0] * v[1] * dv[2])
+    p = Problem(dim=3, nx=nx, ny=ny, nz=nz, batch=1, nu_mode=NU_KL_GAUSS, kl_modes=2, kl_w=w3, flags=NO_MASK)
+    J, Jd, Jl, r = oracle.energy_grad(p, u)
+    assert J[0] == pytest.approx(ref, rel=1e-13)
+    assert r[0, iz, iy, ix] == pytest.approx(rref, rel=1e-12)
+
+
 def test_kl_gauss_converges_to_nodal_mode_under_refinement():
     """Both modes discretise the same continuous energy: their difference is O(h^2)."""
     w = inputs.draw_weights(np.random.default_rng(4), 2, 2)[None]
