@@ -24,8 +24,10 @@
  *    those with ix == 0 or ix == nx-1.
  *  - Every pointer is a DEVICE pointer unless its name ends in _host; structs are read
  *    on the host.  The caller owns every buffer.  The library allocates no memory,
- *    keeps no state between calls and never synchronises (the *_host entry point
- *    excepted, which returns after its last copy has finished).
+ *    keeps no state between calls and never synchronises.  Two exceptions: the *_host entry
+ *    points return after their last copy has finished (also when they fail half-way), and
+ *    dn_energy_grad_static remembers, per device, the address of its built-in scratch array
+ *    (looked up on the first call on that device; it goes stale if the device is reset).
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
  *    enqueued on it in order; outputs are valid once that work has finished.
  *  - Return value: DN_OK or an error code; nothing is thrown, nothing aborts.  When
@@ -144,7 +146,9 @@ dn_status dn_energy_grad_traced(const dn_problem* problem, const float* u, const
  *  - Inputs, outputs and results are exactly those of dn_energy_grad.
  *  - A problem that needs more scratch than the array holds (large grids on the any-size kernels,
  *    very large batches) is refused with DN_ERR_WORKSPACE and nothing is enqueued; use
- *    dn_energy_grad with your own workspace for those.
+ *    dn_energy_grad with your own workspace for those.  A wide 2D grid whose per-row coefficient
+ *    table does not fit runs on another kernel family if that one's scratch fits, else it is refused
+ *    the same way (e.g. 4096 x 4096 nodes, batch 16, 6 KL modes).
  *  - The first call on each device looks up the array's device address (one runtime query, with
  *    that device current); make that first call before starting any stream capture.
  *  - All calls on a device share the one array and it keeps whatever the previous call left in it.

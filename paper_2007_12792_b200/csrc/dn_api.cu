@@ -111,9 +111,24 @@ static Params make_params(const dn_problem& p, const WsLayout& w, const float* u
     return P;
 }
 
-static dn_status run(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
-                     size_t ws_bytes, void* stream, void* ev_before = nullptr, void* ev_after = nullptr,
-                     bool tight = false) {
+// The KL tables of a problem, written into its workspace: scaled weights and cosines (the same for every kernel
+// family) and, where the chosen family is the strip kernel, its per-row polynomials.
+static cudaError_t tables_into(const dn_problem& p, const Params& P, const WsLayout& w, const Launch& l, void* ws,
+                               cudaStream_t s) {
+    char* base = static_cast<char*>(ws);
+    float* cg[3] = {reinterpret_cast<float*>(base + w.cg[0]), reinterpret_cast<float*>(base + w.cg[1]),
+                    reinterpret_cast<float*>(base + w.cg[2])};
+    float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
+                    reinterpret_cast<float*>(base + w.cn[2])};
+    return launch_tables(P, p.kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
+                         (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
+                         strip2d_rowpoly_stride(p.kl_modes), p.nu_mode == DN_NU_KL_NODAL);
+}
+
+// Everything that is decided before anything is enqueued: validation, the kernel family, the workspace layout and
+// whether it fits ws_bytes.
+static dn_status plan(const dn_problem* p, const float* u, const float* r, size_t ws_bytes, bool tight, Launch& l,
+                      WsLayout& w) {
     dn_status st = validate(p);
     if (st != DN_OK) return st;
     if (!u) return DN_ERR_NULL;
@@ -123,27 +138,42 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
         const char* b = reinterpret_cast<const char*>(r);
         if (a < b + bytes && b < a + bytes) return DN_ERR_ALIAS;
     }
-    Launch l = choose_launch(*p, u, r);
-    WsLayout w = make_layout(*p, l, tight);
-    if (tight && l.path == PATH_STRIP2D && ws_bytes < w.total) {       // its coefficient table does not fit: tiled kernel
-        l = tiled2d_geometry(*p);
+    l = choose_launch(*p, u, r);
+    w = make_layout(*p, l, tight);
+    if (tight && l.path == PATH_STRIP2D && ws_bytes < w.total) {
+        // the strip kernel's coefficient table does not fit: the tiled kernel where it can run (rows of at most
+        // 2048 nodes), else the any-size kernel; if that does not fit either the call is refused
+        if (tiled2d_applicable(*p)) {
+            l = tiled2d_geometry(*p);
+        } else {
+            l = Launch{};
+            l.path = PATH_GENERIC;
+            l.nblk = generic_blocks_per_sample(nodes_per_sample(p->grid));
+        }
         w = make_layout(*p, l, tight);
     }
+    return (ws_bytes < w.total) ? DN_ERR_WORKSPACE : DN_OK;
+}
+
+dn_status check_tight(const dn_problem* p, const float* u, const float* r, size_t ws_bytes) {
+    if (!r) return DN_ERR_NULL;
+    Launch l{};
+    WsLayout w{};
+    return plan(p, u, r, ws_bytes, true, l, w);
+}
+
+static dn_status run(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
+                     size_t ws_bytes, void* stream, void* ev_before = nullptr, void* ev_after = nullptr,
+                     bool tight = false) {
+    Launch l{};
+    WsLayout w{};
+    const dn_status st = plan(p, u, r, ws_bytes, tight, l, w);
+    if (st != DN_OK && st != DN_ERR_WORKSPACE) return st;
     if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign) != 0 || ws_bytes < w.total) return DN_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Params P = make_params(*p, w, u, gJ, r, ws);
     cudaError_t e = cudaSuccess;
-    if (p->nu_mode != DN_NU_NODAL) {
-        char* base = static_cast<char*>(ws);
-        float* cg[3] = {reinterpret_cast<float*>(base + w.cg[0]), reinterpret_cast<float*>(base + w.cg[1]),
-                        reinterpret_cast<float*>(base + w.cg[2])};
-        float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
-                        reinterpret_cast<float*>(base + w.cn[2])};
-        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
-                          (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
-                          strip2d_rowpoly_stride(p->kl_modes), p->nu_mode == DN_NU_KL_NODAL);
-        if (e != cudaSuccess) return DN_ERR_CUDA;
-    }
+    if (p->nu_mode != DN_NU_NODAL && tables_into(*p, P, w, l, ws, s) != cudaSuccess) return DN_ERR_CUDA;
     if (ev_before && cudaEventRecord(static_cast<cudaEvent_t>(ev_before), s) != cudaSuccess) return DN_ERR_CUDA;
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
     else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
@@ -168,17 +198,7 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
     if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign) != 0 || ws_bytes < w.total) return DN_ERR_WORKSPACE;
     Params P = make_params(*p, w, u, nullptr, r, ws);
     cudaError_t e = cudaSuccess;
-    if (build_tables && p->nu_mode != DN_NU_NODAL) {
-        char* base = static_cast<char*>(ws);
-        float* cg[3] = {reinterpret_cast<float*>(base + w.cg[0]), reinterpret_cast<float*>(base + w.cg[1]),
-                        reinterpret_cast<float*>(base + w.cg[2])};
-        float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
-                        reinterpret_cast<float*>(base + w.cn[2])};
-        e = launch_tables(P, p->kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
-                          (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
-                          strip2d_rowpoly_stride(p->kl_modes), p->nu_mode == DN_NU_KL_NODAL);
-        if (e != cudaSuccess) return DN_ERR_CUDA;
-    }
+    if (build_tables && p->nu_mode != DN_NU_NODAL && tables_into(*p, P, w, l, ws, s) != cudaSuccess) return DN_ERR_CUDA;
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
     else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
     else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
@@ -187,6 +207,17 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
     if (partials) *partials = P.partials;
     if (nblk) *nblk = w.nblk;
     return DN_OK;
+}
+
+dn_status build_tables(const dn_problem* p, const float* u, float* r, void* ws, size_t ws_bytes, cudaStream_t s) {
+    dn_status st = validate(p);
+    if (st != DN_OK) return st;
+    if (p->nu_mode == DN_NU_NODAL) return DN_OK;
+    const Launch l = choose_launch(*p, u, r);
+    const WsLayout w = make_layout(*p, l, false);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) % kAlign) != 0 || ws_bytes < w.total) return DN_ERR_WORKSPACE;
+    const Params P = make_params(*p, w, u, nullptr, r, ws);
+    return tables_into(*p, P, w, l, ws, s) == cudaSuccess ? DN_OK : DN_ERR_CUDA;
 }
 
 dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
@@ -257,9 +288,6 @@ dn_status dn_apply_bc(const dn_grid* g, int32_t batch, float b0, float b1, int32
                                                                                                             : DN_ERR_CUDA;
 }
 
-// The batch is cut into chunks of whole samples that flow through three stages on three streams:
-// host->device copy, kernels (on the caller's stream), device->host copy.  Chunk c+1 is copied in
-// and chunk c-1 copied out while chunk c computes, so both directions of the host link stay busy.
 dn_status dn_apply_bc_per_sample(const dn_grid* g, int32_t batch, const float* b0, const float* b1, float* field,
                                  void* stream) {
     if (!g || !field || !b0 || !b1) return DN_ERR_NULL;
@@ -270,6 +298,9 @@ dn_status dn_apply_bc_per_sample(const dn_grid* g, int32_t batch, const float* b
                ? DN_OK : DN_ERR_CUDA;
 }
 
+// The batch is cut into chunks of whole samples that flow through three stages on three streams:
+// host->device copy, kernels (on the caller's stream), device->host copy.  Chunk c+1 is copied in
+// and chunk c-1 copied out while chunk c computes, so both directions of the host link stay busy.
 dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const float* gJ_host, float* J_host,
                               float* r_host, void* staging, size_t staging_bytes, void* stream) {
     dn_status st = validate(p);
@@ -307,14 +338,20 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
     if ((size_t)csize * sample_bytes < min_chunk) csize = (int)((min_chunk + sample_bytes - 1) / sample_bytes);
     if (csize > p->batch) csize = p->batch;
     int nchunks = (p->batch + csize - 1) / csize;
-    {
+    {   // both chunk sizes that will occur (full chunks and the shorter last one) must fit the workspace
         dn_problem q = *p;
         q.batch = csize;
-        if (dn_workspace_bytes(&q) > ws_bytes) { csize = p->batch; nchunks = 1; }
+        bool fits = dn_workspace_bytes(&q) <= ws_bytes;
+        const int last = p->batch - (nchunks - 1) * csize;
+        if (fits && last != csize) { q.batch = last; fits = dn_workspace_bytes(&q) <= ws_bytes; }
+        if (!fits) { csize = p->batch; nchunks = 1; }
     }
     HostPipe pipe;
     if (!pipe.create(nchunks)) return DN_ERR_CUDA;
-#define DN_TRY(x) do { if ((x) != cudaSuccess) return DN_ERR_CUDA; } while (0)
+    // On any failure the copies and kernels already enqueued are waited for before the call returns (they read and
+    // write the caller's host buffers, and the streams are destroyed on return).
+    auto drain = [&]() { cudaStreamSynchronize(pipe.in); cudaStreamSynchronize(s); cudaStreamSynchronize(pipe.out); };
+#define DN_TRY(x) do { if ((x) != cudaSuccess) { drain(); return DN_ERR_CUDA; } } while (0)
     DN_TRY(cudaEventRecord(pipe.start, s));                       // the call is ordered after earlier work on `stream`
     DN_TRY(cudaStreamWaitEvent(pipe.in, pipe.start, 0));
     DN_TRY(cudaStreamWaitEvent(pipe.out, pipe.start, 0));
@@ -340,7 +377,7 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
         q.bc_x0_b = p->bc_x0_b ? d_b0 + b0 : nullptr;
         q.bc_x1_b = p->bc_x1_b ? d_b1 + b0 : nullptr;
         st = run(&q, d_u + o, gJ_host ? d_g + b0 : nullptr, J_host ? d_J + b0 : nullptr, d_r + o, ws, ws_bytes, s);
-        if (st != DN_OK) { cudaStreamSynchronize(pipe.in); cudaStreamSynchronize(s); cudaStreamSynchronize(pipe.out); return st; }
+        if (st != DN_OK) { drain(); return st; }
         DN_TRY(cudaEventRecord(pipe.computed[c], s));
         DN_TRY(cudaStreamWaitEvent(pipe.out, pipe.computed[c], 0));
         DN_TRY(cudaMemcpyAsync(r_host + o, d_r + o, sizeof(float) * n, cudaMemcpyDeviceToHost, pipe.out));

@@ -210,7 +210,10 @@ CgLayout cg_layout(const dn_problem& p) {
     L.dinv = off; off += field;
     L.partials = off; off += align_up(sizeof(double) * 2 * (size_t)p.batch * vec_blocks(nodes_of(p)));
     L.scalars = off; off += align_up(sizeof(CgScalars) * (size_t)p.batch);
-    L.op = off; off += dn_workspace_bytes(&p);
+    dn_problem pop = p;                      // the operator on directions has no nodal forcing and may take a kernel
+    pop.f = nullptr;                         // family with a larger workspace than the caller's problem
+    const size_t a = dn_workspace_bytes(&p), b = dn_workspace_bytes(&pop);
+    L.op = off; off += (a > b) ? a : b;
     L.total = off;
     return L;
 }
@@ -257,12 +260,16 @@ dn_status dn_cg_solve(const dn_problem* p, float* u, int32_t max_iters, float rt
     dn_status st = DN_OK;
     dn_problem p1 = *p;
     p1.flags &= ~(DN_NO_MASK | DN_IMPOSE_BC_ON_LOAD);
-    st = run_operator(&p1, u, r, op_ws, op_bytes, s, true, nullptr, nullptr);
-    if (st != DN_OK) return st;
-
-    // the operator on directions: zero forcing, zero boundary values, same diffusivity (tables stay valid)
+    // the operator on directions: zero forcing, zero boundary values, same diffusivity
     dn_problem p0 = p1;
     p0.f = nullptr; p0.f_const = 0.0f; p0.bc_x0 = 0.0f; p0.bc_x1 = 0.0f; p0.bc_x0_b = nullptr; p0.bc_x1_b = nullptr;
+    // The KL tables are built once, for the kernel family the direction operator takes (aligned scratch fields, no
+    // nodal forcing: the family that needs the most, e.g. the strip kernel's per-row polynomials); the caller's
+    // problem may run on another family (nodal forcing, unaligned u), which reads a subset of the same tables.
+    st = build_tables(&p0, pd, q, op_ws, op_bytes, s);
+    if (st != DN_OK) return st;
+    st = run_operator(&p1, u, r, op_ws, op_bytes, s, false, nullptr, nullptr);
+    if (st != DN_OK) return st;
     {   // Jacobi preconditioner: the diagonal of K, one colour class per application (p and q serve as scratch)
         const int nz = p->grid.dim == 3 ? p->grid.nz : 1;
         const unsigned rows = (unsigned)((long long)p->batch * nz * p->grid.ny);

@@ -69,6 +69,8 @@ struct Launch {           // tiled-path launch geometry chosen on the host
 Launch choose_launch(const dn_problem& p, const float* u, const float* r);
 WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight = false);
 // dn_energy_grad with the workspace sized for the chosen kernel family only (tight = true).
+// What run_tight would answer for a scratch area of ws_bytes, without enqueuing anything or touching the device.
+dn_status check_tight(const dn_problem* p, const float* u, const float* r, size_t ws_bytes);
 dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float* J, float* r, void* ws,
                     size_t ws_bytes, void* stream);
 // The fused kernel alone, for callers that apply the operator repeatedly: no energy finaliser; the KL tables are
@@ -76,6 +78,11 @@ dn_status run_tight(const dn_problem* p, const float* u, const float* gJ, float*
 // kernel left its per-block energy pairs (diffusion part, load part), [batch][*nblk][2] doubles.
 dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, size_t ws_bytes, cudaStream_t s,
                        bool build_tables, const double** partials, int* nblk);
+
+// The KL tables alone, laid out as the kernel family chosen for (p, u, r) reads them.  For callers of run_operator
+// that apply the operator to several problems sharing one diffusivity: build for the problem whose family needs
+// the most (the cosine tables and scaled weights are common to all families).
+dn_status build_tables(const dn_problem* p, const float* u, float* r, void* ws, size_t ws_bytes, cudaStream_t s);
 
 // rowpoly (optional, 2D): also writes the per-Gauss-row polynomials the strip kernel reads, rows of rowpoly_stride floats
 cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float* const cg[3], float* const cn[3],

@@ -621,7 +621,7 @@ Geo2 geometry(const dn_problem& p) {
     const int nx = p.grid.nx, ny = p.grid.ny;
     g.K = (nx > 128) ? 2 : 1;
     g.W = (nx + 128 * g.K - 1) / (128 * g.K);
-    g.WY = T2_MAX_WARPS / g.W;
+    g.WY = (g.W <= T2_MAX_WARPS) ? T2_MAX_WARPS / g.W : 1;    // rows wider than the kernel handles: never 0 (callers check tiled2d_applicable)
     g.full = (g.W * 128 * g.K == nx);
     const int m = (p.nu_mode != DN_NU_NODAL) ? p.kl_modes : 0;
     g.GS = m ? (2 * (m + 1) + 3) / 4 * 4 : 0;

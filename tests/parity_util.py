@@ -25,13 +25,41 @@ def make_problems(inp, nu_mode, nu=None, f=None, flags=0, f_const=None, bc=None)
     return po, pg
 
 
+GUARD = 4096          # sentinel bytes before and after every output buffer and the workspace
+_SENTINEL = 0xA5
+
+
+def guarded(nbytes, dtype=torch.uint8):
+    """(whole, view): a device byte buffer filled with a sentinel, and the nbytes in its middle (GUARD bytes of
+    sentinel on either side; GUARD is a multiple of 256, so the view keeps the allocation's alignment)."""
+    whole = torch.full((nbytes + 2 * GUARD,), _SENTINEL, dtype=torch.uint8, device="cuda")
+    return whole, whole[GUARD:GUARD + nbytes]
+
+
+def guards_intact(whole, nbytes):
+    """Nothing wrote outside the middle nbytes (the stand-in for a memory checker: a kernel that stores one
+    element before or after r, J or its workspace changes a sentinel byte)."""
+    return bool((whole[:GUARD] == _SENTINEL).all()) and bool((whole[GUARD + nbytes:] == _SENTINEL).all())
+
+
 def run_gpu(pg, u, gJ=None, want_J=True):
     ud = dev(u)
-    r = torch.full(pg.shape, float("nan"), dtype=torch.float32, device="cuda")
-    J = torch.full((pg.batch,), float("nan"), dtype=torch.float32, device="cuda") if want_J else None
-    ws = B.new_workspace(pg)
-    B.dn_energy_grad(pg, ud, dev(gJ), J, r, ws)
+    n = int(np.prod(pg.shape))
+    r_whole, r_bytes = guarded(4 * n)
+    r = r_bytes.view(torch.float32).view(pg.shape)
+    r.fill_(float("nan"))
+    J_whole, J_bytes = guarded(4 * pg.batch)
+    J = J_bytes.view(torch.float32)
+    J.fill_(float("nan"))
+    ws_n = max(B.dn_workspace_bytes(pg), 256)
+    ws_whole, ws = guarded(ws_n)
+    B.dn_energy_grad(pg, ud, dev(gJ), J if want_J else None, r, ws)
     torch.cuda.synchronize()
+    assert guards_intact(r_whole, 4 * n), "bytes outside r were written"
+    assert guards_intact(J_whole, 4 * pg.batch), "bytes outside J were written"
+    assert guards_intact(ws_whole, ws_n), "bytes outside the workspace were written"
+    if not want_J:
+        assert bool(torch.isnan(J).all()), "J was written although it was not asked for"
     return (J.cpu().numpy().astype(np.float64) if want_J else None), r.cpu().numpy().astype(np.float64)
 
 

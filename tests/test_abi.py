@@ -89,6 +89,36 @@ def test_host_side_validation(L):
     assert L.dn_path_name(C.byref(prob(nx=7))) == b"generic"
 
 
+def test_entry_point_without_workspace_refuses_on_the_host(L):
+    """dn_energy_grad_static decides on the host, before touching the device, whether its built-in 1 MiB of scratch
+    is enough: wide 2D grids whose strip-kernel table does not fit and that no other kernel family can serve
+    within the limit are refused with DN_ERR_WORKSPACE (they used to divide by zero in the tiled geometry)."""
+    from paper_2007_12792_b200 import binding as B
+    fake = 0x100000
+
+    def prob(nx, ny, batch, m, mode=B.DN_NU_KL_GAUSS, dim=2, nz=1):
+        p = B.DnProblem()
+        p.grid = B.DnGrid(dim, nx, ny, nz)
+        p.batch = batch; p.nu_mode = mode; p.kl_modes = m; p.kl_w = fake
+        p.nu = fake if mode == B.DN_NU_NODAL else None
+        return p
+
+    def st(p, u=fake, r=fake << 12):
+        return L.dn_energy_grad_static(C.byref(p), u, None, None, r, None)
+
+    assert st(prob(4096, 4096, 16, 6)) == B.DN_ERR_WORKSPACE
+    assert st(prob(4096, 4096, 2, 6)) == B.DN_ERR_WORKSPACE
+    assert st(prob(4096, 4096, 2, 6, mode=B.DN_NU_KL_NODAL)) == B.DN_ERR_WORKSPACE
+    assert st(prob(8192, 64, 1, 8)) in (B.DN_ERR_WORKSPACE, B.DN_ERR_CUDA)   # fits or not (no device here), no crash
+    assert st(prob(256, 256, 4, 3, dim=3, nz=256)) == B.DN_ERR_WORKSPACE   # 3D tile seams beyond 1 MiB
+    assert st(prob(4001, 4001, 16, 2)) == B.DN_ERR_WORKSPACE               # any-size kernel: too many partials
+    # validation comes first here too
+    assert st(prob(4096, 4096, 16, 0)) == B.DN_ERR_MODE
+    assert st(prob(64, 64, 2, 2), u=None) == B.DN_ERR_NULL
+    assert st(prob(64, 64, 2, 2), r=fake + 64) == B.DN_ERR_ALIAS
+    assert L.dn_energy_grad_static(C.byref(prob(64, 64, 2, 2)), fake, None, None, None, None) == B.DN_ERR_NULL
+
+
 def test_binding_rejects_host_tensors_and_missing_library(monkeypatch):
     import torch
     from paper_2007_12792_b200 import binding as B

@@ -86,6 +86,39 @@ def test_cg_with_nodal_forcing_and_zero_iterations():
     assert np.array_equal(u0.cpu().numpy(), ref) and np.all(its == 0) and np.all(relres == 1.0)
 
 
+def _oracle_residual(inp, omode, nu, f, f_const, bc, u):
+    po = oracle.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=omode, nu=nu,
+                        kl_modes=inp.kl_modes, kl_w=inp.kl_w, f_const=f_const, f=f, bc_x0=bc[0], bc_x1=bc[1])
+    return oracle.energy_grad(po, u)
+
+
+@pytest.mark.parametrize("nx,ny,mode,with_f", [(1024, 24, "kl", False), (2052, 17, "kl", False), (1024, 24, "klnodal", False),
+                                                (1024, 24, "nodal", False), (1024, 24, "kl", True)])
+def test_cg_on_wide_rows_where_the_strip_kernel_is_the_operator(nx, ny, mode, with_f):
+    """Grids too large for a dense direct solve: the result is checked through the oracle's own residual and energy.
+    CG started from a random field (|r0| = O(1) per node) must bring the oracle's residual of the returned field
+    below 3e-5 |r0| -- it would not if the operator the iteration applies were not the oracle's K(nu) -- and the
+    energy the library reports for that field must be the oracle's.  With nodal forcing the caller's problem runs on
+    another kernel family than the direction operator, which still reads the tables built for it."""
+    inp = inputs.random_inputs(2, nx, ny, 1, 2, 3, seed=50 + ny, sigma=1.0)
+    f = inputs.random_field((2, ny, nx), seed=12).astype(np.float32) if with_f else None
+    bc = (0.75, -0.25)
+    p, u, relres, its, (omode, nu) = solve(inp, mode, f=f, f_const=1.5, bc=bc, iters=30000, rtol=1e-5)
+    pd = B.Problem(dim=2, nx=nx, ny=ny, nz=1, batch=2, nu_mode=p.nu_mode, nu=p.nu, kl_modes=3, kl_w=p.kl_w)
+    assert B.dn_path_name(pd) == "strip2d"
+    assert np.all(relres <= 1e-5) and np.all(its < 30000), (relres, its)
+    u0 = inp.u.copy(); u0[..., 0] = bc[0]; u0[..., -1] = bc[1]
+    _, _, _, r0 = _oracle_residual(inp, omode, nu, f, 1.5, bc, u0)
+    ug = u.cpu().numpy()
+    Jo, _, _, ro = _oracle_residual(inp, omode, nu, f, 1.5, bc, ug)
+    for b in range(2):
+        assert np.linalg.norm(ro[b]) <= 3e-5 * np.linalg.norm(r0[b]), (np.linalg.norm(ro[b]), np.linalg.norm(r0[b]))
+    assert np.all(ug[..., 0] == np.float32(bc[0])) and np.all(ug[..., -1] == np.float32(bc[1]))
+    J = torch.empty(2, device="cuda"); r = torch.empty_like(u)
+    B.dn_energy_grad(p, u, None, J, r, B.new_workspace(p))
+    assert np.all(np.abs(J.cpu().numpy() - Jo) <= J_RTOL * np.abs(Jo))
+
+
 def test_cg_is_deterministic_and_freezes_converged_samples():
     inp = inputs.random_inputs(2, 32, 32, 1, 3, 2, seed=3, f_const=1.0)
     _, ua, ra, ia, _ = solve(inp, "kl", iters=300, rtol=1e-4)

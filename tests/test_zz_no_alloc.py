@@ -33,6 +33,9 @@ def test_static_scratch_matches_workspace_entry_point_on_consecutive_calls():
              # wide 2D rows: the strip kernel when its coefficient table fits the array, else the tiled kernel
              (inputs.random_inputs(2, 1024, 64, 1, 2, 4, seed=9, f_const=0.5), B.DN_NU_KL_GAUSS),
              (inputs.random_inputs(2, 1024, 4000, 1, 6, 6, seed=10), B.DN_NU_KL_GAUSS),
+             # rows wider than the tiled kernel takes (2048): the strip kernel, its table within the array
+             (inputs.random_inputs(2, 2052, 40, 1, 2, 5, seed=11, f_const=0.25), B.DN_NU_KL_GAUSS),
+             (inputs.random_inputs(2, 2052, 40, 1, 2, 5, seed=11, f_const=0.25), B.DN_NU_KL_NODAL),
              (inputs.make_inputs(0), B.DN_NU_KL_GAUSS)]
     for inp, mode in cases:
         nu = None
@@ -54,3 +57,13 @@ def test_static_scratch_refuses_problems_beyond_its_size():
         B.dn_energy_grad_static(p, u, None, None, r)
     assert e.value.status == B.DN_ERR_WORKSPACE
     assert float(r.abs().max()) == 0.0                                   # nothing was enqueued
+    # a wide 2D grid whose strip-kernel table exceeds the array and that no other kernel family serves within 1 MiB
+    inp = inputs.random_inputs(2, 4096, 1200, 1, 2, 6, seed=2)
+    w = torch.from_numpy(inp.kl_w).cuda(); u = torch.from_numpy(inp.u).cuda()
+    p = B.Problem(dim=2, nx=4096, ny=1200, batch=2, kl_modes=6, kl_w=w)
+    r = torch.zeros_like(u)
+    with pytest.raises(B.DnError) as e:
+        B.dn_energy_grad_static(p, u, None, None, r)
+    assert e.value.status == B.DN_ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert float(r.abs().max()) == 0.0
