@@ -58,9 +58,9 @@ def test_static_scratch_refuses_problems_beyond_its_size():
     assert e.value.status == B.DN_ERR_WORKSPACE
     assert float(r.abs().max()) == 0.0                                   # nothing was enqueued
     # a wide 2D grid whose strip-kernel table exceeds the array and that no other kernel family serves within 1 MiB
-    inp = inputs.random_inputs(2, 4096, 1200, 1, 2, 6, seed=2)
+    inp = inputs.random_inputs(2, 4096, 4096, 1, 2, 6, seed=2)
     w = torch.from_numpy(inp.kl_w).cuda(); u = torch.from_numpy(inp.u).cuda()
-    p = B.Problem(dim=2, nx=4096, ny=1200, batch=2, kl_modes=6, kl_w=w)
+    p = B.Problem(dim=2, nx=4096, ny=4096, batch=2, kl_modes=6, kl_w=w)
     r = torch.zeros_like(u)
     with pytest.raises(B.DnError) as e:
         B.dn_energy_grad_static(p, u, None, None, r)
