@@ -42,6 +42,7 @@ Launch choose_launch(const dn_problem& p, const float* u, const float* r) {
     const bool vec_ok = aligned16(u) && aligned16(r) && (p.nu_mode != DN_NU_NODAL || aligned16(p.nu));
     if (!(p.flags & DN_FORCE_GENERIC) && vec_ok && p.f == nullptr) {
         if (r && strip2d_applicable(p)) return strip2d_geometry(p);
+        if (r && strip3d_applicable(p)) return strip3d_geometry(p);
         if (tiled2d_applicable(p)) return tiled2d_geometry(p);
         if (tiled3d_applicable(p)) return tiled3d_geometry(p);
     }
@@ -58,6 +59,7 @@ static int max_nblk(const dn_problem& p) {
     if (tiled2d_applicable(p)) { int t = tiled2d_geometry(p).nblk; if (t > n) n = t; }
     if (strip2d_applicable(p)) { int t = strip2d_geometry(p).nblk; if (t > n) n = t; }
     if (tiled3d_applicable(p)) { int t = tiled3d_geometry(p).nblk; if (t > n) n = t; }
+    if (strip3d_applicable(p)) { int t = strip3d_geometry(p).nblk; if (t > n) n = t; }
     return n;
 }
 
@@ -84,9 +86,17 @@ WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
         off += align_up(sizeof(float) * (size_t)m * w.nstride[a] + 16);
     }
     w.seam = off;
-    if ((tight ? l.path == PATH_TILED3D : tiled3d_applicable(p))) off += align_up(sizeof(float) * tiled3d_seam_floats(p) + 16);
+    {   // tile seams of the 3D kernel families: the family in use (tight), or the larger of the two that may be chosen
+        size_t fl = 0;
+        if (tight ? l.path == PATH_TILED3D : tiled3d_applicable(p)) fl = tiled3d_seam_floats(p);
+        if (tight ? l.path == PATH_STRIP3D : strip3d_applicable(p)) { const size_t t = strip3d_seam_floats(p); if (t > fl) fl = t; }
+        if (tight ? (l.path == PATH_TILED3D || l.path == PATH_STRIP3D) : (tiled3d_applicable(p) || strip3d_applicable(p)))
+            off += align_up(sizeof(float) * fl + 16);
+    }
     w.rowpoly = off;
     if ((tight ? l.path == PATH_STRIP2D : strip2d_applicable(p))) off += align_up(sizeof(float) * strip2d_rowpoly_floats(p) + 16);
+    w.linepoly = off;
+    if ((tight ? l.path == PATH_STRIP3D : strip3d_applicable(p))) off += align_up(sizeof(float) * strip3d_linepoly_floats(p) + 16);
     w.total = off;
     return w;
 }
@@ -120,9 +130,11 @@ static cudaError_t tables_into(const dn_problem& p, const Params& P, const WsLay
                     reinterpret_cast<float*>(base + w.cg[2])};
     float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
                     reinterpret_cast<float*>(base + w.cn[2])};
-    return launch_tables(P, p.kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
-                         (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
-                         strip2d_rowpoly_stride(p.kl_modes), p.nu_mode == DN_NU_KL_NODAL);
+    const cudaError_t e = launch_tables(P, p.kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
+                                        (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
+                                        strip2d_rowpoly_stride(p.kl_modes), p.nu_mode == DN_NU_KL_NODAL);
+    if (e != cudaSuccess || l.path != PATH_STRIP3D) return e;
+    return launch_linepoly3d(P, reinterpret_cast<float*>(base + w.linepoly), s);
 }
 
 // Everything that is decided before anything is enqueued: validation, the kernel family, the workspace layout and
@@ -178,6 +190,7 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
     else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
     else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
+    else if (l.path == PATH_STRIP3D) e = launch_strip3d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.linepoly), s);
     else e = launch_generic(P, s);
     if (e != cudaSuccess) return DN_ERR_CUDA;
     if (ev_after && cudaEventRecord(static_cast<cudaEvent_t>(ev_after), s) != cudaSuccess) return DN_ERR_CUDA;
@@ -202,6 +215,7 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
     else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
     else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
+    else if (l.path == PATH_STRIP3D) e = launch_strip3d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.linepoly), s);
     else e = launch_generic(P, s);
     if (e != cudaSuccess) return DN_ERR_CUDA;
     if (partials) *partials = P.partials;
@@ -392,7 +406,10 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
 
 int32_t dn_launches_per_call(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
-    const bool t3 = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
+    const bool fast = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr;
+    if (fast && strip3d_applicable(*p))                 // tables, line polynomials, fused kernel, seam fix-up, finaliser
+        return 4 + (strip3d_seam_floats(*p) > 0 ? 1 : 0);
+    const bool t3 = fast && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
     return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
 }
 
@@ -401,6 +418,7 @@ const char* dn_path_name(const dn_problem* p) {
     if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr) {
         if (strip2d_applicable(*p)) return "strip2d";      // the fused call; the energy-only call of such a problem runs tiled2d
         if (tiled2d_applicable(*p)) return "tiled2d";
+        if (strip3d_applicable(*p)) return "strip3d";      // the fused call; the energy-only call runs tiled3d
         if (tiled3d_applicable(*p)) return "tiled3d";
     }
     return "generic";

@@ -17,7 +17,7 @@ constexpr int kAlign = 256;
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
-enum Path { PATH_GENERIC = 0, PATH_TILED2D = 1, PATH_TILED3D = 2, PATH_STRIP2D = 3 };
+enum Path { PATH_GENERIC = 0, PATH_TILED2D = 1, PATH_TILED3D = 2, PATH_STRIP2D = 3, PATH_STRIP3D = 4 };
 
 // Where things live inside the caller's workspace (byte offsets, all 256-B aligned).
 struct WsLayout {
@@ -29,6 +29,7 @@ struct WsLayout {
     size_t cn[3];         // float  [m][nstride[a]] cos(i pi x) at the nodes of axis a
     int nstride[3];
     size_t rowpoly;       // float  [B][ny-1][GS] polynomial of the KL exponent along every Gauss row (strip 2D kernel)
+    size_t linepoly;      // float  [B][nz-1][ny-1][2 GS] the same along the four Gauss lines of every element row (strip 3D kernel)
     int nblk;             // energy partials per sample
     size_t total;
 };
@@ -107,6 +108,15 @@ int strip2d_rowpoly_stride(int kl_modes);          // floats per element row of 
 Launch tiled2d_geometry(const dn_problem& p);
 Launch tiled3d_geometry(const dn_problem& p);
 size_t tiled3d_seam_floats(const dn_problem& p);   // scratch floats the tiled 3D kernel needs for its tile seams
+// adds seam[b][s][plane][x] to node row (s + 1) * rows_per_tile of r, for every sample, seam and plane
+cudaError_t launch_seam_fixup(float* r, const float* seam, int nx, int ny, int nz, int rows_per_tile, int nseam, int batch,
+                              cudaStream_t s);
+bool strip3d_applicable(const dn_problem& p);      // fused energy+residual, KL at the Gauss points, 3D rows of at most 256 nodes
+Launch strip3d_geometry(const dn_problem& p);
+size_t strip3d_seam_floats(const dn_problem& p);
+size_t strip3d_linepoly_floats(const dn_problem& p);
+cudaError_t launch_linepoly3d(const Params& P, float* linepoly, cudaStream_t s);   // after launch_tables (reads ckl, cg)
+cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t s);
 
 // Streams and events of one *_host call (created and destroyed inside the call).
 struct HostPipe {

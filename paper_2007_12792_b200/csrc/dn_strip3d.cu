@@ -1,0 +1,622 @@
+// Strip kernel for 3D grids whose rows fit one warp (nx <= 256): fused element quadrature, energy reduction,
+// node gather, mask and store on hexahedra, without any barrier between warps.
+//
+// Layout of the work.  A work unit is one sample, one tile of Ry element rows (y) across the whole x extent, one
+// chunk of Z element planes (z).  A unit belongs to LW = 8, 16 or 32 lanes of one warp (a lane owns NX = 4 or 8
+// consecutive nodes of a row, so LW * NX >= nx); a warp with LW < 32 carries 32 / LW units that have nothing to do
+// with one another.  No warp ever waits for another warp: there is no block-wide barrier and no exchange between
+// warps through shared memory.
+//
+// A unit marches over its element planes from bottom to top, and inside a plane over its element rows.  The node
+// rows it needs stream through a ring of rows in shared memory that belongs to the unit alone: row (plane k, row j)
+// of the tile is entry k * T + j of a linear sequence (T node rows per plane), entry n lives in slot n mod C, and
+// the ring always holds the two planes being worked on plus D rows in flight (cp.async, one group per row; every
+// lane copies the 16-byte pieces of its own nodes, a few lanes also copy the coefficients described below).  Every
+// node is read from global memory once per unit.
+//
+// Element (x, j, k) is computed once, by the lane that owns node x.  Of its 8 corner contributions those to column
+// x + 1 pass to the next element of the lane (to the next lane by shuffle), those to row j + 1 are kept until the
+// next row of the same plane, and those to plane k + 1 are parked in the output array itself: the lane stores the
+// partial sums of node row (j, k + 1) into r, and one plane later reads them back, adds what element plane k + 1
+// contributes, and stores the finished value (same thread, same address: program order makes the read see the
+// write; the lines stay in L2 in between).  So the registers hold one row of pending values, not a plane.
+//
+// Tiles do not overlap in y: the top element row of a tile leaves what it contributes to the first node row of
+// the next tile in a scratch array (seam, [B][ntile-1][nz][nx]), parked there between planes in the same way, and
+// the small fix-up kernel of the tiled 3D path adds those rows to r afterwards in a fixed order.  Chunks overlap by
+// one element plane in z: a chunk recomputes the last element plane of the chunk below for the sake of its
+// contributions to the chunk's first node plane (1 / Z more work).  No atomics; every sum has a fixed order.
+//
+// Arithmetic of one element: hierarchical coordinates of the trilinear field (edge differences e, s, w at the low
+// corner, second differences txy, txz, tyz, third difference txyz), derivatives at the 4 Gauss lines of each
+// direction, sums of nu along each derivative's own axis, the adjoint of the interpolation and the chain rule to
+// the 8 corners -- the formulas of the tiled 3D kernel.  The diffusion energy is taken from the residual by
+// Euler's identity for quadratic forms: 1/2 sum over (node, contribution) pairs of u_node times contribution, each
+// pair counted by the unit that computes it.
+//
+// KL diffusivity at the Gauss points: along a Gauss line (y_q, z_s fixed) the exponent is a polynomial of degree m
+// in c = cos(pi x).  A table kernel prepares the coefficients of all four lines of every element row of every
+// element plane once per call in double ([B][nz-1][ny-1][2][GS] floats: Gauss row q, then coefficient i and Gauss
+// plane s interleaved for packed two-wide FMAs); they travel through the ring with the node row that completes
+// the element row.
+#include "dn_internal.cuh"
+
+namespace dn {
+
+namespace {
+
+constexpr int S3_WARPS = 4;                       // warps per block (each warp is on its own)
+constexpr int S3_D = 3;                           // rows in flight beyond the two planes in use
+
+typedef unsigned long long u64;
+
+__device__ __forceinline__ float s3_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void s3_unpack(u64 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 s3_pack(float lo, float hi) {
+    u64 v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ u64 s3_fma2(u64 a, u64 b, u64 c) {
+    u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ void s3_cp16(float* smem_dst, const float* gsrc) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void s3_cp16_if(float* smem_dst, const float* gsrc, int pred) {    // predicated, no branch
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.s32 p, %2, 0;\n\t@p cp.async.cg.shared.global [%0], [%1], 16;\n\t}"
+                 ::"r"(d), "l"(gsrc), "r"(pred) : "memory");
+}
+__device__ __forceinline__ void s3_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void s3_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Floats per Gauss row (q fixed) of an element row in the coefficient table: (plane s = a, s = b) pairs for
+// i = 0..M, padded to a multiple of 4.
+__host__ __device__ constexpr int s3_gs(int m) { return (2 * (m + 1) + 3) / 4 * 4; }
+
+struct S3Geo {
+    int Ry, Z;            // element rows per tile, element planes per chunk
+    int ntile, nchunk;
+    int LW, lwsh;         // lanes per unit and log2 of it
+    int C, RS;            // ring slots (rows) per unit, floats per slot
+    long long units;
+};
+
+// nu at the 8 Gauss points of one element, index [p][q][s] -> n[4 p + 2 q + s]: four packed Horner chains
+// (column p, row q), each over the planes s = a, b.
+template <int M>
+__device__ __forceinline__ void s3_nu_gauss(const u64 (&ga)[s3_gs(M) / 2], const u64 (&gb)[s3_gs(M) / 2], const u64 ca2,
+                                            const u64 cb2, float (&n)[8]) {
+    u64 h_aa = ga[M], h_ab = gb[M], h_ba = ga[M], h_bb = gb[M];          // h_{p q}
+#pragma unroll
+    for (int i = M - 1; i >= 0; --i) {
+        h_aa = s3_fma2(h_aa, ca2, ga[i]); h_ab = s3_fma2(h_ab, ca2, gb[i]);
+        h_ba = s3_fma2(h_ba, cb2, ga[i]); h_bb = s3_fma2(h_bb, cb2, gb[i]);
+    }
+    float x[8];
+    s3_unpack(h_aa, x[0], x[1]); s3_unpack(h_ab, x[2], x[3]);
+    s3_unpack(h_ba, x[4], x[5]); s3_unpack(h_bb, x[6], x[7]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) n[i] = s3_ex2(x[i]);
+}
+
+// The element: from the 8 diffusivities n[4p + 2q + s] and the 7 hierarchical coordinates of u to the 8 corner
+// contributions r[i + 2j + 4k] (i, j, k the x, y, z bits of the corner), all in units of kap = hx hy hz / (8 h^2)
+// on isotropic cells (iso), else scaled by kx, ky, kz here.
+__device__ __forceinline__ void s3_element(const float (&n)[8], const float e0, const float s0, const float w0,
+                                           const float txy, const float txz, const float tyz, const float txyz,
+                                           const bool iso, const float kx, const float ky, const float kz,
+                                           float (&r)[8]) {
+    const float a = DN_GA, bq = DN_GB;
+    float Nx_aa = n[0] + n[4], Nx_ab = n[1] + n[5], Nx_ba = n[2] + n[6], Nx_bb = n[3] + n[7];   // (q, s)
+    float Ny_aa = n[0] + n[2], Ny_ab = n[1] + n[3], Ny_ba = n[4] + n[6], Ny_bb = n[5] + n[7];   // (p, s)
+    float Nz_aa = n[0] + n[1], Nz_ab = n[2] + n[3], Nz_ba = n[4] + n[5], Nz_bb = n[6] + n[7];   // (p, q)
+    if (!iso) {
+        Nx_aa *= kx; Nx_ab *= kx; Nx_ba *= kx; Nx_bb *= kx;
+        Ny_aa *= ky; Ny_ab *= ky; Ny_ba *= ky; Ny_bb *= ky;
+        Nz_aa *= kz; Nz_ab *= kz; Nz_ba *= kz; Nz_bb *= kz;
+    }
+    // derivatives at the Gauss lines: d/dx at (eta q, zeta s) = (e + q txy) + s (txz + q txyz), and cyclically
+    const float Axa = fmaf(a, txy, e0), Axb = fmaf(bq, txy, e0);
+    const float Bxa = fmaf(a, txyz, txz), Bxb = fmaf(bq, txyz, txz);
+    const float Dx_aa = fmaf(a, Bxa, Axa), Dx_ab = fmaf(bq, Bxa, Axa), Dx_ba = fmaf(a, Bxb, Axb), Dx_bb = fmaf(bq, Bxb, Axb);
+    const float Aya = fmaf(a, txy, s0), Ayb = fmaf(bq, txy, s0);
+    const float Bya = fmaf(a, txyz, tyz), Byb = fmaf(bq, txyz, tyz);
+    const float Dy_aa = fmaf(a, Bya, Aya), Dy_ab = fmaf(bq, Bya, Aya), Dy_ba = fmaf(a, Byb, Ayb), Dy_bb = fmaf(bq, Byb, Ayb);
+    const float Aza = fmaf(a, txz, w0), Azb = fmaf(bq, txz, w0);
+    const float Dz_aa = fmaf(a, Bya, Aza), Dz_ab = fmaf(bq, Bya, Aza), Dz_ba = fmaf(a, Byb, Azb), Dz_bb = fmaf(bq, Byb, Azb);
+    const float Gx_aa = Nx_aa * Dx_aa, Gx_ab = Nx_ab * Dx_ab, Gx_ba = Nx_ba * Dx_ba, Gx_bb = Nx_bb * Dx_bb;
+    const float Gy_aa = Ny_aa * Dy_aa, Gy_ab = Ny_ab * Dy_ab, Gy_ba = Ny_ba * Dy_ba, Gy_bb = Ny_bb * Dy_bb;
+    const float Gz_aa = Nz_aa * Dz_aa, Gz_ab = Nz_ab * Dz_ab, Gz_ba = Nz_ba * Dz_ba, Gz_bb = Nz_bb * Dz_bb;
+    // adjoint of the three interpolations: partial derivatives of the element energy
+    const float AXa = Gx_aa + Gx_ab, AXb = Gx_ba + Gx_bb;
+    const float BXa = fmaf(bq, Gx_ab, a * Gx_aa), BXb = fmaf(bq, Gx_bb, a * Gx_ba);
+    const float AYa = Gy_aa + Gy_ab, AYb = Gy_ba + Gy_bb;
+    const float BYa = fmaf(bq, Gy_ab, a * Gy_aa), BYb = fmaf(bq, Gy_bb, a * Gy_ba);
+    const float AZa = Gz_aa + Gz_ab, AZb = Gz_ba + Gz_bb;
+    const float BZa = fmaf(bq, Gz_ab, a * Gz_aa), BZb = fmaf(bq, Gz_bb, a * Gz_ba);
+    const float dE = AXa + AXb, dS = AYa + AYb, dW = AZa + AZb;
+    float dXY = fmaf(bq, AXb, a * AXa);
+    dXY = fmaf(a, AYa, dXY); dXY = fmaf(bq, AYb, dXY);
+    float dXZ = BXa + BXb;
+    dXZ = fmaf(a, AZa, dXZ); dXZ = fmaf(bq, AZb, dXZ);
+    const float dYZ = (BYa + BYb) + (BZa + BZb);
+    float dXYZ = fmaf(bq, BXb, a * BXa);
+    dXYZ = fmaf(a, BYa, dXYZ); dXYZ = fmaf(bq, BYb, dXYZ);
+    dXYZ = fmaf(a, BZa, dXYZ); dXYZ = fmaf(bq, BZb, dXYZ);
+    // chain rule to the corners
+    const float r110 = dXY - dXYZ, r101 = dXZ - dXYZ, r011 = dYZ - dXYZ;
+    const float r100 = (dE - r110) - dXZ, r010 = (dS - r110) - dYZ, r001 = (dW - r101) - dYZ;
+    const float r000 = ((r011 - dW) + (dXY - dE)) + (dXZ - dS);
+    r[0] = r000; r[1] = r100; r[2] = r010; r[3] = r110; r[4] = r001; r[5] = r101; r[6] = r011; r[7] = dXYZ;
+}
+
+template <int NX, int M, int MINB>
+__global__ void __launch_bounds__(S3_WARPS * 32, MINB)
+strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G) {
+    extern __shared__ __align__(16) float smem[];
+    constexpr int GS = s3_gs(M);
+    constexpr int CF = 2 * GS;                          // coefficient floats per element row (Gauss rows q = a, b)
+    constexpr int CFQ = CF / 4;                         // ... in 16-byte pieces
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int LW = G.LW, SUBS = 32 >> G.lwsh;
+    const int sub = lane >> G.lwsh, lx = lane & (LW - 1);
+    const unsigned submask = (LW == 32) ? 0xffffffffu : (((1u << LW) - 1u) << (sub * LW));
+    const long long su = ((long long)blockIdx.x * S3_WARPS + warp) * SUBS + sub;
+    if (su >= G.units) return;                          // the other units of the warp synchronise among themselves only
+    const int C = G.C, RS = G.RS;
+    float* ring = smem + (size_t)(warp * SUBS + sub) * C * RS;
+    const int COEF = NX * LW + 4;                       // offset of the coefficient row inside a slot
+    const int H1 = 4 * LW + 4;                          // NX = 8: offset of the second 16 bytes of every lane
+
+    const int b = (int)(su % P.batch);
+    const int tile = (int)((su / P.batch) % G.ntile);
+    const int chunk = (int)(su / ((long long)P.batch * G.ntile));
+    const int nx = P.nx, ny = P.ny, nz = P.nz;
+    const int y0 = tile * G.Ry, e1 = min(y0 + G.Ry, ny - 1);     // element rows y0 .. e1-1, node rows y0 .. e1
+    const int T = e1 - y0 + 1;
+    const bool lasttile = (e1 == ny - 1);               // then node row e1 = ny-1 is this tile's own, else the next tile's
+    const int z0 = chunk * G.Z, ke = min(z0 + G.Z, nz - 1);
+    const int kbeg = max(z0 - 1, 0);                    // element planes kbeg .. ke-1 (kbeg = z0-1: the recomputed one)
+    const int nplanes = ke - kbeg + 1;                  // node planes kbeg .. ke
+    const bool lastchunk = (ke == nz - 1);              // then node plane ke = nz-1 is this chunk's own
+
+    const int x0 = NX * lx;
+    const bool act = x0 < nx;                           // this lane holds nodes of the grid
+    const int x0c = act ? x0 : nx - NX;                 // lanes beyond the grid load valid memory and store nothing
+    const bool first_col = (x0 == 0), last_col = act && (x0 + NX == nx);
+    const size_t plane = (size_t)nx * ny;
+    const float* ub = P.u + (size_t)b * P.nodes + x0c;
+    float* rb = P.r + (size_t)b * P.nodes + x0c;
+    float* sb = lasttile ? nullptr : P.seam + (((size_t)b * (G.ntile - 1) + tile) * nz) * nx + x0c;
+
+    const bool impose = (P.flags & DN_IMPOSE_BC_ON_LOAD) != 0;
+    const bool nomask = (P.flags & DN_NO_MASK) != 0;
+    float bc0 = P.bc_x0, bc1 = P.bc_x1;
+    if (impose) {
+        if (P.bc0_b) bc0 = __ldg(P.bc0_b + b);
+        if (P.bc1_b) bc1 = __ldg(P.bc1_b + b);
+    }
+    const bool iso = (P.hx == P.hy) && (P.hy == P.hz);
+    const float W8 = 0.125f * P.hx * P.hy * P.hz;
+    const float kx = W8 / (P.hx * P.hx), ky = W8 / (P.hy * P.hy), kz = W8 / (P.hz * P.hz);
+    const float kap = iso ? kx : 1.f;                   // isotropic cells: one scale applied at the end
+    const float gs = P.gJ ? __ldg(P.gJ + b) : 1.f;
+    const float fw = P.f_const * P.hx * P.hy * P.hz;    // nodal load of an interior node
+    const bool hasf = (P.f_const != 0.f);
+    // Lane constants that keep the finish of a node row branch-free: output scale, share of the nodal load and
+    // weight in the load energy of the lane's first / last node (Dirichlet columns: masked, or with DN_NO_MASK
+    // carrying half a load); g3 = 0 in the lane whose last element lies right of node nx-1 (it does not exist).
+    const float sc = gs * kap;
+    const float sc0 = (first_col && !nomask) ? 0.f : sc, scL = (last_col && !nomask) ? 0.f : sc;
+    const float lw0 = first_col ? (nomask ? 0.5f : 0.f) : 1.f, lwL = last_col ? (nomask ? 0.5f : 0.f) : 1.f;
+    const float wx0 = first_col ? 0.5f : 1.f, wxL = last_col ? 0.5f : 1.f;
+    const float g3 = last_col ? 0.f : 1.f;
+    const float lm = (lx == 0) ? 0.f : 1.f;             // nothing arrives from the left in the first lane
+
+    // cos(pi x) at the two Gauss columns of each element, duplicated into both halves of a pair
+    u64 cda[NX], cdb[NX];
+#pragma unroll
+    for (int h = 0; h < NX / 2; ++h) {
+        const float4 q = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0c + 4 * h));
+        cda[2 * h] = s3_pack(q.x, q.x); cdb[2 * h] = s3_pack(q.y, q.y);
+        cda[2 * h + 1] = s3_pack(q.z, q.z); cdb[2 * h + 1] = s3_pack(q.w, q.w);
+    }
+
+    // ---- the ring.  Entry n = (plane index pk, row index pj) of the unit goes to slot n mod C: the node row
+    // (every lane its own 16-byte pieces) and, for pk, pj >= 1, the coefficients of element row (pk-1, pj-1).
+    for (int s = lx; s < C; s += LW)                    // the 4 floats right of the last lane's nodes stay zero
+        *reinterpret_cast<float4*>(ring + (size_t)s * RS + 4 * LW) = make_float4(0.f, 0.f, 0.f, 0.f);
+    int pf = 0, pfj = 0, pfk = 0, spf = 0;
+    const float* usrc = ub + (size_t)kbeg * plane + (size_t)y0 * nx;
+    const float* cbase = linepoly + (((size_t)b * (nz - 1) + kbeg) * (ny - 1) + y0) * CF;
+    auto issue = [&]() {
+        if (pfk < nplanes) {                            // uniform in the unit
+            float* slot = ring + (size_t)spf * RS;
+            s3_cp16(slot + 4 * lx, usrc);
+            if constexpr (NX == 8) s3_cp16(slot + H1 + 4 * lx, usrc + 4);
+            if (pfk >= 1 && pfj >= 1) {
+                const float* csrc = cbase + ((size_t)(pfk - 1) * (ny - 1) + (pfj - 1)) * CF;
+                for (int ch = lx; ch < CFQ; ch += LW) s3_cp16(slot + COEF + 4 * ch, csrc + 4 * ch);   // CFQ <= 10, LW >= 8
+            }
+        }
+        s3_commit();                                    // one group per entry, possibly empty
+        ++pf; ++pfj; usrc += nx;
+        if (pfj == T) { pfj = 0; ++pfk; usrc += plane - (size_t)T * nx; }
+        spf = (spf + 1 == C) ? 0 : spf + 1;
+    };
+    for (int i = 0; i < C; ++i) issue();
+
+    auto ldrow = [&](const float* slot, float (&v)[NX + 1]) {
+        const float4 q = *reinterpret_cast<const float4*>(slot + 4 * lx);
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+        if constexpr (NX == 8) {
+            const float4 q1 = *reinterpret_cast<const float4*>(slot + H1 + 4 * lx);
+            v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+        }
+        v[NX] = slot[4 * (lx + 1)];                     // first node of the next lane, or the zero pad
+        if (impose) {
+            if (first_col) v[0] = bc0;
+            if (last_col) v[NX - 1] = bc1;
+        }
+    };
+    // parked partial sums of one node row (plain loads: this thread wrote them one plane ago)
+    auto ld4 = [&](const float* p, float (&v)[NX]) {
+#pragma unroll
+        for (int h = 0; h < NX / 4; ++h) {
+            const float4 q = *reinterpret_cast<const float4*>(p + 4 * h);
+            v[4 * h] = q.x; v[4 * h + 1] = q.y; v[4 * h + 2] = q.z; v[4 * h + 3] = q.w;
+        }
+    };
+    auto st4 = [&](float* p, const float (&v)[NX]) {
+#pragma unroll
+        for (int h = 0; h < NX / 4; ++h)
+            *reinterpret_cast<float4*>(p + 4 * h) = make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]);
+    };
+    // Finish of a node row: from the complete sums `raw` (in units of kap) to the outputs, with the energy terms.
+    // nlrow: the (signed, scaled) nodal load of an interior node of this row and plane; wrow: its weight in the load energy.
+    float en = 0.f, ell = 0.f;
+    auto finish = [&](const float (&raw)[NX], const float (&uv)[NX + 1], const float nlrow, const float wrow, float (&o)[NX]) {
+#pragma unroll
+        for (int c = 0; c < NX; ++c) {
+            en = fmaf(uv[c], raw[c], en);
+            const float s = (c == 0) ? sc0 : (c == NX - 1) ? scL : sc;
+            const float l = (c == 0) ? lw0 * nlrow : (c == NX - 1) ? lwL * nlrow : nlrow;
+            o[c] = fmaf(s, raw[c], l);
+        }
+        if (hasf) {
+            float a = wx0 * uv[0];
+#pragma unroll
+            for (int c = 1; c < NX - 1; ++c) a += uv[c];
+            a = fmaf(wxL, uv[NX - 1], a);
+            ell = fmaf(wrow, a, ell);
+        }
+    };
+
+    auto wrap = [&](int s) { return s >= C ? s - C : s; };
+    float pendL1[NX], pendU1[NX];                       // what the element row below left for the current node row
+    double end = 0.0, eld = 0.0;
+    int sA = 0;                                         // slot of the lower-plane, lower row of the current element row
+    int n = 0;                                          // ... and its entry index
+    for (int kk = 0; kk + 1 < nplanes; ++kk) {
+        const int k = kbeg + kk;                        // element plane k lies between node planes k and k + 1
+        const bool ownlo = (k >= z0);                   // node plane k is finished here (not so in the recomputed plane)
+        const bool hascarry = (kk > 0);                 // ... and has partial sums parked from the step before
+        const bool uptop = lastchunk && (k + 1 == ke);  // node plane k + 1 is the top of the domain: finished now
+        const bool storeup = (k + 1 < ke) || lastchunk; // else plane k + 1 belongs to the next chunk, which recomputes
+        const float wzlo = (k == 0) ? 0.5f : 1.f;
+#pragma unroll
+        for (int c = 0; c < NX; ++c) { pendL1[c] = 0.f; pendU1[c] = 0.f; }
+        for (int jj = 0; jj + 1 < T; ++jj) {
+            s3_wait<0>();                               // everything issued up to the previous step has landed ...
+            __syncwarp(submask);                        // ... is visible to the unit, and the rows it retired are free
+            while (pf < n + C) issue();
+            const int sB = wrap(sA + 1), sC = wrap(sA + T), sD = wrap(sC + 1);
+            const int j = y0 + jj;
+            const float wy = (j == 0) ? 0.5f : 1.f;
+            float* rlo = rb + ((size_t)k * ny + j) * nx;
+            float* rup = rlo + plane;
+            float cin[NX];
+#pragma unroll
+            for (int c = 0; c < NX; ++c) cin[c] = 0.f;
+            if (ownlo && hascarry && act) ld4(rlo, cin);
+            float uA[NX + 1], uB[NX + 1], uC[NX + 1], uD[NX + 1];
+            ldrow(ring + (size_t)sA * RS, uA); ldrow(ring + (size_t)sB * RS, uB);
+            ldrow(ring + (size_t)sC * RS, uC); ldrow(ring + (size_t)sD * RS, uD);
+            u64 ga[GS / 2], gb[GS / 2];                 // Gauss row q = a / b; each entry holds (plane s = a, s = b)
+            {
+                const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(ring + (size_t)sD * RS + COEF);
+#pragma unroll
+                for (int i = 0; i < GS / 4; ++i) {
+                    const ulonglong2 t0 = gp[i], t1 = gp[GS / 4 + i];
+                    ga[2 * i] = t0.x; ga[2 * i + 1] = t0.y; gb[2 * i] = t1.x; gb[2 * i + 1] = t1.y;
+                }
+            }
+            // ---- the NX elements of this lane; what each leaves for its own low-x corner column
+            float tl0[NX], tl1[NX], tu0[NX], tu1[NX];   // to node (c, j, k), (c, j+1, k), (c, j, k+1), (c, j+1, k+1)
+            float p100 = 0.f, p110 = 0.f, p101 = 0.f, p111 = 0.f;
+#pragma unroll
+            for (int c = 0; c < NX; ++c) {
+                const float eA = uA[c + 1] - uA[c], eB = uB[c + 1] - uB[c];
+                const float eC = uC[c + 1] - uC[c], eD = uD[c + 1] - uD[c];
+                const float slo = uB[c] - uA[c], sup = uD[c] - uC[c], w0 = uC[c] - uA[c];
+                const float txy = eB - eA, txyu = eD - eC, txz = eC - eA, tyz = sup - slo, txyz = txyu - txy;
+                float nu[8], r[8];
+                s3_nu_gauss<M>(ga, gb, cda[c], cdb[c], nu);
+                s3_element(nu, eA, slo, w0, txy, txz, tyz, txyz, iso, kx, ky, kz, r);
+                if (c == NX - 1) { r[0] *= g3; r[2] *= g3; r[4] *= g3; r[6] *= g3; }
+                tl0[c] = r[0] + p100; tl1[c] = r[2] + p110; tu0[c] = r[4] + p101; tu1[c] = r[6] + p111;
+                p100 = r[1]; p110 = r[3]; p101 = r[5]; p111 = r[7];
+            }
+            // the last element of the lane on the left feeds this lane's first column
+            {
+                const float a100 = __shfl_up_sync(submask, p100, 1, LW), a110 = __shfl_up_sync(submask, p110, 1, LW);
+                const float a101 = __shfl_up_sync(submask, p101, 1, LW), a111 = __shfl_up_sync(submask, p111, 1, LW);
+                tl0[0] = fmaf(a100, lm, tl0[0]); tl1[0] = fmaf(a110, lm, tl1[0]);
+                tu0[0] = fmaf(a101, lm, tu0[0]); tu1[0] = fmaf(a111, lm, tu1[0]);
+            }
+            float o[NX];
+            // ---- node row (j, k): complete now
+            if (ownlo) {
+                float raw[NX];
+#pragma unroll
+                for (int c = 0; c < NX; ++c) raw[c] = (tl0[c] + pendL1[c]) + cin[c];
+                finish(raw, uA, -gs * fw * wy * wzlo, wy * wzlo, o);
+                if (act) st4(rlo, o);
+            }
+            // ---- node row (j, k + 1): parked until the next plane, or complete if that plane is the top of the domain
+            {
+                float part[NX];
+#pragma unroll
+                for (int c = 0; c < NX; ++c) { part[c] = tu0[c] + pendU1[c]; pendL1[c] = tl1[c]; pendU1[c] = tu1[c]; }
+                if (uptop) {
+                    finish(part, uC, -gs * fw * wy * 0.5f, wy * 0.5f, o);
+                    if (act) st4(rup, o);
+                } else if (storeup && act) {
+                    st4(rup, part);
+                }
+            }
+            sA = sB; ++n;
+        }
+        // ---- the top node row e1 of the tile gets nothing more in this plane.  It is this tile's own if it is the
+        // top of the domain; else it belongs to the next tile and its sums go to the seam array (no load term: the
+        // owner adds it).
+        {
+            const int sU = wrap(sA + T);
+            float uT[NX + 1], uTu[NX + 1];
+            ldrow(ring + (size_t)sA * RS, uT); ldrow(ring + (size_t)sU * RS, uTu);
+            float* plo = lasttile ? rb + ((size_t)k * ny + e1) * nx : sb + (size_t)k * nx;
+            float* pup = lasttile ? plo + plane : plo + nx;
+            const float wyT = lasttile ? 0.5f : 0.f;
+            float o[NX];
+            if (ownlo) {
+                float cin[NX], raw[NX];
+#pragma unroll
+                for (int c = 0; c < NX; ++c) cin[c] = 0.f;
+                if (hascarry && act) ld4(plo, cin);
+#pragma unroll
+                for (int c = 0; c < NX; ++c) raw[c] = pendL1[c] + cin[c];
+                finish(raw, uT, -gs * fw * wyT * wzlo, wyT * wzlo, o);
+                if (act) st4(plo, o);
+            }
+            if (uptop) {
+                finish(pendU1, uTu, -gs * fw * wyT * 0.5f, wyT * 0.5f, o);
+                if (act) st4(pup, o);
+            } else if (storeup && act) {
+                st4(pup, pendU1);
+            }
+            sA = wrap(sA + 1); ++n;
+        }
+        end += (double)en; eld += (double)ell;          // per-plane sums go to double
+        en = 0.f; ell = 0.f;
+    }
+    s3_wait<0>();
+
+    // ---- energy partial of this unit: its lanes summed in a fixed order in double
+    double d = act ? 0.5 * (double)kap * end : 0.0, l = (act && hasf) ? (double)fw * eld : 0.0;
+    for (int off = LW >> 1; off > 0; off >>= 1) {
+        d += __shfl_down_sync(submask, d, off, LW);
+        l += __shfl_down_sync(submask, l, off, LW);
+    }
+    if (lx == 0) {
+        double* slot = P.partials + 2 * ((size_t)b * P.nblk + (size_t)chunk * G.ntile + tile);
+        slot[0] = d; slot[1] = l;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Coefficient table: for element row ey of element plane ez of sample b, the polynomials (in c = cos(pi x)) of
+// the KL exponent along the four Gauss lines (y_q, z_s):  sum_i g_i T_i(c)  with
+// g_i = sum_{j,k} ckl[i][j][k] cos(j pi y_q) cos(k pi z_s), converted from the Chebyshev basis to monomials in
+// double.  The scaled weights and the cosines are the float tables every kernel family reads.  One thread per line.
+// ---------------------------------------------------------------------------------------------------------
+__global__ void linepoly3d_kernel(const Params P, float* __restrict__ out, const int gs, const long long nlines) {
+    constexpr int MX = DN_MAX_KL_MODES;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= nlines) return;
+    const int m = P.m;
+    const int s = (int)(idx & 1), q = (int)((idx >> 1) & 1);
+    const long long row = idx >> 2;                                     // (b * (nz-1) + ez) * (ny-1) + ey
+    const int ey = (int)(row % (P.ny - 1));
+    const int ez = (int)((row / (P.ny - 1)) % (P.nz - 1));
+    const long long b = row / ((long long)(P.ny - 1) * (P.nz - 1));
+    const float* cy = P.cg[1] + 2 * ey + q;
+    const float* cz = P.cg[2] + 2 * ez + s;
+    const float* w = P.ckl + b * m * m * m;
+    double g[MX];
+#pragma unroll
+    for (int i = 0; i < MX; ++i) {
+        double acc = 0.0;
+        if (i < m) {
+            for (int j = 0; j < m; ++j) {
+                double inner = 0.0;
+                for (int k = 0; k < m; ++k) inner += (double)w[(i * m + j) * m + k] * (double)cz[(size_t)k * P.gstride[2]];
+                acc += inner * (double)cy[(size_t)j * P.gstride[1]];
+            }
+        }
+        g[i] = acc;
+    }
+    // sum_i g_i T_i(c) in the monomial basis, T_{i+1} = 2 c T_i - T_{i-1}
+    double acc[MX + 1], tp[MX + 1], tc[MX + 1];
+#pragma unroll
+    for (int k = 0; k <= MX; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
+#pragma unroll
+    for (int i = 1; i <= MX; ++i) {
+        if (i > m) break;                              // uniform; the remaining terms are zero
+#pragma unroll
+        for (int k = 0; k <= MX; ++k) acc[k] += g[i - 1] * tc[k];
+        double tn[MX + 1];
+#pragma unroll
+        for (int k = 0; k <= MX; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
+#pragma unroll
+        for (int k = 0; k <= MX; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
+    }
+    float* dst = out + row * (2 * gs) + q * gs + s;
+#pragma unroll
+    for (int i = 0; i < s3_gs(MX) / 2; ++i)            // coefficient i of plane s; the padding of the row is zero
+        if (2 * i + s < gs) dst[2 * i] = (i <= m) ? (float)acc[i <= MX ? i : MX] : 0.f;
+}
+
+int s3_sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        (void)cudaGetLastError();
+        n = 148;
+    }
+    return n;
+}
+
+constexpr size_t S3_SMEM_SM = 233472;              // shared memory of an SM; a block also reserves 1 KiB
+constexpr size_t S3_SMEM_BLOCK = 232448;           // most a block can ask for
+
+int s3_nxl(int nx) { return (nx > 128) ? 8 : 4; }  // nodes per lane
+int s3_minb(int nxl) { return (nxl == 8) ? 3 : 4; } // resident blocks of 4 warps per SM the kernel is compiled for
+
+S3Geo geometry3s(const dn_problem& p) {
+    S3Geo g{};
+    const int nx = p.grid.nx, ny = p.grid.ny, nz = p.grid.nz;
+    const int NX = s3_nxl(nx), minb = s3_minb(NX);
+    g.LW = 8; g.lwsh = 3;
+    while (g.LW * NX < nx) { g.LW *= 2; ++g.lwsh; }
+    const int subs = 32 / g.LW;
+    const int m = p.kl_modes;
+    g.RS = NX * g.LW + 4 + 2 * s3_gs(m);
+    size_t per_block = (S3_SMEM_SM - (size_t)minb * 1024) / minb;
+    if (per_block > S3_SMEM_BLOCK) per_block = S3_SMEM_BLOCK;
+    const int cmax = (int)(per_block / ((size_t)S3_WARPS * subs * g.RS * sizeof(float)));
+    int ry_max = cmax - 2 - S3_D;
+    if (ry_max > ny - 1) ry_max = ny - 1;
+    if (ry_max > 64) ry_max = 64;
+    if (ry_max < 1) ry_max = 1;
+    const long long slots = (long long)s3_sm_count() * minb * S3_WARPS * subs;
+    // (Ry, Z) by a cost model: whole waves of units; a unit pays one more plane (the recomputed one) and, per plane,
+    // the finish of its top row; flat tiles also pay the seam traffic and the fix-up pass.
+    double best = -1.0;
+    for (int Ry = 1; Ry <= ry_max; ++Ry) {
+        const long long ntile = (ny - 1 + Ry - 1) / Ry;
+        for (int Z = 1; Z <= nz - 1; ++Z) {
+            const long long nchunk = (nz - 1 + Z - 1) / Z;
+            const long long units = (long long)p.batch * ntile * nchunk;
+            const long long waves = (units + slots - 1) / slots;
+            const double cost = (double)waves * (Z + 1) * (Ry + 0.8) * (1.0 + 0.25 / Ry);
+            if (best < 0 || cost < best * (1.0 - 1e-9)) {
+                best = cost;
+                g.Ry = Ry; g.Z = Z; g.ntile = (int)ntile; g.nchunk = (int)nchunk; g.units = units;
+            }
+        }
+    }
+    g.C = g.Ry + 2 + S3_D;
+    return g;
+}
+
+template <int NX, int M, int MINB>
+cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+    const int subs = 32 / g.LW;
+    const size_t smem = sizeof(float) * (size_t)S3_WARPS * subs * g.C * g.RS;
+    const long long per_block = (long long)S3_WARPS * subs;
+    const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
+    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    strip3d_kernel<NX, M, MINB><<<blocks, S3_WARPS * 32, smem, s>>>(P, linepoly, g);
+    return cudaGetLastError();
+}
+
+template <int M>
+cudaError_t launch_m3(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+    return (s3_nxl(P.nx) == 8) ? launch_nm<8, M, 3>(P, linepoly, g, s) : launch_nm<4, M, 4>(P, linepoly, g, s);
+}
+
+dn_problem s3_problem_of(const Params& P) {
+    dn_problem p{};
+    p.grid.dim = 3; p.grid.nx = P.nx; p.grid.ny = P.ny; p.grid.nz = P.nz; p.batch = P.batch;
+    p.nu_mode = P.nu_mode; p.kl_modes = P.m;
+    return p;
+}
+
+}  // namespace
+
+// Rows of at most 128 nodes take 4 nodes per lane, rows of at most 256 nodes 8 (then nx must be a multiple of 8,
+// so that only the last element of the last lane falls outside the grid).
+bool strip3d_applicable(const dn_problem& p) {
+    if (!(p.grid.dim == 3 && p.f == nullptr && p.nu_mode == DN_NU_KL_GAUSS && p.grid.nx % 4 == 0 && p.grid.nx >= 8 &&
+          p.grid.nx <= 256 && p.grid.ny >= 2 && p.grid.nz >= 2))
+        return false;
+    return p.grid.nx <= 128 || p.grid.nx % 8 == 0;
+}
+
+Launch strip3d_geometry(const dn_problem& p) {
+    const S3Geo g = geometry3s(p);
+    Launch l{};
+    l.path = PATH_STRIP3D;
+    l.nblk = g.ntile * g.nchunk;
+    l.chunk = g.Z;
+    l.variant = g.Ry;
+    return l;
+}
+
+size_t strip3d_seam_floats(const dn_problem& p) {
+    if (!strip3d_applicable(p)) return 0;
+    const S3Geo g = geometry3s(p);
+    return (size_t)p.batch * (g.ntile - 1) * p.grid.nz * p.grid.nx;
+}
+
+size_t strip3d_linepoly_floats(const dn_problem& p) {
+    if (!strip3d_applicable(p)) return 0;
+    return (size_t)p.batch * (p.grid.nz - 1) * (p.grid.ny - 1) * 2 * s3_gs(p.kl_modes);
+}
+
+cudaError_t launch_linepoly3d(const Params& P, float* linepoly, cudaStream_t s) {
+    const long long nlines = 4ll * P.batch * (P.nz - 1) * (P.ny - 1);
+    linepoly3d_kernel<<<(unsigned)((nlines + 127) / 128), 128, 0, s>>>(P, linepoly, s3_gs(P.m), nlines);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t s) {
+    const S3Geo g = geometry3s(s3_problem_of(P));
+    cudaError_t e = cudaErrorInvalidValue;
+    switch (P.m) {
+        case 1: e = launch_m3<1>(P, linepoly, g, s); break;
+        case 2: e = launch_m3<2>(P, linepoly, g, s); break;
+        case 3: e = launch_m3<3>(P, linepoly, g, s); break;
+        case 4: e = launch_m3<4>(P, linepoly, g, s); break;
+        case 5: e = launch_m3<5>(P, linepoly, g, s); break;
+        case 6: e = launch_m3<6>(P, linepoly, g, s); break;
+        case 7: e = launch_m3<7>(P, linepoly, g, s); break;
+        case 8: e = launch_m3<8>(P, linepoly, g, s); break;
+    }
+    if (e != cudaSuccess) return e;
+    if (g.ntile > 1) return launch_seam_fixup(P.r, P.seam, P.nx, P.ny, P.nz, g.Ry, g.ntile - 1, P.batch, s);
+    return cudaSuccess;
+}
+
+}  // namespace dn

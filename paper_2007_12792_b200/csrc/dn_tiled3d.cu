@@ -671,6 +671,13 @@ Launch tiled3d_geometry(const dn_problem& p) {
     return l;
 }
 
+cudaError_t launch_seam_fixup(float* r, const float* seam, int nx, int ny, int nz, int rows_per_tile, int nseam, int batch,
+                              cudaStream_t s) {
+    const long long total4 = (long long)batch * nseam * nz * (nx / 4);
+    seam_fixup_kernel<<<(unsigned)((total4 + 255) / 256), 256, 0, s>>>(r, seam, nx, ny, nz, rows_per_tile, nseam, total4);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s) {
     dn_problem p{};
     p.grid.dim = 3; p.grid.nx = P.nx; p.grid.ny = P.ny; p.grid.nz = P.nz; p.batch = P.batch;

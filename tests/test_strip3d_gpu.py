@@ -1,0 +1,73 @@
+"""GPU parity of the 3D strip kernel (rows of at most 256 nodes, KL diffusivity at the Gauss points, energy and residual
+fused) against the fp64 oracle: every lane layout (4 or 8 nodes per lane; 8, 16 or 32 lanes per unit, i.e. 4, 2 or 1
+units per warp), rows that end inside a lane group, one and many tiles and chunks, batches that leave units of a warp
+idle, and every option the kernel serves."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2007_12792_b200 import binding as B
+from paper_2007_12792_b200 import inputs
+from parity_util import dev, make_problems, run_gpu, check
+
+pytestmark = pytest.mark.gpu
+
+# (nx, ny, nz, batch, m)
+SIZES = [(8, 2, 2, 1, 1), (12, 11, 6, 2, 2), (32, 9, 7, 3, 3), (28, 45, 5, 1, 2), (36, 10, 6, 5, 2), (64, 20, 3, 1, 2),
+         (60, 37, 6, 2, 3), (64, 64, 17, 3, 2), (100, 7, 9, 2, 4), (128, 13, 12, 1, 8), (132, 9, 5, 1, 3), (136, 6, 7, 2, 2),
+         (200, 5, 4, 1, 5), (256, 17, 5, 1, 3), (256, 40, 30, 2, 6), (64, 150, 40, 9, 2), (16, 8, 300, 1, 1)]
+
+
+@pytest.mark.parametrize("nx,ny,nz,batch,m", SIZES)
+def test_strip3d_parity(nx, ny, nz, batch, m):
+    inp = inputs.random_inputs(3, nx, ny, nz, batch, m, seed=11 + nx + 3 * ny + nz, f_const=0.6)
+    po, pg = make_problems(inp, B.DN_NU_KL_GAUSS)
+    expect = "strip3d" if (nx <= 128 or nx % 8 == 0) else "tiled3d"
+    assert B.dn_path_name(pg) == expect
+    Jo, _, _, ro = oracle.energy_grad(po, inp.u)
+    Jg, rg = run_gpu(pg, inp.u)
+    check(Jg, rg, Jo, ro, f"strip3d {nx}x{ny}x{nz} b{batch} m{m}")
+    assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
+
+
+@pytest.mark.parametrize("nx,ny,nz", [(64, 9, 6), (24, 6, 5), (256, 7, 6), (128, 12, 9)])
+def test_strip3d_options(nx, ny, nz):
+    inp = inputs.random_inputs(3, nx, ny, nz, 3, 3, seed=42, f_const=-0.4)
+    u = inputs.random_field(inp.u.shape, 8)           # boundary values NOT satisfied
+    gJ = np.array([1.5, -2.0, 0.25], dtype=np.float32)
+    for flags in (0, B.DN_NO_MASK, B.DN_IMPOSE_BC_ON_LOAD, B.DN_IMPOSE_BC_ON_LOAD | B.DN_NO_MASK):
+        po, pg = make_problems(inp, B.DN_NU_KL_GAUSS, flags=flags, bc=(0.8, -0.3))
+        assert B.dn_path_name(pg) == "strip3d"
+        Jo, _, _, ro = oracle.energy_grad(po, u, gJ=gJ.astype(np.float64))
+        Jg, rg = run_gpu(pg, u, gJ=gJ)
+        check(Jg, rg, Jo, ro, f"flags={flags}")
+        if not (flags & B.DN_NO_MASK):
+            assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
+    # rectangular cells (hx != hy != hz take the scaled path), residual-only call, determinism with a stale workspace
+    po, pg = make_problems(inp, B.DN_NU_KL_GAUSS)
+    ws = B.new_workspace(pg)
+    outs = []
+    for it in range(3):
+        ws.fill_(255 if it == 1 else 0)
+        r = torch.empty(pg.shape, device="cuda"); J = torch.empty(3, device="cuda")
+        B.dn_energy_grad(pg, dev(u), None, J if it < 2 else None, r, ws)
+        torch.cuda.synchronize()
+        outs.append((J.cpu().numpy().copy(), r.cpu().numpy().copy()))
+    assert outs[0][0].tobytes() == outs[1][0].tobytes()
+    assert outs[0][1].tobytes() == outs[1][1].tobytes() == outs[2][1].tobytes()
+    J1 = torch.empty(3, device="cuda")
+    B.dn_energy(pg, dev(u), J1, ws)                   # the energy-only call runs another kernel family
+    assert np.allclose(J1.cpu().numpy(), outs[0][0], rtol=1e-5, atol=0)
+
+
+def test_strip3d_isotropic_cells_and_closed_form():
+    """Cubic cells take the unscaled path; u = 1 - x with all weights zero (nu = 1) has J = 1/2 and r = 0 off the faces."""
+    n = 48
+    u = np.broadcast_to((1 - np.arange(n) / (n - 1)).astype(np.float32), (2, n, n, n)).copy()
+    pg = B.Problem(dim=3, nx=n, ny=n, nz=n, batch=2, nu_mode=B.DN_NU_KL_GAUSS, kl_modes=2,
+                   kl_w=torch.zeros(2, 2, 2, 2, device="cuda"))
+    assert B.dn_path_name(pg) == "strip3d"
+    Jg, rg = run_gpu(pg, u)
+    assert np.allclose(Jg, 0.5, rtol=1e-5)
+    assert np.abs(rg).max() < 1e-5 / n
