@@ -39,6 +39,7 @@
 // element plane once per call in double ([B][nz-1][ny-1][2][GS] floats: Gauss row q, then coefficient i and Gauss
 // plane s interleaved for packed two-wide FMAs); they travel through the ring with the node row that completes
 // the element row.
+#include <cstdlib>
 #include "dn_internal.cuh"
 
 namespace dn {
@@ -74,6 +75,14 @@ __device__ __forceinline__ void s3_cp16(float* smem_dst, const float* gsrc) {
 }
 __device__ __forceinline__ void s3_cp16_if(float* smem_dst, const float* gsrc, int pred) {    // predicated, no branch
     const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.s32 p, %2, 0;\n\t@p cp.async.cg.shared.global [%0], [%1], 16;\n\t}"
+                 ::"r"(d), "l"(gsrc), "r"(pred) : "memory");
+}
+// the same with the shared-memory address already converted
+__device__ __forceinline__ void s3_cp16s(unsigned d, const float* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void s3_cp16s_if(unsigned d, const float* gsrc, int pred) {
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.s32 p, %2, 0;\n\t@p cp.async.cg.shared.global [%0], [%1], 16;\n\t}"
                  ::"r"(d), "l"(gsrc), "r"(pred) : "memory");
 }
@@ -172,17 +181,35 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const int LW = G.LW, SUBS = 32 >> G.lwsh;
     const int sub = lane >> G.lwsh, lx = lane & (LW - 1);
     const unsigned submask = (LW == 32) ? 0xffffffffu : (((1u << LW) - 1u) << (sub * LW));
+    const int nx = P.nx, ny = P.ny, nz = P.nz;
+    const int x0 = NX * lx;
+    const bool act = x0 < nx;                           // this lane holds nodes of the grid
+    const int x0c = act ? x0 : nx - NX;                 // lanes beyond the grid load valid memory and store nothing
+
+    // ---- shared by the block: cos(pi x) at the two Gauss columns of each element of a lane, duplicated into both
+    // halves of a pair, as float4 (ca, ca, cb, cb) at [element c][lane of the unit]
+    float4* cps = reinterpret_cast<float4*>(smem);
+    for (int i = threadIdx.x; i < NX * LW; i += blockDim.x) {
+        const int c = i >> G.lwsh, l = i & (LW - 1);
+        const int xe = min(NX * l, nx - NX) + c;        // element index = index of its left node
+        const float ca = __ldg(P.cg[0] + 2 * xe), cb = __ldg(P.cg[0] + 2 * xe + 1);
+        cps[i] = make_float4(ca, ca, cb, cb);
+    }
+    __syncthreads();                                    // the only block-wide barrier: before the march starts
+    const float4* cpl = cps + lx;
+
     const long long su = ((long long)blockIdx.x * S3_WARPS + warp) * SUBS + sub;
     if (su >= G.units) return;                          // the other units of the warp synchronise among themselves only
     const int C = G.C, RS = G.RS;
-    float* ring = smem + (size_t)(warp * SUBS + sub) * C * RS;
+    const unsigned RSB = (unsigned)RS * 4u, RINGB = (unsigned)C * RSB;
+    float* ring = smem + 4 * NX * LW + (size_t)(warp * SUBS + sub) * C * RS;
+    const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring);
     const int COEF = NX * LW + 4;                       // offset of the coefficient row inside a slot
     const int H1 = 4 * LW + 4;                          // NX = 8: offset of the second 16 bytes of every lane
 
     const int b = (int)(su % P.batch);
     const int tile = (int)((su / P.batch) % G.ntile);
     const int chunk = (int)(su / ((long long)P.batch * G.ntile));
-    const int nx = P.nx, ny = P.ny, nz = P.nz;
     const int y0 = tile * G.Ry, e1 = min(y0 + G.Ry, ny - 1);     // element rows y0 .. e1-1, node rows y0 .. e1
     const int T = e1 - y0 + 1;
     const bool lasttile = (e1 == ny - 1);               // then node row e1 = ny-1 is this tile's own, else the next tile's
@@ -191,9 +218,6 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const int nplanes = ke - kbeg + 1;                  // node planes kbeg .. ke
     const bool lastchunk = (ke == nz - 1);              // then node plane ke = nz-1 is this chunk's own
 
-    const int x0 = NX * lx;
-    const bool act = x0 < nx;                           // this lane holds nodes of the grid
-    const int x0c = act ? x0 : nx - NX;                 // lanes beyond the grid load valid memory and store nothing
     const bool first_col = (x0 == 0), last_col = act && (x0 + NX == nx);
     const size_t plane = (size_t)nx * ny;
     const float* ub = P.u + (size_t)b * P.nodes + x0c;
@@ -224,40 +248,36 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const float g3 = last_col ? 0.f : 1.f;
     const float lm = (lx == 0) ? 0.f : 1.f;             // nothing arrives from the left in the first lane
 
-    // cos(pi x) at the two Gauss columns of each element, duplicated into both halves of a pair
-    u64 cda[NX], cdb[NX];
-#pragma unroll
-    for (int h = 0; h < NX / 2; ++h) {
-        const float4 q = __ldg(reinterpret_cast<const float4*>(P.cg[0] + 2 * x0c + 4 * h));
-        cda[2 * h] = s3_pack(q.x, q.x); cdb[2 * h] = s3_pack(q.y, q.y);
-        cda[2 * h + 1] = s3_pack(q.z, q.z); cdb[2 * h + 1] = s3_pack(q.w, q.w);
-    }
-
     // ---- the ring.  Entry n = (plane index pk, row index pj) of the unit goes to slot n mod C: the node row
     // (every lane its own 16-byte pieces) and, for pk, pj >= 1, the coefficients of element row (pk-1, pj-1).
     for (int s = lx; s < C; s += LW)                    // the 4 floats right of the last lane's nodes stay zero
         *reinterpret_cast<float4*>(ring + (size_t)s * RS + 4 * LW) = make_float4(0.f, 0.f, 0.f, 0.f);
-    int pf = 0, pfj = 0, pfk = 0, spf = 0;
+    int pf = 0, pfj = 0, pfk = 0;
+    unsigned pfo = 0;                                   // byte offset of the slot the next entry goes to
     const float* usrc = ub + (size_t)kbeg * plane + (size_t)y0 * nx;
-    const float* cbase = linepoly + (((size_t)b * (nz - 1) + kbeg) * (ny - 1) + y0) * CF;
+    // coefficient piece of this lane: of element row (pfk-1, pfj-1), so the pointer starts one row and one plane low
+    const float* csrc = linepoly + (((size_t)b * (nz - 1) + kbeg) * (ny - 1) + y0) * CF
+                        - ((size_t)(ny - 1) + 1) * CF + 4 * (lx < CFQ ? lx : 0);
+    const long long uwrap = (long long)plane - (long long)T * nx, cwrap = ((long long)(ny - 1) - T) * CF;
+    const unsigned d0 = ring_s + 16u * lx, d1 = ring_s + 4u * H1 + 16u * lx, dc = ring_s + 4u * COEF + 16u * (lx < CFQ ? lx : 0);
     auto issue = [&]() {
         if (pfk < nplanes) {                            // uniform in the unit
-            float* slot = ring + (size_t)spf * RS;
-            s3_cp16(slot + 4 * lx, usrc);
-            if constexpr (NX == 8) s3_cp16(slot + H1 + 4 * lx, usrc + 4);
-            if (pfk >= 1 && pfj >= 1) {
-                const float* csrc = cbase + ((size_t)(pfk - 1) * (ny - 1) + (pfj - 1)) * CF;
-                for (int ch = lx; ch < CFQ; ch += LW) s3_cp16(slot + COEF + 4 * ch, csrc + 4 * ch);   // CFQ <= 10, LW >= 8
-            }
+            s3_cp16s(d0 + pfo, usrc);
+            if constexpr (NX == 8) s3_cp16s(d1 + pfo, usrc + 4);
+            const int cok = (pfk >= 1 && pfj >= 1) ? 1 : 0;
+            s3_cp16s_if(dc + pfo, csrc, (lx < CFQ) ? cok : 0);
+            if constexpr (CFQ > 8) s3_cp16s_if(dc + pfo + 16u * 8u, csrc + 32, (lx + 8 < CFQ && LW == 8) ? cok : 0);
         }
         s3_commit();                                    // one group per entry, possibly empty
-        ++pf; ++pfj; usrc += nx;
-        if (pfj == T) { pfj = 0; ++pfk; usrc += plane - (size_t)T * nx; }
-        spf = (spf + 1 == C) ? 0 : spf + 1;
+        ++pf; ++pfj; usrc += nx; csrc += CF;
+        if (pfj == T) { pfj = 0; ++pfk; usrc += uwrap; csrc += cwrap; }
+        pfo += RSB;
+        if (pfo == RINGB) pfo = 0;
     };
     for (int i = 0; i < C; ++i) issue();
 
-    auto ldrow = [&](const float* slot, float (&v)[NX + 1]) {
+    auto ldrow = [&](const unsigned off, float (&v)[NX + 1]) {
+        const float* slot = reinterpret_cast<const float*>(reinterpret_cast<const char*>(ring) + off);
         const float4 q = *reinterpret_cast<const float4*>(slot + 4 * lx);
         v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
         if constexpr (NX == 8) {
@@ -283,144 +303,166 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
         for (int h = 0; h < NX / 4; ++h)
             *reinterpret_cast<float4*>(p + 4 * h) = make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]);
     };
-    // Finish of a node row: from the complete sums `raw` (in units of kap) to the outputs, with the energy terms.
-    // nlrow: the (signed, scaled) nodal load of an interior node of this row and plane; wrow: its weight in the load energy.
-    float en = 0.f, ell = 0.f;
-    auto finish = [&](const float (&raw)[NX], const float (&uv)[NX + 1], const float nlrow, const float wrow, float (&o)[NX]) {
-#pragma unroll
-        for (int c = 0; c < NX; ++c) {
-            en = fmaf(uv[c], raw[c], en);
-            const float s = (c == 0) ? sc0 : (c == NX - 1) ? scL : sc;
-            const float l = (c == 0) ? lw0 * nlrow : (c == NX - 1) ? lwL * nlrow : nlrow;
-            o[c] = fmaf(s, raw[c], l);
-        }
-        if (hasf) {
-            float a = wx0 * uv[0];
-#pragma unroll
-            for (int c = 1; c < NX - 1; ++c) a += uv[c];
-            a = fmaf(wxL, uv[NX - 1], a);
-            ell = fmaf(wrow, a, ell);
-        }
-    };
+    auto wrapb = [&](unsigned o) { return o >= RINGB ? o - RINGB : o; };
 
-    auto wrap = [&](int s) { return s >= C ? s - C : s; };
     float pendL1[NX], pendU1[NX];                       // what the element row below left for the current node row
     double end = 0.0, eld = 0.0;
-    int sA = 0;                                         // slot of the lower-plane, lower row of the current element row
+    unsigned oA = 0;                                    // slot (byte offset) of the lower-plane, lower row of the current element row
     int n = 0;                                          // ... and its entry index
+    const unsigned TB = (unsigned)T * RSB;
     for (int kk = 0; kk + 1 < nplanes; ++kk) {
         const int k = kbeg + kk;                        // element plane k lies between node planes k and k + 1
         const bool ownlo = (k >= z0);                   // node plane k is finished here (not so in the recomputed plane)
-        const bool hascarry = (kk > 0);                 // ... and has partial sums parked from the step before
-        const bool uptop = lastchunk && (k + 1 == ke);  // node plane k + 1 is the top of the domain: finished now
-        const bool storeup = (k + 1 < ke) || lastchunk; // else plane k + 1 belongs to the next chunk, which recomputes
+        const bool hascarry = ownlo && (kk > 0) && act; // ... and has partial sums parked from the step before
+        // the sums of node plane k + 1 are parked; not so if that plane belongs to the next chunk, which recomputes
+        // them (the top plane of the domain is this chunk's own: it is finished after the march)
+        const bool storeup = ((k + 1 < ke) || lastchunk) && act;
         const float wzlo = (k == 0) ? 0.5f : 1.f;
+        const float nllo = -gs * fw * wzlo;
+        float enlo = 0.f, ello = 0.f;
 #pragma unroll
         for (int c = 0; c < NX; ++c) { pendL1[c] = 0.f; pendU1[c] = 0.f; }
+        float* rlo = rb + ((size_t)k * ny + y0) * nx;
         for (int jj = 0; jj + 1 < T; ++jj) {
             s3_wait<0>();                               // everything issued up to the previous step has landed ...
             __syncwarp(submask);                        // ... is visible to the unit, and the rows it retired are free
             while (pf < n + C) issue();
-            const int sB = wrap(sA + 1), sC = wrap(sA + T), sD = wrap(sC + 1);
-            const int j = y0 + jj;
-            const float wy = (j == 0) ? 0.5f : 1.f;
-            float* rlo = rb + ((size_t)k * ny + j) * nx;
-            float* rup = rlo + plane;
             float cin[NX];
 #pragma unroll
             for (int c = 0; c < NX; ++c) cin[c] = 0.f;
-            if (ownlo && hascarry && act) ld4(rlo, cin);
+            if (hascarry) ld4(rlo, cin);
+            const unsigned oB = wrapb(oA + RSB), oC = wrapb(oA + TB), oD = wrapb(oC + RSB);
+            const float wy = (y0 + jj == 0) ? 0.5f : 1.f;
             float uA[NX + 1], uB[NX + 1], uC[NX + 1], uD[NX + 1];
-            ldrow(ring + (size_t)sA * RS, uA); ldrow(ring + (size_t)sB * RS, uB);
-            ldrow(ring + (size_t)sC * RS, uC); ldrow(ring + (size_t)sD * RS, uD);
+            ldrow(oA, uA); ldrow(oB, uB); ldrow(oC, uC); ldrow(oD, uD);
             u64 ga[GS / 2], gb[GS / 2];                 // Gauss row q = a / b; each entry holds (plane s = a, s = b)
             {
-                const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(ring + (size_t)sD * RS + COEF);
+                const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(reinterpret_cast<const char*>(ring) + oD) + COEF / 4;
 #pragma unroll
                 for (int i = 0; i < GS / 4; ++i) {
                     const ulonglong2 t0 = gp[i], t1 = gp[GS / 4 + i];
                     ga[2 * i] = t0.x; ga[2 * i + 1] = t0.y; gb[2 * i] = t1.x; gb[2 * i + 1] = t1.y;
                 }
             }
-            // ---- the NX elements of this lane; what each leaves for its own low-x corner column
-            float tl0[NX], tl1[NX], tu0[NX], tu1[NX];   // to node (c, j, k), (c, j+1, k), (c, j, k+1), (c, j+1, k+1)
-            float p100 = 0.f, p110 = 0.f, p101 = 0.f, p111 = 0.f;
+            const float nlrow = nllo * wy;
+            float olo[NX], oup[NX];
+            // Finish of node column c of this row on both planes: `lo` / `up` are everything the lane's elements of this
+            // row contribute to node (c, j, k) / (c, j, k+1), `lo1` / `up1` what they leave for row j + 1.
+            auto node = [&](const int c, const float lo, const float lo1, const float up, const float up1) {
+                const float raw = (lo + pendL1[c]) + cin[c];
+                oup[c] = up + pendU1[c];
+                pendL1[c] = lo1; pendU1[c] = up1;
+                enlo = fmaf(uA[c], raw, enlo);
+                const float s = (c == 0) ? sc0 : (c == NX - 1) ? scL : sc;
+                const float l = (c == 0) ? lw0 * nlrow : (c == NX - 1) ? lwL * nlrow : nlrow;
+                olo[c] = fmaf(s, raw, l);
+            };
+            // ---- the NX elements of this lane, from right to left: element c completes node column c + 1
+            float q000 = 0.f, q010 = 0.f, q001 = 0.f, q011 = 0.f;   // own-corner contributions of the element on the right
+            float a100 = 0.f, a110 = 0.f, a101 = 0.f, a111 = 0.f;   // from the last element of the lane on the left
 #pragma unroll
-            for (int c = 0; c < NX; ++c) {
+            for (int c = NX - 1; c >= 0; --c) {
                 const float eA = uA[c + 1] - uA[c], eB = uB[c + 1] - uB[c];
                 const float eC = uC[c + 1] - uC[c], eD = uD[c + 1] - uD[c];
                 const float slo = uB[c] - uA[c], sup = uD[c] - uC[c], w0 = uC[c] - uA[c];
                 const float txy = eB - eA, txyu = eD - eC, txz = eC - eA, tyz = sup - slo, txyz = txyu - txy;
                 float nu[8], r[8];
-                s3_nu_gauss<M>(ga, gb, cda[c], cdb[c], nu);
+                const ulonglong2 cc = *reinterpret_cast<const ulonglong2*>(cpl + c * LW);
+                s3_nu_gauss<M>(ga, gb, cc.x, cc.y, nu);
                 s3_element(nu, eA, slo, w0, txy, txz, tyz, txyz, iso, kx, ky, kz, r);
-                if (c == NX - 1) { r[0] *= g3; r[2] *= g3; r[4] *= g3; r[6] *= g3; }
-                tl0[c] = r[0] + p100; tl1[c] = r[2] + p110; tu0[c] = r[4] + p101; tu1[c] = r[6] + p111;
-                p100 = r[1]; p110 = r[3]; p101 = r[5]; p111 = r[7];
-            }
-            // the last element of the lane on the left feeds this lane's first column
-            {
-                const float a100 = __shfl_up_sync(submask, p100, 1, LW), a110 = __shfl_up_sync(submask, p110, 1, LW);
-                const float a101 = __shfl_up_sync(submask, p101, 1, LW), a111 = __shfl_up_sync(submask, p111, 1, LW);
-                tl0[0] = fmaf(a100, lm, tl0[0]); tl1[0] = fmaf(a110, lm, tl1[0]);
-                tu0[0] = fmaf(a101, lm, tu0[0]); tu1[0] = fmaf(a111, lm, tu1[0]);
-            }
-            float o[NX];
-            // ---- node row (j, k): complete now
-            if (ownlo) {
-                float raw[NX];
-#pragma unroll
-                for (int c = 0; c < NX; ++c) raw[c] = (tl0[c] + pendL1[c]) + cin[c];
-                finish(raw, uA, -gs * fw * wy * wzlo, wy * wzlo, o);
-                if (act) st4(rlo, o);
-            }
-            // ---- node row (j, k + 1): parked until the next plane, or complete if that plane is the top of the domain
-            {
-                float part[NX];
-#pragma unroll
-                for (int c = 0; c < NX; ++c) { part[c] = tu0[c] + pendU1[c]; pendL1[c] = tl1[c]; pendU1[c] = tu1[c]; }
-                if (uptop) {
-                    finish(part, uC, -gs * fw * wy * 0.5f, wy * 0.5f, o);
-                    if (act) st4(rup, o);
-                } else if (storeup && act) {
-                    st4(rup, part);
+                if (c == NX - 1) {
+                    // the lane's last element: its right-hand corners belong to the next lane; in the lane that ends the
+                    // row it does not exist (g3 = 0)
+                    a100 = __shfl_up_sync(submask, r[1], 1, LW); a110 = __shfl_up_sync(submask, r[3], 1, LW);
+                    a101 = __shfl_up_sync(submask, r[5], 1, LW); a111 = __shfl_up_sync(submask, r[7], 1, LW);
+                    q000 = r[0] * g3; q010 = r[2] * g3; q001 = r[4] * g3; q011 = r[6] * g3;
+                } else {
+                    node(c + 1, q000 + r[1], q010 + r[3], q001 + r[5], q011 + r[7]);
+                    q000 = r[0]; q010 = r[2]; q001 = r[4]; q011 = r[6];
                 }
             }
-            sA = sB; ++n;
+            node(0, fmaf(a100, lm, q000), fmaf(a110, lm, q010), fmaf(a101, lm, q001), fmaf(a111, lm, q011));
+            if (hasf) {
+                float a = wx0 * uA[0];
+#pragma unroll
+                for (int c = 1; c < NX - 1; ++c) a += uA[c];
+                ello = fmaf(wy, fmaf(wxL, uA[NX - 1], a), ello);
+            }
+            if (ownlo && act) st4(rlo, olo);
+            if (storeup) st4(rlo + plane, oup);
+            rlo += nx;
+            oA = oB; ++n;
         }
         // ---- the top node row e1 of the tile gets nothing more in this plane.  It is this tile's own if it is the
         // top of the domain; else it belongs to the next tile and its sums go to the seam array (no load term: the
         // owner adds it).
         {
-            const int sU = wrap(sA + T);
-            float uT[NX + 1], uTu[NX + 1];
-            ldrow(ring + (size_t)sA * RS, uT); ldrow(ring + (size_t)sU * RS, uTu);
-            float* plo = lasttile ? rb + ((size_t)k * ny + e1) * nx : sb + (size_t)k * nx;
+            float uA[NX + 1];
+            ldrow(oA, uA);
+            float* plo = lasttile ? rlo : sb + (size_t)k * nx;
             float* pup = lasttile ? plo + plane : plo + nx;
-            const float wyT = lasttile ? 0.5f : 0.f;
-            float o[NX];
-            if (ownlo) {
-                float cin[NX], raw[NX];
+            const float wy = lasttile ? 0.5f : 0.f;
+            const float nlrow = nllo * wy;
+            float cin[NX], olo[NX];
 #pragma unroll
-                for (int c = 0; c < NX; ++c) cin[c] = 0.f;
-                if (hascarry && act) ld4(plo, cin);
+            for (int c = 0; c < NX; ++c) cin[c] = 0.f;
+            if (hascarry) ld4(plo, cin);
 #pragma unroll
-                for (int c = 0; c < NX; ++c) raw[c] = pendL1[c] + cin[c];
-                finish(raw, uT, -gs * fw * wyT * wzlo, wyT * wzlo, o);
-                if (act) st4(plo, o);
+            for (int c = 0; c < NX; ++c) {
+                const float raw = pendL1[c] + cin[c];
+                enlo = fmaf(uA[c], raw, enlo);
+                const float s = (c == 0) ? sc0 : (c == NX - 1) ? scL : sc;
+                const float l = (c == 0) ? lw0 * nlrow : (c == NX - 1) ? lwL * nlrow : nlrow;
+                olo[c] = fmaf(s, raw, l);
             }
-            if (uptop) {
-                finish(pendU1, uTu, -gs * fw * wyT * 0.5f, wyT * 0.5f, o);
-                if (act) st4(pup, o);
-            } else if (storeup && act) {
-                st4(pup, pendU1);
+            if (hasf) {
+                float a = wx0 * uA[0];
+#pragma unroll
+                for (int c = 1; c < NX - 1; ++c) a += uA[c];
+                ello = fmaf(wy, fmaf(wxL, uA[NX - 1], a), ello);
             }
-            sA = wrap(sA + 1); ++n;
+            if (ownlo && act) st4(plo, olo);
+            if (storeup) st4(pup, pendU1);
+            oA = wrapb(oA + RSB); ++n;
         }
-        end += (double)en; eld += (double)ell;          // per-plane sums go to double
-        en = 0.f; ell = 0.f;
+        // per-plane sums go to double; a plane counts where it is finished
+        if (ownlo) { end += (double)enlo; eld += (double)(wzlo * ello); }
     }
     s3_wait<0>();
+
+    // ---- the top node plane of the domain has no element plane above it: what was parked there is complete.  Its
+    // rows are still in the ring (entry n is row 0 of that plane).
+    if (lastchunk) {
+        float entop = 0.f, eltop = 0.f;
+        float* rtop = rb + ((size_t)ke * ny + y0) * nx;
+        for (int jj = 0; jj < T; ++jj) {
+            const bool seamrow = (jj == T - 1) && !lasttile;
+            float* p = seamrow ? sb + (size_t)ke * nx : rtop;
+            const int j = y0 + jj;
+            const float wy = seamrow ? 0.f : (j == 0 || j == ny - 1) ? 0.5f : 1.f;
+            const float nlrow = -gs * fw * 0.5f * wy;
+            float part[NX], uT[NX + 1], o[NX];
+#pragma unroll
+            for (int c = 0; c < NX; ++c) part[c] = 0.f;
+            if (act) ld4(p, part);
+            ldrow(oA, uT);
+#pragma unroll
+            for (int c = 0; c < NX; ++c) {
+                entop = fmaf(uT[c], part[c], entop);
+                const float s = (c == 0) ? sc0 : (c == NX - 1) ? scL : sc;
+                const float l = (c == 0) ? lw0 * nlrow : (c == NX - 1) ? lwL * nlrow : nlrow;
+                o[c] = fmaf(s, part[c], l);
+            }
+            float a = wx0 * uT[0];
+#pragma unroll
+            for (int c = 1; c < NX - 1; ++c) a += uT[c];
+            eltop = fmaf(wy, fmaf(wxL, uT[NX - 1], a), eltop);
+            if (act) st4(p, o);
+            rtop += nx;
+            oA = wrapb(oA + RSB);
+        }
+        end += (double)entop; eld += (double)(0.5f * eltop);
+    }
 
     // ---- energy partial of this unit: its lanes summed in a fixed order in double
     double d = act ? 0.5 * (double)kap * end : 0.0, l = (act && hasf) ? (double)fw * eld : 0.0;
@@ -438,53 +480,60 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
 // Coefficient table: for element row ey of element plane ez of sample b, the polynomials (in c = cos(pi x)) of
 // the KL exponent along the four Gauss lines (y_q, z_s):  sum_i g_i T_i(c)  with
 // g_i = sum_{j,k} ckl[i][j][k] cos(j pi y_q) cos(k pi z_s), converted from the Chebyshev basis to monomials in
-// double.  The scaled weights and the cosines are the float tables every kernel family reads.  One thread per line.
+// double.  The scaled weights and the cosines are the float tables every kernel family reads.  One block per
+// (sample, element plane, 128 element rows); a thread writes the four lines of its element row.
 // ---------------------------------------------------------------------------------------------------------
-__global__ void linepoly3d_kernel(const Params P, float* __restrict__ out, const int gs, const long long nlines) {
-    constexpr int MX = DN_MAX_KL_MODES;
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= nlines) return;
-    const int m = P.m;
-    const int s = (int)(idx & 1), q = (int)((idx >> 1) & 1);
-    const long long row = idx >> 2;                                     // (b * (nz-1) + ez) * (ny-1) + ey
-    const int ey = (int)(row % (P.ny - 1));
-    const int ez = (int)((row / (P.ny - 1)) % (P.nz - 1));
-    const long long b = row / ((long long)(P.ny - 1) * (P.nz - 1));
-    const float* cy = P.cg[1] + 2 * ey + q;
-    const float* cz = P.cg[2] + 2 * ez + s;
-    const float* w = P.ckl + b * m * m * m;
-    double g[MX];
-#pragma unroll
-    for (int i = 0; i < MX; ++i) {
+template <int M>
+__global__ void __launch_bounds__(128) linepoly3d_kernel(const Params P, float* __restrict__ out) {
+    constexpr int GS = s3_gs(M);
+    __shared__ double h[2][M][M];                       // h[s][i][j] = sum_k ckl[i][j][k] cos(k pi z_s)
+    const int ez = blockIdx.y, b = blockIdx.z;
+    const float* w = P.ckl + (size_t)b * M * M * M;
+    for (int t = threadIdx.x; t < 2 * M * M; t += blockDim.x) {
+        const int s = t / (M * M), ij = t % (M * M);
+        const float* cz = P.cg[2] + 2 * ez + s;
         double acc = 0.0;
-        if (i < m) {
-            for (int j = 0; j < m; ++j) {
-                double inner = 0.0;
-                for (int k = 0; k < m; ++k) inner += (double)w[(i * m + j) * m + k] * (double)cz[(size_t)k * P.gstride[2]];
-                acc += inner * (double)cy[(size_t)j * P.gstride[1]];
+#pragma unroll
+        for (int k = 0; k < M; ++k) acc += (double)w[ij * M + k] * (double)cz[(size_t)k * P.gstride[2]];
+        h[s][ij / M][ij % M] = acc;
+    }
+    __syncthreads();
+    const int ey = blockIdx.x * blockDim.x + threadIdx.x;
+    if (ey >= P.ny - 1) return;
+    float row[2 * GS];
+#pragma unroll
+    for (int i = 0; i < 2 * GS; ++i) row[i] = 0.f;      // the padding of a Gauss row stays zero
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        double cy[M];
+#pragma unroll
+        for (int j = 0; j < M; ++j) cy[j] = (double)P.cg[1][(size_t)j * P.gstride[1] + 2 * ey + q];
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            // sum_i g_i T_i(c) in the monomial basis, T_{i+1} = 2 c T_i - T_{i-1}
+            double acc[M + 1], tp[M + 1], tc[M + 1];
+#pragma unroll
+            for (int k = 0; k <= M; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
+#pragma unroll
+            for (int i = 1; i <= M; ++i) {
+                double g = 0.0;
+#pragma unroll
+                for (int j = 0; j < M; ++j) g += h[s][i - 1][j] * cy[j];
+#pragma unroll
+                for (int k = 0; k <= i; ++k) acc[k] += g * tc[k];
+                double tn[M + 1];
+#pragma unroll
+                for (int k = 0; k <= M; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
+#pragma unroll
+                for (int k = 0; k <= M; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
             }
+#pragma unroll
+            for (int k = 0; k <= M; ++k) row[q * GS + 2 * k + s] = (float)acc[k];
         }
-        g[i] = acc;
     }
-    // sum_i g_i T_i(c) in the monomial basis, T_{i+1} = 2 c T_i - T_{i-1}
-    double acc[MX + 1], tp[MX + 1], tc[MX + 1];
+    float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * (P.nz - 1) + ez) * (P.ny - 1) + ey) * (2 * GS));
 #pragma unroll
-    for (int k = 0; k <= MX; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
-#pragma unroll
-    for (int i = 1; i <= MX; ++i) {
-        if (i > m) break;                              // uniform; the remaining terms are zero
-#pragma unroll
-        for (int k = 0; k <= MX; ++k) acc[k] += g[i - 1] * tc[k];
-        double tn[MX + 1];
-#pragma unroll
-        for (int k = 0; k <= MX; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
-#pragma unroll
-        for (int k = 0; k <= MX; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
-    }
-    float* dst = out + row * (2 * gs) + q * gs + s;
-#pragma unroll
-    for (int i = 0; i < s3_gs(MX) / 2; ++i)            // coefficient i of plane s; the padding of the row is zero
-        if (2 * i + s < gs) dst[2 * i] = (i <= m) ? (float)acc[i <= MX ? i : MX] : 0.f;
+    for (int i = 0; i < GS / 2; ++i) dst[i] = make_float4(row[4 * i], row[4 * i + 1], row[4 * i + 2], row[4 * i + 3]);
 }
 
 int s3_sm_count() {
@@ -500,7 +549,8 @@ constexpr size_t S3_SMEM_SM = 233472;              // shared memory of an SM; a 
 constexpr size_t S3_SMEM_BLOCK = 232448;           // most a block can ask for
 
 int s3_nxl(int nx) { return (nx > 128) ? 8 : 4; }  // nodes per lane
-int s3_minb(int nxl) { return (nxl == 8) ? 3 : 4; } // resident blocks of 4 warps per SM the kernel is compiled for
+int s3_env(const char* n, int d) { const char* e = getenv(n); return e ? atoi(e) : d; }   // EXPERIMENT
+int s3_minb(int nxl) { return s3_env("DN_S3_MINB", (nxl == 8) ? 3 : 4); } // resident blocks of 4 warps per SM the kernel is compiled for
 
 S3Geo geometry3s(const dn_problem& p) {
     S3Geo g{};
@@ -513,6 +563,7 @@ S3Geo geometry3s(const dn_problem& p) {
     g.RS = NX * g.LW + 4 + 2 * s3_gs(m);
     size_t per_block = (S3_SMEM_SM - (size_t)minb * 1024) / minb;
     if (per_block > S3_SMEM_BLOCK) per_block = S3_SMEM_BLOCK;
+    per_block -= sizeof(float) * 4 * NX * g.LW;      // the block's table of cosine pairs
     const int cmax = (int)(per_block / ((size_t)S3_WARPS * subs * g.RS * sizeof(float)));
     int ry_max = cmax - 2 - S3_D;
     if (ry_max > ny - 1) ry_max = ny - 1;
@@ -535,6 +586,10 @@ S3Geo geometry3s(const dn_problem& p) {
             }
         }
     }
+    if (getenv("DN_S3_RY")) {   // EXPERIMENT
+        g.Ry = atoi(getenv("DN_S3_RY")); g.Z = s3_env("DN_S3_Z", g.Z);
+        g.ntile = (ny - 1 + g.Ry - 1) / g.Ry; g.nchunk = (nz - 1 + g.Z - 1) / g.Z; g.units = (long long)p.batch * g.ntile * g.nchunk;
+    }
     g.C = g.Ry + 2 + S3_D;
     return g;
 }
@@ -542,7 +597,7 @@ S3Geo geometry3s(const dn_problem& p) {
 template <int NX, int M, int MINB>
 cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
     const int subs = 32 / g.LW;
-    const size_t smem = sizeof(float) * (size_t)S3_WARPS * subs * g.C * g.RS;
+    const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * g.C * g.RS + 4 * NX * g.LW);
     const long long per_block = (long long)S3_WARPS * subs;
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
     const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -553,6 +608,11 @@ cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cu
 
 template <int M>
 cudaError_t launch_m3(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+    if (M == 3 && s3_nxl(P.nx) == 8) {   // EXPERIMENT
+        const int mb = s3_minb(8);
+        if (mb == 2) return launch_nm<8, 3, 2>(P, linepoly, g, s);
+        if (mb == 4) return launch_nm<8, 3, 4>(P, linepoly, g, s);
+    }
     return (s3_nxl(P.nx) == 8) ? launch_nm<8, M, 3>(P, linepoly, g, s) : launch_nm<4, M, 4>(P, linepoly, g, s);
 }
 
@@ -595,10 +655,25 @@ size_t strip3d_linepoly_floats(const dn_problem& p) {
     return (size_t)p.batch * (p.grid.nz - 1) * (p.grid.ny - 1) * 2 * s3_gs(p.kl_modes);
 }
 
-cudaError_t launch_linepoly3d(const Params& P, float* linepoly, cudaStream_t s) {
-    const long long nlines = 4ll * P.batch * (P.nz - 1) * (P.ny - 1);
-    linepoly3d_kernel<<<(unsigned)((nlines + 127) / 128), 128, 0, s>>>(P, linepoly, s3_gs(P.m), nlines);
+template <int M>
+static cudaError_t launch_linepoly3d_m(const Params& P, float* linepoly, cudaStream_t s) {
+    const dim3 grid((unsigned)((P.ny - 1 + 127) / 128), (unsigned)(P.nz - 1), (unsigned)P.batch);
+    linepoly3d_kernel<M><<<grid, 128, 0, s>>>(P, linepoly);
     return cudaGetLastError();
+}
+
+cudaError_t launch_linepoly3d(const Params& P, float* linepoly, cudaStream_t s) {
+    switch (P.m) {
+        case 1: return launch_linepoly3d_m<1>(P, linepoly, s);
+        case 2: return launch_linepoly3d_m<2>(P, linepoly, s);
+        case 3: return launch_linepoly3d_m<3>(P, linepoly, s);
+        case 4: return launch_linepoly3d_m<4>(P, linepoly, s);
+        case 5: return launch_linepoly3d_m<5>(P, linepoly, s);
+        case 6: return launch_linepoly3d_m<6>(P, linepoly, s);
+        case 7: return launch_linepoly3d_m<7>(P, linepoly, s);
+        case 8: return launch_linepoly3d_m<8>(P, linepoly, s);
+    }
+    return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t s) {
