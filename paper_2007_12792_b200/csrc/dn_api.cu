@@ -95,8 +95,13 @@ WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
     }
     w.rowpoly = off;
     if ((tight ? l.path == PATH_STRIP2D : strip2d_applicable(p))) off += align_up(sizeof(float) * strip2d_rowpoly_floats(p) + 16);
+    w.zseam = off;
     w.linepoly = off;
-    if ((tight ? l.path == PATH_STRIP3D : strip3d_applicable(p))) off += align_up(sizeof(float) * strip3d_linepoly_floats(p) + 16);
+    if ((tight ? l.path == PATH_STRIP3D : strip3d_applicable(p))) {
+        off += align_up(sizeof(float) * strip3d_zseam_floats(p) + 16);
+        w.linepoly = off;
+        off += align_up(sizeof(float) * strip3d_linepoly_floats(p) + 16);
+    }
     w.total = off;
     return w;
 }
@@ -117,6 +122,7 @@ static Params make_params(const dn_problem& p, const WsLayout& w, const float* u
     for (int a = 0; a < 3; ++a) { P.cn[a] = reinterpret_cast<const float*>(base + w.cn[a]); P.nstride[a] = w.nstride[a]; }
     P.nblk = w.nblk;
     P.seam = reinterpret_cast<float*>(base + w.seam);
+    P.zseam = reinterpret_cast<float*>(base + w.zseam);
     P.nodes = nodes_per_sample(p.grid);
     return P;
 }
@@ -162,6 +168,10 @@ static dn_status plan(const dn_problem* p, const float* u, const float* r, size_
             l.path = PATH_GENERIC;
             l.nblk = generic_blocks_per_sample(nodes_per_sample(p->grid));
         }
+        w = make_layout(*p, l, tight);
+    }
+    if (tight && l.path == PATH_STRIP3D && ws_bytes < w.total && tiled3d_applicable(*p)) {
+        l = tiled3d_geometry(*p);                       // smaller scratch: no coefficient table, one kind of seam
         w = make_layout(*p, l, tight);
     }
     return (ws_bytes < w.total) ? DN_ERR_WORKSPACE : DN_OK;
@@ -408,7 +418,7 @@ int32_t dn_launches_per_call(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
     const bool fast = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr;
     if (fast && strip3d_applicable(*p))                 // tables, line polynomials, fused kernel, seam fix-up, finaliser
-        return 4 + (strip3d_seam_floats(*p) > 0 ? 1 : 0);
+        return 4 + ((strip3d_seam_floats(*p) + strip3d_zseam_floats(*p)) > 0 ? 1 : 0);
     const bool t3 = fast && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
     return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
 }

@@ -29,6 +29,7 @@ struct WsLayout {
     size_t cn[3];         // float  [m][nstride[a]] cos(i pi x) at the nodes of axis a
     int nstride[3];
     size_t rowpoly;       // float  [B][ny-1][GS] polynomial of the KL exponent along every Gauss row (strip 2D kernel)
+    size_t zseam;         // float  contributions across the chunk seams of the strip 3D kernel
     size_t linepoly;      // float  [B][nz-1][ny-1][2 GS] the same along the four Gauss lines of every element row (strip 3D kernel)
     int nblk;             // energy partials per sample
     size_t total;
@@ -58,6 +59,7 @@ struct Params {
     long long nodes;      // per sample
     float* seam;          // tiled 3D: contributions of a tile's top element row to the next tile's first node row
     int nseam;
+    float* zseam;         // strip 3D: contributions of a chunk's last element plane to the next chunk's first node plane
 };
 
 struct Launch {           // tiled-path launch geometry chosen on the host
@@ -114,6 +116,7 @@ cudaError_t launch_seam_fixup(float* r, const float* seam, int nx, int ny, int n
 bool strip3d_applicable(const dn_problem& p);      // fused energy+residual, KL at the Gauss points, 3D rows of at most 256 nodes
 Launch strip3d_geometry(const dn_problem& p);
 size_t strip3d_seam_floats(const dn_problem& p);
+size_t strip3d_zseam_floats(const dn_problem& p);
 size_t strip3d_linepoly_floats(const dn_problem& p);
 cudaError_t launch_linepoly3d(const Params& P, float* linepoly, cudaStream_t s);   // after launch_tables (reads ckl, cg)
 cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t s);

@@ -23,9 +23,10 @@
 //
 // Tiles do not overlap in y: the top element row of a tile leaves what it contributes to the first node row of
 // the next tile in a scratch array (seam, [B][ntile-1][nz][nx]), parked there between planes in the same way, and
-// the small fix-up kernel of the tiled 3D path adds those rows to r afterwards in a fixed order.  Chunks overlap by
-// one element plane in z: a chunk recomputes the last element plane of the chunk below for the sake of its
-// contributions to the chunk's first node plane (1 / Z more work).  No atomics; every sum has a fixed order.
+// a small fix-up kernel adds those rows to r afterwards.  Chunks do not overlap in z either: what the last element
+// plane of a chunk contributes to the first node plane of the next chunk goes to a second scratch array (zseam,
+// [B][nchunk-1][ny][nx], plus [B][nchunk-1][ntile-1][nx] for the nodes that are on a tile seam as well), added by the
+// same fix-up kernel.  Every element is computed exactly once.  No atomics; every sum has a fixed order.
 //
 // Arithmetic of one element: hierarchical coordinates of the trilinear field (edge differences e, s, w at the low
 // corner, second differences txy, txz, tyz, third difference txyz), derivatives at the 4 Gauss lines of each
@@ -147,22 +148,20 @@ __device__ __forceinline__ void s3_element(const float (&n)[8], const float e0, 
     const float Gx_aa = Nx_aa * Dx_aa, Gx_ab = Nx_ab * Dx_ab, Gx_ba = Nx_ba * Dx_ba, Gx_bb = Nx_bb * Dx_bb;
     const float Gy_aa = Ny_aa * Dy_aa, Gy_ab = Ny_ab * Dy_ab, Gy_ba = Ny_ba * Dy_ba, Gy_bb = Ny_bb * Dy_bb;
     const float Gz_aa = Nz_aa * Dz_aa, Gz_ab = Nz_ab * Dz_ab, Gz_ba = Nz_ba * Dz_ba, Gz_bb = Nz_bb * Dz_bb;
-    // adjoint of the three interpolations: partial derivatives of the element energy
-    const float AXa = Gx_aa + Gx_ab, AXb = Gx_ba + Gx_bb;
-    const float BXa = fmaf(bq, Gx_ab, a * Gx_aa), BXb = fmaf(bq, Gx_bb, a * Gx_ba);
-    const float AYa = Gy_aa + Gy_ab, AYb = Gy_ba + Gy_bb;
-    const float BYa = fmaf(bq, Gy_ab, a * Gy_aa), BYb = fmaf(bq, Gy_bb, a * Gy_ba);
-    const float AZa = Gz_aa + Gz_ab, AZb = Gz_ba + Gz_bb;
-    const float BZa = fmaf(bq, Gz_ab, a * Gz_aa), BZb = fmaf(bq, Gz_bb, a * Gz_ba);
-    const float dE = AXa + AXb, dS = AYa + AYb, dW = AZa + AZb;
-    float dXY = fmaf(bq, AXb, a * AXa);
-    dXY = fmaf(a, AYa, dXY); dXY = fmaf(bq, AYb, dXY);
-    float dXZ = BXa + BXb;
-    dXZ = fmaf(a, AZa, dXZ); dXZ = fmaf(bq, AZb, dXZ);
-    const float dYZ = (BYa + BYb) + (BZa + BZb);
-    float dXYZ = fmaf(bq, BXb, a * BXa);
-    dXYZ = fmaf(a, BYa, dXYZ); dXYZ = fmaf(bq, BYb, dXYZ);
-    dXYZ = fmaf(a, BZa, dXYZ); dXYZ = fmaf(bq, BZb, dXYZ);
+    // Adjoint of the three interpolations: partial derivatives of the element energy.  With b = a + dl the weighted
+    // sums over a 2 x 2 set of Gauss lines reduce to its total S, the sum R over the lines whose first index is b, the
+    // sum C over those whose second index is b, and the (b, b) entry:
+    //   sum i1 G = a S + dl R,   sum i2 G = a S + dl C,   sum i1 i2 G = a^2 S + a dl (R + C) + dl^2 G_bb.
+    constexpr float dl = DN_GB - DN_GA;
+    const float R1x = Gx_ba + Gx_bb, Cx = Gx_ab + Gx_bb, dE = (Gx_aa + Gx_ab) + R1x;     // Gx[q][s]
+    const float R1y = Gy_ba + Gy_bb, Cy = Gy_ab + Gy_bb, dS = (Gy_aa + Gy_ab) + R1y;     // Gy[p][s]
+    const float R1z = Gz_ba + Gz_bb, Cz = Gz_ab + Gz_bb, dW = (Gz_aa + Gz_ab) + R1z;     // Gz[p][q]
+    const float Sxy = dE + dS, Sxz = dE + dW, Syz = dS + dW;
+    const float P1 = R1x + R1y, P2 = Cx + R1z, P3 = Cy + Cz;
+    const float dXY = fmaf(dl, P1, a * Sxy);           // txy enters d/dx through q and d/dy through p
+    const float dXZ = fmaf(dl, P2, a * Sxz);           // txz enters d/dx through s and d/dz through p
+    const float dYZ = fmaf(dl, P3, a * Syz);           // tyz enters d/dy through s and d/dz through q
+    const float dXYZ = fmaf(dl * dl, (Gx_bb + Gy_bb) + Gz_bb, fmaf(a * dl, (P1 + P2) + P3, (a * a) * (Sxy + dW)));
     // chain rule to the corners
     const float r110 = dXY - dXYZ, r101 = dXZ - dXYZ, r011 = dYZ - dXYZ;
     const float r100 = (dE - r110) - dXZ, r010 = (dS - r110) - dYZ, r001 = (dW - r101) - dYZ;
@@ -214,15 +213,23 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const int T = e1 - y0 + 1;
     const bool lasttile = (e1 == ny - 1);               // then node row e1 = ny-1 is this tile's own, else the next tile's
     const int z0 = chunk * G.Z, ke = min(z0 + G.Z, nz - 1);
-    const int kbeg = max(z0 - 1, 0);                    // element planes kbeg .. ke-1 (kbeg = z0-1: the recomputed one)
-    const int nplanes = ke - kbeg + 1;                  // node planes kbeg .. ke
-    const bool lastchunk = (ke == nz - 1);              // then node plane ke = nz-1 is this chunk's own
+    const int kbeg = z0;                                // element planes z0 .. ke-1
+    const int nplanes = ke - kbeg + 1;                  // node planes z0 .. ke
+    const bool lastchunk = (ke == nz - 1);              // then node plane ke = nz-1 is this chunk's own, else the next chunk's
 
     const bool first_col = (x0 == 0), last_col = act && (x0 + NX == nx);
     const size_t plane = (size_t)nx * ny;
     const float* ub = P.u + (size_t)b * P.nodes + x0c;
     float* rb = P.r + (size_t)b * P.nodes + x0c;
     float* sb = lasttile ? nullptr : P.seam + (((size_t)b * (G.ntile - 1) + tile) * nz) * nx + x0c;
+    // where the sums of node plane ke go: r, or for a chunk below another the z seam (row y0 of it; and the entry of
+    // this tile's seam row among the nodes that lie on both seams)
+    float* ztop = lastchunk ? rb + ((size_t)ke * ny + y0) * nx
+                            : P.zseam + (((size_t)b * (G.nchunk - 1) + chunk) * ny + y0) * nx + x0c;
+    float* zstop = lasttile ? nullptr
+                 : lastchunk ? sb + (size_t)ke * nx
+                             : P.zseam + (size_t)P.batch * (G.nchunk - 1) * ny * nx
+                               + (((size_t)b * (G.nchunk - 1) + chunk) * (G.ntile - 1) + tile) * nx + x0c;
 
     const bool impose = (P.flags & DN_IMPOSE_BC_ON_LOAD) != 0;
     const bool nomask = (P.flags & DN_NO_MASK) != 0;
@@ -311,18 +318,16 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     int n = 0;                                          // ... and its entry index
     const unsigned TB = (unsigned)T * RSB;
     for (int kk = 0; kk + 1 < nplanes; ++kk) {
-        const int k = kbeg + kk;                        // element plane k lies between node planes k and k + 1
-        const bool ownlo = (k >= z0);                   // node plane k is finished here (not so in the recomputed plane)
-        const bool hascarry = ownlo && (kk > 0) && act; // ... and has partial sums parked from the step before
-        // the sums of node plane k + 1 are parked; not so if that plane belongs to the next chunk, which recomputes
-        // them (the top plane of the domain is this chunk's own: it is finished after the march)
-        const bool storeup = ((k + 1 < ke) || lastchunk) && act;
+        const int k = kbeg + kk;                        // element plane k lies between node planes k and k + 1: plane k is
+        const bool hascarry = (kk > 0) && act;          // finished now, with the partial sums parked one step before;
+        const bool last = (k + 1 == ke);                // the sums of plane k + 1 are parked (plane ke: finished after the march)
         const float wzlo = (k == 0) ? 0.5f : 1.f;
         const float nllo = -gs * fw * wzlo;
         float enlo = 0.f, ello = 0.f;
 #pragma unroll
         for (int c = 0; c < NX; ++c) { pendL1[c] = 0.f; pendU1[c] = 0.f; }
         float* rlo = rb + ((size_t)k * ny + y0) * nx;
+        float* rup = last ? ztop : rlo + plane;
         for (int jj = 0; jj + 1 < T; ++jj) {
             s3_wait<0>();                               // everything issued up to the previous step has landed ...
             __syncwarp(submask);                        // ... is visible to the unit, and the rows it retired are free
@@ -388,9 +393,8 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                 for (int c = 1; c < NX - 1; ++c) a += uA[c];
                 ello = fmaf(wy, fmaf(wxL, uA[NX - 1], a), ello);
             }
-            if (ownlo && act) st4(rlo, olo);
-            if (storeup) st4(rlo + plane, oup);
-            rlo += nx;
+            if (act) { st4(rlo, olo); st4(rup, oup); }
+            rlo += nx; rup += nx;
             oA = oB; ++n;
         }
         // ---- the top node row e1 of the tile gets nothing more in this plane.  It is this tile's own if it is the
@@ -400,7 +404,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
             float uA[NX + 1];
             ldrow(oA, uA);
             float* plo = lasttile ? rlo : sb + (size_t)k * nx;
-            float* pup = lasttile ? plo + plane : plo + nx;
+            float* pup = lasttile ? rup : last ? zstop : plo + nx;
             const float wy = lasttile ? 0.5f : 0.f;
             const float nlrow = nllo * wy;
             float cin[NX], olo[NX];
@@ -421,25 +425,25 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                 for (int c = 1; c < NX - 1; ++c) a += uA[c];
                 ello = fmaf(wy, fmaf(wxL, uA[NX - 1], a), ello);
             }
-            if (ownlo && act) st4(plo, olo);
-            if (storeup) st4(pup, pendU1);
+            if (act) { st4(plo, olo); st4(pup, pendU1); }
             oA = wrapb(oA + RSB); ++n;
         }
-        // per-plane sums go to double; a plane counts where it is finished
-        if (ownlo) { end += (double)enlo; eld += (double)(wzlo * ello); }
+        end += (double)enlo; eld += (double)(wzlo * ello);   // per-plane sums go to double
     }
     s3_wait<0>();
 
-    // ---- the top node plane of the domain has no element plane above it: what was parked there is complete.  Its
-    // rows are still in the ring (entry n is row 0 of that plane).
-    if (lastchunk) {
+    // ---- node plane ke gets nothing more from this chunk: what was parked for it is complete as far as this chunk
+    // goes.  Top of the domain: finished into r with its load.  Else the plane is the next chunk's: the scaled, masked
+    // sums stay in the z seam (no load term: the owner adds it).  Its rows are still in the ring (entry n is row 0).
+    {
         float entop = 0.f, eltop = 0.f;
-        float* rtop = rb + ((size_t)ke * ny + y0) * nx;
+        const float lf = lastchunk ? 1.f : 0.f;
+        float* ptop = ztop;
         for (int jj = 0; jj < T; ++jj) {
             const bool seamrow = (jj == T - 1) && !lasttile;
-            float* p = seamrow ? sb + (size_t)ke * nx : rtop;
+            float* p = seamrow ? zstop : ptop;
             const int j = y0 + jj;
-            const float wy = seamrow ? 0.f : (j == 0 || j == ny - 1) ? 0.5f : 1.f;
+            const float wy = seamrow ? 0.f : (j == 0 || j == ny - 1) ? 0.5f * lf : lf;
             const float nlrow = -gs * fw * 0.5f * wy;
             float part[NX], uT[NX + 1], o[NX];
 #pragma unroll
@@ -458,7 +462,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
             for (int c = 1; c < NX - 1; ++c) a += uT[c];
             eltop = fmaf(wy, fmaf(wxL, uT[NX - 1], a), eltop);
             if (act) st4(p, o);
-            rtop += nx;
+            ptop += nx;
             oA = wrapb(oA + RSB);
         }
         end += (double)entop; eld += (double)(0.5f * eltop);
@@ -536,6 +540,51 @@ __global__ void __launch_bounds__(128) linepoly3d_kernel(const Params P, float* 
     for (int i = 0; i < GS / 2; ++i) dst[i] = make_float4(row[4 * i], row[4 * i + 1], row[4 * i + 2], row[4 * i + 3]);
 }
 
+// Adds the seam contributions to r (fixed order per node: own sums, tile seam, chunk seam, the entry for nodes on both).
+// First range of threads: the nodes of the tile seam rows (t + 1) Ry on every plane; second range: the nodes of the
+// chunk seam planes (c + 1) Z that are not on a tile seam row.  The two ranges touch different nodes.
+__global__ void seam_fixup3_kernel(float* __restrict__ r, const float* __restrict__ yseam, const float* __restrict__ zseam,
+                                   int nx, int ny, int nz, int batch, int Ry, int ntile, int Z, int nchunk,
+                                   long long nA, long long nB) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int nx4 = nx / 4;
+    const float4* zy = reinterpret_cast<const float4*>(zseam + (size_t)batch * (nchunk - 1) * ny * nx);
+    if (i < nA) {
+        const int x4 = (int)(i % nx4);
+        long long t = i / nx4;
+        const int k = (int)(t % nz); t /= nz;
+        const int sm = (int)(t % (ntile - 1));
+        const int b = (int)(t / (ntile - 1));
+        const int j = (sm + 1) * Ry;
+        float4* dst = reinterpret_cast<float4*>(r + (((size_t)b * nz + k) * ny + j) * nx) + x4;
+        float4 v = *dst;
+        const float4 a = __ldg(reinterpret_cast<const float4*>(yseam) + i);
+        v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+        if (k % Z == 0 && k > 0 && k < nz - 1) {        // also the first plane of a chunk
+            const int c = k / Z - 1;
+            const float4 z = __ldg(reinterpret_cast<const float4*>(zseam + (((size_t)b * (nchunk - 1) + c) * ny + j) * nx) + x4);
+            v.x += z.x; v.y += z.y; v.z += z.z; v.w += z.w;
+            const float4 w = __ldg(zy + (((size_t)b * (nchunk - 1) + c) * (ntile - 1) + sm) * nx4 + x4);
+            v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+        }
+        *dst = v;
+    } else if (i < nA + nB) {
+        const long long q = i - nA;
+        const int x4 = (int)(q % nx4);
+        long long t = q / nx4;
+        const int j = (int)(t % ny); t /= ny;
+        const int c = (int)(t % (nchunk - 1));
+        const int b = (int)(t / (nchunk - 1));
+        if (j % Ry == 0 && j > 0 && j < ny - 1) return;  // a tile seam row: done by the first range
+        const int k = (c + 1) * Z;
+        float4* dst = reinterpret_cast<float4*>(r + (((size_t)b * nz + k) * ny + j) * nx) + x4;
+        float4 v = *dst;
+        const float4 z = __ldg(reinterpret_cast<const float4*>(zseam) + q);
+        v.x += z.x; v.y += z.y; v.z += z.z; v.w += z.w;
+        *dst = v;
+    }
+}
+
 int s3_sm_count() {
     int dev = 0, n = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
@@ -548,7 +597,8 @@ int s3_sm_count() {
 constexpr size_t S3_SMEM_SM = 233472;              // shared memory of an SM; a block also reserves 1 KiB
 constexpr size_t S3_SMEM_BLOCK = 232448;           // most a block can ask for
 
-int s3_nxl(int nx) { return (nx > 128) ? 8 : 4; }  // nodes per lane
+int s3_env(const char* n, int d);
+int s3_nxl(int nx) { if (nx > 128) return 8; return (nx % 8 == 0 && s3_env("DN_S3_NX", 4) == 8) ? 8 : 4; }  // nodes per lane
 int s3_env(const char* n, int d) { const char* e = getenv(n); return e ? atoi(e) : d; }   // EXPERIMENT
 int s3_minb(int nxl) { return s3_env("DN_S3_MINB", (nxl == 8) ? 3 : 4); } // resident blocks of 4 warps per SM the kernel is compiled for
 
@@ -570,8 +620,8 @@ S3Geo geometry3s(const dn_problem& p) {
     if (ry_max > 64) ry_max = 64;
     if (ry_max < 1) ry_max = 1;
     const long long slots = (long long)s3_sm_count() * minb * S3_WARPS * subs;
-    // (Ry, Z) by a cost model: whole waves of units; a unit pays one more plane (the recomputed one) and, per plane,
-    // the finish of its top row; flat tiles also pay the seam traffic and the fix-up pass.
+    // (Ry, Z) by a cost model: whole waves of units; a unit pays, per plane, the finish of its top row, and once the
+    // filling of its ring and the finish of its last plane; flat tiles and short chunks also pay seam traffic.
     double best = -1.0;
     for (int Ry = 1; Ry <= ry_max; ++Ry) {
         const long long ntile = (ny - 1 + Ry - 1) / Ry;
@@ -579,7 +629,7 @@ S3Geo geometry3s(const dn_problem& p) {
             const long long nchunk = (nz - 1 + Z - 1) / Z;
             const long long units = (long long)p.batch * ntile * nchunk;
             const long long waves = (units + slots - 1) / slots;
-            const double cost = (double)waves * (Z + 1) * (Ry + 0.8) * (1.0 + 0.25 / Ry);
+            const double cost = (double)waves * (Z * (Ry + 0.5) + 0.4 * Ry + 3.0) * (1.0 + 0.15 / Ry + 0.15 / Z);
             if (best < 0 || cost < best * (1.0 - 1e-9)) {
                 best = cost;
                 g.Ry = Ry; g.Z = Z; g.ntile = (int)ntile; g.nchunk = (int)nchunk; g.units = units;
@@ -650,6 +700,13 @@ size_t strip3d_seam_floats(const dn_problem& p) {
     return (size_t)p.batch * (g.ntile - 1) * p.grid.nz * p.grid.nx;
 }
 
+// the chunk seams: [B][nchunk-1][ny][nx], then [B][nchunk-1][ntile-1][nx] for the nodes on a tile seam as well
+size_t strip3d_zseam_floats(const dn_problem& p) {
+    if (!strip3d_applicable(p)) return 0;
+    const S3Geo g = geometry3s(p);
+    return (size_t)p.batch * (g.nchunk - 1) * ((size_t)p.grid.ny + (g.ntile - 1)) * p.grid.nx;
+}
+
 size_t strip3d_linepoly_floats(const dn_problem& p) {
     if (!strip3d_applicable(p)) return 0;
     return (size_t)p.batch * (p.grid.nz - 1) * (p.grid.ny - 1) * 2 * s3_gs(p.kl_modes);
@@ -690,7 +747,13 @@ cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t 
         case 8: e = launch_m3<8>(P, linepoly, g, s); break;
     }
     if (e != cudaSuccess) return e;
-    if (g.ntile > 1) return launch_seam_fixup(P.r, P.seam, P.nx, P.ny, P.nz, g.Ry, g.ntile - 1, P.batch, s);
+    const long long nA = (long long)P.batch * (g.ntile - 1) * P.nz * (P.nx / 4);
+    const long long nB = (long long)P.batch * (g.nchunk - 1) * P.ny * (P.nx / 4);
+    if (nA + nB > 0) {
+        seam_fixup3_kernel<<<(unsigned)((nA + nB + 255) / 256), 256, 0, s>>>(P.r, P.seam, P.zseam, P.nx, P.ny, P.nz, P.batch,
+                                                                            g.Ry, g.ntile, g.Z, g.nchunk, nA, nB);
+        return cudaGetLastError();
+    }
     return cudaSuccess;
 }
 
