@@ -417,8 +417,8 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
 int32_t dn_launches_per_call(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
     const bool fast = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr;
-    if (fast && strip3d_applicable(*p))                 // tables, line polynomials, fused kernel, seam fix-up, finaliser
-        return 4 + ((strip3d_seam_floats(*p) + strip3d_zseam_floats(*p)) > 0 ? 1 : 0);
+    if (fast && strip3d_applicable(*p))                 // (tables, line polynomials,) fused kernel, seam fix-up, finaliser
+        return 2 + (p->nu_mode != DN_NU_NODAL ? 2 : 0) + ((strip3d_seam_floats(*p) + strip3d_zseam_floats(*p)) > 0 ? 1 : 0);
     const bool t3 = fast && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
     return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
 }

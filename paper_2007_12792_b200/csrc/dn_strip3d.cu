@@ -40,7 +40,6 @@
 // element plane once per call in double ([B][nz-1][ny-1][2][GS] floats: Gauss row q, then coefficient i and Gauss
 // plane s interleaved for packed two-wide FMAs); they travel through the ring with the node row that completes
 // the element row.
-#include <cstdlib>
 #include "dn_internal.cuh"
 
 namespace dn {
@@ -120,17 +119,39 @@ __device__ __forceinline__ void s3_nu_gauss(const u64 (&ga)[s3_gs(M) / 2], const
     for (int i = 0; i < 8; ++i) n[i] = s3_ex2(x[i]);
 }
 
-// The element: from the 8 diffusivities n[4p + 2q + s] and the 7 hierarchical coordinates of u to the 8 corner
-// contributions r[i + 2j + 4k] (i, j, k the x, y, z bits of the corner), all in units of kap = hx hy hz / (8 h^2)
-// on isotropic cells (iso), else scaled by kx, ky, kz here.
-__device__ __forceinline__ void s3_element(const float (&n)[8], const float e0, const float s0, const float w0,
+// Sums of nu along each derivative's own axis, from nu at the 8 Gauss points n[4p + 2q + s]:
+// Nx[2q + s] = sum_p, Ny[2p + s] = sum_q, Nz[2p + q] = sum_s.
+__device__ __forceinline__ void s3_sums_gauss(const float (&n)[8], float (&Nx)[4], float (&Ny)[4], float (&Nz)[4]) {
+    Nx[0] = n[0] + n[4]; Nx[1] = n[1] + n[5]; Nx[2] = n[2] + n[6]; Nx[3] = n[3] + n[7];
+    Ny[0] = n[0] + n[2]; Ny[1] = n[1] + n[3]; Ny[2] = n[4] + n[6]; Ny[3] = n[5] + n[7];
+    Nz[0] = n[0] + n[1]; Nz[1] = n[2] + n[3]; Nz[2] = n[4] + n[5]; Nz[3] = n[6] + n[7];
+}
+
+// The same sums for a trilinear nu given at the corners.  Summing the interpolant over the two Gauss points of an axis
+// leaves the sum of the two corner values along that axis (the weights a and b add up to 1), interpolated in the other
+// two.  h00, h10, h01, h11: those edge sums at (first, second) other coordinate = low/high; out[2 i1 + i2] at the
+// Gauss abscissae (i1, i2) of the two other axes.
+__device__ __forceinline__ void s3_bilerp(const float h00, const float h10, const float h01, const float h11, float (&out)[4]) {
+    const float d0 = h10 - h00, d1 = h11 - h01;
+    const float ma0 = fmaf(DN_GA, d0, h00), mb0 = fmaf(DN_GB, d0, h00);     // first coordinate a / b, second low
+    const float ma1 = fmaf(DN_GA, d1, h01), mb1 = fmaf(DN_GB, d1, h01);     // ... second high
+    const float da = ma1 - ma0, db = mb1 - mb0;
+    out[0] = fmaf(DN_GA, da, ma0); out[1] = fmaf(DN_GB, da, ma0);
+    out[2] = fmaf(DN_GA, db, mb0); out[3] = fmaf(DN_GB, db, mb0);
+}
+
+// The element: from the 12 sums of nu and the 7 hierarchical coordinates of u to the 8 corner contributions
+// r[i + 2j + 4k] (i, j, k the x, y, z bits of the corner), all in units of kap = hx hy hz / (8 h^2) on isotropic cells
+// (iso), else scaled by kx, ky, kz here.
+__device__ __forceinline__ void s3_element(const float (&Nx)[4], const float (&Ny)[4], const float (&Nz)[4],
+                                           const float e0, const float s0, const float w0,
                                            const float txy, const float txz, const float tyz, const float txyz,
                                            const bool iso, const float kx, const float ky, const float kz,
                                            float (&r)[8]) {
     const float a = DN_GA, bq = DN_GB;
-    float Nx_aa = n[0] + n[4], Nx_ab = n[1] + n[5], Nx_ba = n[2] + n[6], Nx_bb = n[3] + n[7];   // (q, s)
-    float Ny_aa = n[0] + n[2], Ny_ab = n[1] + n[3], Ny_ba = n[4] + n[6], Ny_bb = n[5] + n[7];   // (p, s)
-    float Nz_aa = n[0] + n[1], Nz_ab = n[2] + n[3], Nz_ba = n[4] + n[5], Nz_bb = n[6] + n[7];   // (p, q)
+    float Nx_aa = Nx[0], Nx_ab = Nx[1], Nx_ba = Nx[2], Nx_bb = Nx[3];   // (q, s)
+    float Ny_aa = Ny[0], Ny_ab = Ny[1], Ny_ba = Ny[2], Ny_bb = Ny[3];   // (p, s)
+    float Nz_aa = Nz[0], Nz_ab = Nz[1], Nz_ba = Nz[2], Nz_bb = Nz[3];   // (p, q)
     if (!iso) {
         Nx_aa *= kx; Nx_ab *= kx; Nx_ba *= kx; Nx_bb *= kx;
         Ny_aa *= ky; Ny_ab *= ky; Ny_ba *= ky; Ny_bb *= ky;
@@ -169,12 +190,17 @@ __device__ __forceinline__ void s3_element(const float (&n)[8], const float e0, 
     r[0] = r000; r[1] = r100; r[2] = r010; r[3] = r110; r[4] = r001; r[5] = r101; r[6] = r011; r[7] = dXYZ;
 }
 
-template <int NX, int M, int MINB>
+// MODE 0: KL at the Gauss points; 1 (KN): KL at the nodes, then Q1 interpolation; 2 (ND): stored nodal field.
+// In the nodal modes a slot of the ring holds the nu row next to the u row: copied from the field (ND), or computed
+// from the polynomial of that node line when the row is first used (KN: the table then holds one polynomial per node
+// line, every coefficient twice, and travels with the row itself).
+template <int NX, int M, int MODE, int MINB>
 __global__ void __launch_bounds__(S3_WARPS * 32, MINB)
 strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G) {
     extern __shared__ __align__(16) float smem[];
+    constexpr bool KG = (MODE == 0), KN = (MODE == 1), ND = (MODE == 2);
     constexpr int GS = s3_gs(M);
-    constexpr int CF = 2 * GS;                          // coefficient floats per element row (Gauss rows q = a, b)
+    constexpr int CF = KG ? 2 * GS : KN ? GS : 0;       // coefficient floats per slot (KG: Gauss rows q = a, b of an element row)
     constexpr int CFQ = CF / 4;                         // ... in 16-byte pieces
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int LW = G.LW, SUBS = 32 >> G.lwsh;
@@ -188,22 +214,33 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     // ---- shared by the block: cos(pi x) at the two Gauss columns of each element of a lane, duplicated into both
     // halves of a pair, as float4 (ca, ca, cb, cb) at [element c][lane of the unit]
     float4* cps = reinterpret_cast<float4*>(smem);
-    for (int i = threadIdx.x; i < NX * LW; i += blockDim.x) {
-        const int c = i >> G.lwsh, l = i & (LW - 1);
-        const int xe = min(NX * l, nx - NX) + c;        // element index = index of its left node
-        const float ca = __ldg(P.cg[0] + 2 * xe), cb = __ldg(P.cg[0] + 2 * xe + 1);
-        cps[i] = make_float4(ca, ca, cb, cb);
+    if constexpr (KG) {
+        for (int i = threadIdx.x; i < NX * LW; i += blockDim.x) {
+            const int c = i >> G.lwsh, l = i & (LW - 1);
+            const int xe = min(NX * l, nx - NX) + c;    // element index = index of its left node
+            const float ca = __ldg(P.cg[0] + 2 * xe), cb = __ldg(P.cg[0] + 2 * xe + 1);
+            cps[i] = make_float4(ca, ca, cb, cb);
+        }
+        __syncthreads();                                // the only block-wide barrier: before the march starts
     }
-    __syncthreads();                                    // the only block-wide barrier: before the march starts
     const float4* cpl = cps + lx;
+    u64 cnp[NX / 2];                                    // KN: cos(pi x) at this lane's nodes, in pairs
+    if constexpr (KN) {
+#pragma unroll
+        for (int h = 0; h < NX / 4; ++h) {
+            const float4 q = __ldg(reinterpret_cast<const float4*>(P.cn[0] + x0c + 4 * h));
+            cnp[2 * h] = s3_pack(q.x, q.y); cnp[2 * h + 1] = s3_pack(q.z, q.w);
+        }
+    }
 
     const long long su = ((long long)blockIdx.x * S3_WARPS + warp) * SUBS + sub;
     if (su >= G.units) return;                          // the other units of the warp synchronise among themselves only
     const int C = G.C, RS = G.RS;
     const unsigned RSB = (unsigned)RS * 4u, RINGB = (unsigned)C * RSB;
-    float* ring = smem + 4 * NX * LW + (size_t)(warp * SUBS + sub) * C * RS;
+    float* ring = smem + (KG ? 4 * NX * LW : 0) + (size_t)(warp * SUBS + sub) * C * RS;
     const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring);
-    const int COEF = NX * LW + 4;                       // offset of the coefficient row inside a slot
+    const int UROW = NX * LW + 4;                       // floats of a node row in a slot (with the 4 floats of padding)
+    const int COEF = KG ? UROW : 2 * UROW;              // offset of the coefficient row inside a slot
     const int H1 = 4 * LW + 4;                          // NX = 8: offset of the second 16 bytes of every lane
 
     const int b = (int)(su % P.batch);
@@ -257,27 +294,42 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
 
     // ---- the ring.  Entry n = (plane index pk, row index pj) of the unit goes to slot n mod C: the node row
     // (every lane its own 16-byte pieces) and, for pk, pj >= 1, the coefficients of element row (pk-1, pj-1).
-    for (int s = lx; s < C; s += LW)                    // the 4 floats right of the last lane's nodes stay zero
+    for (int s = lx; s < C; s += LW) {                  // the 4 floats right of the last lane's nodes stay zero
         *reinterpret_cast<float4*>(ring + (size_t)s * RS + 4 * LW) = make_float4(0.f, 0.f, 0.f, 0.f);
+        if constexpr (!KG) *reinterpret_cast<float4*>(ring + (size_t)s * RS + UROW + 4 * LW) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     int pf = 0, pfj = 0, pfk = 0;
     unsigned pfo = 0;                                   // byte offset of the slot the next entry goes to
     const float* usrc = ub + (size_t)kbeg * plane + (size_t)y0 * nx;
-    // coefficient piece of this lane: of element row (pfk-1, pfj-1), so the pointer starts one row and one plane low
-    const float* csrc = linepoly + (((size_t)b * (nz - 1) + kbeg) * (ny - 1) + y0) * CF
-                        - ((size_t)(ny - 1) + 1) * CF + 4 * (lx < CFQ ? lx : 0);
-    const long long uwrap = (long long)plane - (long long)T * nx, cwrap = ((long long)(ny - 1) - T) * CF;
-    const unsigned d0 = ring_s + 16u * lx, d1 = ring_s + 4u * H1 + 16u * lx, dc = ring_s + 4u * COEF + 16u * (lx < CFQ ? lx : 0);
+    // coefficient piece of this lane.  KG: of element row (pfk-1, pfj-1), so the pointer starts one row and one plane
+    // low; KN: of the node line of the entry itself
+    const int clx = (lx < CFQ) ? lx : 0;
+    const float* csrc = KG ? linepoly + (((size_t)b * (nz - 1) + kbeg) * (ny - 1) + y0) * CF - ((size_t)(ny - 1) + 1) * CF + 4 * clx
+                           : linepoly + (((size_t)b * nz + kbeg) * ny + y0) * CF + 4 * clx;
+    const float* nsrc = ND ? P.nu + (size_t)b * P.nodes + x0c + (size_t)kbeg * plane + (size_t)y0 * nx : nullptr;
+    const long long uwrap = (long long)plane - (long long)T * nx, cwrap = ((long long)(KG ? ny - 1 : ny) - T) * CF;
+    const unsigned d0 = ring_s + 16u * lx, d1 = ring_s + 4u * H1 + 16u * lx, dc = ring_s + 4u * COEF + 16u * clx;
     auto issue = [&]() {
         if (pfk < nplanes) {                            // uniform in the unit
             s3_cp16s(d0 + pfo, usrc);
             if constexpr (NX == 8) s3_cp16s(d1 + pfo, usrc + 4);
-            const int cok = (pfk >= 1 && pfj >= 1) ? 1 : 0;
-            s3_cp16s_if(dc + pfo, csrc, (lx < CFQ) ? cok : 0);
-            if constexpr (CFQ > 8) s3_cp16s_if(dc + pfo + 16u * 8u, csrc + 32, (lx + 8 < CFQ && LW == 8) ? cok : 0);
+            if constexpr (ND) {
+                s3_cp16s(d0 + 4u * UROW + pfo, nsrc);
+                if constexpr (NX == 8) s3_cp16s(d1 + 4u * UROW + pfo, nsrc + 4);
+            }
+            if constexpr (CF > 0) {
+                const int cok = (KN || (pfk >= 1 && pfj >= 1)) ? 1 : 0;
+                s3_cp16s_if(dc + pfo, csrc, (lx < CFQ) ? cok : 0);
+                if constexpr (CFQ > 8) s3_cp16s_if(dc + pfo + 16u * 8u, csrc + 32, (lx + 8 < CFQ && LW == 8) ? cok : 0);
+            }
         }
         s3_commit();                                    // one group per entry, possibly empty
         ++pf; ++pfj; usrc += nx; csrc += CF;
-        if (pfj == T) { pfj = 0; ++pfk; usrc += uwrap; csrc += cwrap; }
+        if constexpr (ND) nsrc += nx;
+        if (pfj == T) {
+            pfj = 0; ++pfk; usrc += uwrap; csrc += cwrap;
+            if constexpr (ND) nsrc += uwrap;
+        }
         pfo += RSB;
         if (pfo == RINGB) pfo = 0;
     };
@@ -296,6 +348,36 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
             if (first_col) v[0] = bc0;
             if (last_col) v[NX - 1] = bc1;
         }
+    };
+    auto ldnu = [&](const unsigned off, float (&v)[NX + 1]) {      // nodal modes: the nu row of a slot
+        const float* slot = reinterpret_cast<const float*>(reinterpret_cast<const char*>(ring) + off) + UROW;
+        const float4 q = *reinterpret_cast<const float4*>(slot + 4 * lx);
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+        if constexpr (NX == 8) {
+            const float4 q1 = *reinterpret_cast<const float4*>(slot + H1 + 4 * lx);
+            v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+        }
+        v[NX] = slot[4 * (lx + 1)];
+    };
+    // KN: nu at this lane's nodes of the row in a slot, from the polynomial that came with the row, into the slot
+    auto nurow = [&](const unsigned off) {
+        float* slot = reinterpret_cast<float*>(reinterpret_cast<char*>(ring) + off);
+        u64 gg[GS / 2];
+        const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(slot + COEF);
+#pragma unroll
+        for (int i = 0; i < GS / 4; ++i) { const ulonglong2 t = gp[i]; gg[2 * i] = t.x; gg[2 * i + 1] = t.y; }
+        float nn[NX];
+#pragma unroll
+        for (int h = 0; h < NX / 2; ++h) {
+            u64 e = gg[M];
+#pragma unroll
+            for (int i = M - 1; i >= 0; --i) e = s3_fma2(e, cnp[h], gg[i]);
+            float e0, e1;
+            s3_unpack(e, e0, e1);
+            nn[2 * h] = s3_ex2(e0); nn[2 * h + 1] = s3_ex2(e1);
+        }
+        *reinterpret_cast<float4*>(slot + UROW + 4 * lx) = make_float4(nn[0], nn[1], nn[2], nn[3]);
+        if constexpr (NX == 8) *reinterpret_cast<float4*>(slot + UROW + H1 + 4 * lx) = make_float4(nn[4], nn[5], nn[6], nn[7]);
     };
     // parked partial sums of one node row (plain loads: this thread wrote them one plane ago)
     auto ld4 = [&](const float* p, float (&v)[NX]) {
@@ -341,7 +423,26 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
             float uA[NX + 1], uB[NX + 1], uC[NX + 1], uD[NX + 1];
             ldrow(oA, uA); ldrow(oB, uB); ldrow(oC, uC); ldrow(oD, uD);
             u64 ga[GS / 2], gb[GS / 2];                 // Gauss row q = a / b; each entry holds (plane s = a, s = b)
-            {
+            float nA[NX + 1], nB[NX + 1], nC[NX + 1], nD[NX + 1];      // nodal modes: nu on the four node rows
+            float yA[NX + 1], yC[NX + 1], zA[NX + 1], zB[NX + 1];      // ... summed over the rows of a plane / the planes of a row
+            if constexpr (KN) {
+                // rows meet the march at its upper, far corner: a row is new when it is D, and also when it is B in the
+                // unit's first plane, C in a plane's first row, A at the very start
+                if (kk == 0 && jj == 0) nurow(oA);
+                if (kk == 0) nurow(oB);
+                if (jj == 0) nurow(oC);
+                nurow(oD);
+                __syncwarp(submask);                    // the node right of a lane's last is the next lane's
+            }
+            if constexpr (!KG) {
+                ldnu(oA, nA); ldnu(oB, nB); ldnu(oC, nC); ldnu(oD, nD);
+#pragma unroll
+                for (int c = 0; c <= NX; ++c) {
+                    yA[c] = nA[c] + nB[c]; yC[c] = nC[c] + nD[c];
+                    zA[c] = nA[c] + nC[c]; zB[c] = nB[c] + nD[c];
+                }
+            }
+            if constexpr (KG) {
                 const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(reinterpret_cast<const char*>(ring) + oD) + COEF / 4;
 #pragma unroll
                 for (int i = 0; i < GS / 4; ++i) {
@@ -371,10 +472,18 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                 const float eC = uC[c + 1] - uC[c], eD = uD[c + 1] - uD[c];
                 const float slo = uB[c] - uA[c], sup = uD[c] - uC[c], w0 = uC[c] - uA[c];
                 const float txy = eB - eA, txyu = eD - eC, txz = eC - eA, tyz = sup - slo, txyz = txyu - txy;
-                float nu[8], r[8];
-                const ulonglong2 cc = *reinterpret_cast<const ulonglong2*>(cpl + c * LW);
-                s3_nu_gauss<M>(ga, gb, cc.x, cc.y, nu);
-                s3_element(nu, eA, slo, w0, txy, txz, tyz, txyz, iso, kx, ky, kz, r);
+                float Nx[4], Ny[4], Nz[4], r[8];
+                if constexpr (KG) {
+                    float nu[8];
+                    const ulonglong2 cc = *reinterpret_cast<const ulonglong2*>(cpl + c * LW);
+                    s3_nu_gauss<M>(ga, gb, cc.x, cc.y, nu);
+                    s3_sums_gauss(nu, Nx, Ny, Nz);
+                } else {
+                    s3_bilerp(nA[c] + nA[c + 1], nB[c] + nB[c + 1], nC[c] + nC[c + 1], nD[c] + nD[c + 1], Nx);   // (q, s)
+                    s3_bilerp(yA[c], yA[c + 1], yC[c], yC[c + 1], Ny);                                           // (p, s)
+                    s3_bilerp(zA[c], zA[c + 1], zB[c], zB[c + 1], Nz);                                           // (p, q)
+                }
+                s3_element(Nx, Ny, Nz, eA, slo, w0, txy, txz, tyz, txyz, iso, kx, ky, kz, r);
                 if (c == NX - 1) {
                     // the lane's last element: its right-hand corners belong to the next lane; in the lane that ends the
                     // row it does not exist (g3 = 0)
@@ -540,6 +649,53 @@ __global__ void __launch_bounds__(128) linepoly3d_kernel(const Params P, float* 
     for (int i = 0; i < GS / 2; ++i) dst[i] = make_float4(row[4 * i], row[4 * i + 1], row[4 * i + 2], row[4 * i + 3]);
 }
 
+// KL at the nodes: the polynomial (in c = cos(pi x)) of the KL exponent along every node line (y_j, z_k), every
+// coefficient twice so that two nodes share a packed FMA: [B][nz][ny][GS] floats.  One block per (sample, node plane,
+// 128 node rows).
+template <int M>
+__global__ void __launch_bounds__(128) nodepoly3d_kernel(const Params P, float* __restrict__ out) {
+    constexpr int GS = s3_gs(M);
+    __shared__ double h[M][M];                          // h[i][j] = sum_k ckl[i][j][k] cos(k pi z)
+    const int iz = blockIdx.y, b = blockIdx.z;
+    const float* w = P.ckl + (size_t)b * M * M * M;
+    for (int t = threadIdx.x; t < M * M; t += blockDim.x) {
+        double acc = 0.0;
+#pragma unroll
+        for (int k = 0; k < M; ++k) acc += (double)w[t * M + k] * (double)P.cn[2][(size_t)k * P.nstride[2] + iz];
+        h[t / M][t % M] = acc;
+    }
+    __syncthreads();
+    const int iy = blockIdx.x * blockDim.x + threadIdx.x;
+    if (iy >= P.ny) return;
+    double cy[M];
+#pragma unroll
+    for (int j = 0; j < M; ++j) cy[j] = (double)P.cn[1][(size_t)j * P.nstride[1] + iy];
+    double acc[M + 1], tp[M + 1], tc[M + 1];
+#pragma unroll
+    for (int k = 0; k <= M; ++k) { acc[k] = 0.0; tp[k] = (k == 0) ? 1.0 : 0.0; tc[k] = (k == 1) ? 1.0 : 0.0; }
+#pragma unroll
+    for (int i = 1; i <= M; ++i) {
+        double g = 0.0;
+#pragma unroll
+        for (int j = 0; j < M; ++j) g += h[i - 1][j] * cy[j];
+#pragma unroll
+        for (int k = 0; k <= i; ++k) acc[k] += g * tc[k];
+        double tn[M + 1];
+#pragma unroll
+        for (int k = 0; k <= M; ++k) tn[k] = ((k > 0) ? 2.0 * tc[k - 1] : 0.0) - tp[k];
+#pragma unroll
+        for (int k = 0; k <= M; ++k) { tp[k] = tc[k]; tc[k] = tn[k]; }
+    }
+    float row[GS];
+#pragma unroll
+    for (int i = 0; i < GS; ++i) row[i] = 0.f;
+#pragma unroll
+    for (int k = 0; k <= M; ++k) { row[2 * k] = (float)acc[k]; row[2 * k + 1] = (float)acc[k]; }
+    float4* dst = reinterpret_cast<float4*>(out + (((size_t)b * P.nz + iz) * P.ny + iy) * GS);
+#pragma unroll
+    for (int i = 0; i < GS / 4; ++i) dst[i] = make_float4(row[4 * i], row[4 * i + 1], row[4 * i + 2], row[4 * i + 3]);
+}
+
 // Adds the seam contributions to r (fixed order per node: own sums, tile seam, chunk seam, the entry for nodes on both).
 // First range of threads: the nodes of the tile seam rows (t + 1) Ry on every plane; second range: the nodes of the
 // chunk seam planes (c + 1) Z that are not on a tile seam row.  The two ranges touch different nodes.
@@ -597,23 +753,26 @@ int s3_sm_count() {
 constexpr size_t S3_SMEM_SM = 233472;              // shared memory of an SM; a block also reserves 1 KiB
 constexpr size_t S3_SMEM_BLOCK = 232448;           // most a block can ask for
 
-int s3_env(const char* n, int d);
-int s3_nxl(int nx) { if (nx > 128) return 8; return (nx % 8 == 0 && s3_env("DN_S3_NX", 4) == 8) ? 8 : 4; }  // nodes per lane
-int s3_env(const char* n, int d) { const char* e = getenv(n); return e ? atoi(e) : d; }   // EXPERIMENT
-int s3_minb(int nxl) { return s3_env("DN_S3_MINB", (nxl == 8) ? 3 : 4); } // resident blocks of 4 warps per SM the kernel is compiled for
+int s3_nxl(int nx) { return (nx > 128) ? 8 : 4; }  // nodes per lane (8 on narrow rows was slower: 89 against 79 us on 64^3 x 32)
+// resident blocks of 4 warps per SM the kernel is compiled for: the nodal modes keep two rows per slot and trade
+// warps for taller tiles on wide rows
+int s3_minb(int nxl, int mode) { return (nxl == 8) ? (mode == DN_NU_KL_GAUSS ? 3 : 2) : 4; }
+int s3_slot_floats(int nxl, int lw, int mode, int m) {
+    const int urow = nxl * lw + 4;
+    return (mode == DN_NU_KL_GAUSS) ? urow + 2 * s3_gs(m) : (mode == DN_NU_KL_NODAL) ? 2 * urow + s3_gs(m) : 2 * urow;
+}
 
 S3Geo geometry3s(const dn_problem& p) {
     S3Geo g{};
     const int nx = p.grid.nx, ny = p.grid.ny, nz = p.grid.nz;
-    const int NX = s3_nxl(nx), minb = s3_minb(NX);
+    const int NX = s3_nxl(nx), minb = s3_minb(NX, p.nu_mode);
     g.LW = 8; g.lwsh = 3;
     while (g.LW * NX < nx) { g.LW *= 2; ++g.lwsh; }
     const int subs = 32 / g.LW;
-    const int m = p.kl_modes;
-    g.RS = NX * g.LW + 4 + 2 * s3_gs(m);
+    g.RS = s3_slot_floats(NX, g.LW, p.nu_mode, p.kl_modes);
     size_t per_block = (S3_SMEM_SM - (size_t)minb * 1024) / minb;
     if (per_block > S3_SMEM_BLOCK) per_block = S3_SMEM_BLOCK;
-    per_block -= sizeof(float) * 4 * NX * g.LW;      // the block's table of cosine pairs
+    if (p.nu_mode == DN_NU_KL_GAUSS) per_block -= sizeof(float) * 4 * NX * g.LW;      // the block's table of cosine pairs
     const int cmax = (int)(per_block / ((size_t)S3_WARPS * subs * g.RS * sizeof(float)));
     int ry_max = cmax - 2 - S3_D;
     if (ry_max > ny - 1) ry_max = ny - 1;
@@ -636,34 +795,28 @@ S3Geo geometry3s(const dn_problem& p) {
             }
         }
     }
-    if (getenv("DN_S3_RY")) {   // EXPERIMENT
-        g.Ry = atoi(getenv("DN_S3_RY")); g.Z = s3_env("DN_S3_Z", g.Z);
-        g.ntile = (ny - 1 + g.Ry - 1) / g.Ry; g.nchunk = (nz - 1 + g.Z - 1) / g.Z; g.units = (long long)p.batch * g.ntile * g.nchunk;
-    }
     g.C = g.Ry + 2 + S3_D;
     return g;
 }
 
-template <int NX, int M, int MINB>
+template <int NX, int M, int MODE, int MINB>
 cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
     const int subs = 32 / g.LW;
-    const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * g.C * g.RS + 4 * NX * g.LW);
+    const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * g.C * g.RS + (MODE == 0 ? 4 * NX * g.LW : 0));
     const long long per_block = (long long)S3_WARPS * subs;
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
-    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    strip3d_kernel<NX, M, MINB><<<blocks, S3_WARPS * 32, smem, s>>>(P, linepoly, g);
+    strip3d_kernel<NX, M, MODE, MINB><<<blocks, S3_WARPS * 32, smem, s>>>(P, linepoly, g);
     return cudaGetLastError();
 }
 
 template <int M>
 cudaError_t launch_m3(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
-    if (M == 3 && s3_nxl(P.nx) == 8) {   // EXPERIMENT
-        const int mb = s3_minb(8);
-        if (mb == 2) return launch_nm<8, 3, 2>(P, linepoly, g, s);
-        if (mb == 4) return launch_nm<8, 3, 4>(P, linepoly, g, s);
-    }
-    return (s3_nxl(P.nx) == 8) ? launch_nm<8, M, 3>(P, linepoly, g, s) : launch_nm<4, M, 4>(P, linepoly, g, s);
+    const bool wide = (s3_nxl(P.nx) == 8);
+    if (P.nu_mode == DN_NU_KL_NODAL)
+        return wide ? launch_nm<8, M, 1, 2>(P, linepoly, g, s) : launch_nm<4, M, 1, 4>(P, linepoly, g, s);
+    return wide ? launch_nm<8, M, 0, 3>(P, linepoly, g, s) : launch_nm<4, M, 0, 4>(P, linepoly, g, s);
 }
 
 dn_problem s3_problem_of(const Params& P) {
@@ -678,7 +831,7 @@ dn_problem s3_problem_of(const Params& P) {
 // Rows of at most 128 nodes take 4 nodes per lane, rows of at most 256 nodes 8 (then nx must be a multiple of 8,
 // so that only the last element of the last lane falls outside the grid).
 bool strip3d_applicable(const dn_problem& p) {
-    if (!(p.grid.dim == 3 && p.f == nullptr && p.nu_mode == DN_NU_KL_GAUSS && p.grid.nx % 4 == 0 && p.grid.nx >= 8 &&
+    if (!(p.grid.dim == 3 && p.f == nullptr && p.grid.nx % 4 == 0 && p.grid.nx >= 8 &&
           p.grid.nx <= 256 && p.grid.ny >= 2 && p.grid.nz >= 2))
         return false;
     return p.grid.nx <= 128 || p.grid.nx % 8 == 0;
@@ -707,15 +860,22 @@ size_t strip3d_zseam_floats(const dn_problem& p) {
     return (size_t)p.batch * (g.nchunk - 1) * ((size_t)p.grid.ny + (g.ntile - 1)) * p.grid.nx;
 }
 
+// the coefficient table: per element row its four Gauss lines (KL at the Gauss points), or per node line (KL at the nodes)
 size_t strip3d_linepoly_floats(const dn_problem& p) {
-    if (!strip3d_applicable(p)) return 0;
+    if (!strip3d_applicable(p) || p.nu_mode == DN_NU_NODAL) return 0;
+    if (p.nu_mode == DN_NU_KL_NODAL) return (size_t)p.batch * p.grid.nz * p.grid.ny * s3_gs(p.kl_modes);
     return (size_t)p.batch * (p.grid.nz - 1) * (p.grid.ny - 1) * 2 * s3_gs(p.kl_modes);
 }
 
 template <int M>
 static cudaError_t launch_linepoly3d_m(const Params& P, float* linepoly, cudaStream_t s) {
-    const dim3 grid((unsigned)((P.ny - 1 + 127) / 128), (unsigned)(P.nz - 1), (unsigned)P.batch);
-    linepoly3d_kernel<M><<<grid, 128, 0, s>>>(P, linepoly);
+    if (P.nu_mode == DN_NU_KL_NODAL) {
+        const dim3 grid((unsigned)((P.ny + 127) / 128), (unsigned)P.nz, (unsigned)P.batch);
+        nodepoly3d_kernel<M><<<grid, 128, 0, s>>>(P, linepoly);
+    } else {
+        const dim3 grid((unsigned)((P.ny - 1 + 127) / 128), (unsigned)(P.nz - 1), (unsigned)P.batch);
+        linepoly3d_kernel<M><<<grid, 128, 0, s>>>(P, linepoly);
+    }
     return cudaGetLastError();
 }
 
@@ -736,7 +896,9 @@ cudaError_t launch_linepoly3d(const Params& P, float* linepoly, cudaStream_t s) 
 cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t s) {
     const S3Geo g = geometry3s(s3_problem_of(P));
     cudaError_t e = cudaErrorInvalidValue;
-    switch (P.m) {
+    if (P.nu_mode == DN_NU_NODAL) {
+        e = (s3_nxl(P.nx) == 8) ? launch_nm<8, 1, 2, 2>(P, linepoly, g, s) : launch_nm<4, 1, 2, 4>(P, linepoly, g, s);
+    } else switch (P.m) {
         case 1: e = launch_m3<1>(P, linepoly, g, s); break;
         case 2: e = launch_m3<2>(P, linepoly, g, s); break;
         case 3: e = launch_m3<3>(P, linepoly, g, s); break;

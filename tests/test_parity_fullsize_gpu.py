@@ -12,7 +12,7 @@ from parity_util import dev, J_RTOL, R_RTOL, guarded, guards_intact
 
 pytestmark = pytest.mark.gpu
 
-PATHS = {2: ("strip2d",), 4: ("strip3d", "tiled3d", "generic")}
+PATHS = {2: ("strip2d",), 4: ("strip3d",)}
 
 
 @pytest.mark.parametrize("mode", [B.DN_NU_KL_GAUSS, B.DN_NU_NODAL, B.DN_NU_KL_NODAL])

@@ -1,5 +1,5 @@
-"""GPU parity of the 3D strip kernel (rows of at most 256 nodes, KL diffusivity at the Gauss points, energy and residual
-fused) against the fp64 oracle: every lane layout (4 or 8 nodes per lane; 8, 16 or 32 lanes per unit, i.e. 4, 2 or 1
+"""GPU parity of the 3D strip kernel (rows of at most 256 nodes, energy and residual fused, all three diffusivity
+modes) against the fp64 oracle: every lane layout (4 or 8 nodes per lane; 8, 16 or 32 lanes per unit, i.e. 4, 2 or 1
 units per warp), rows that end inside a lane group, one and many tiles and chunks, batches that leave units of a warp
 idle, and every option the kernel serves."""
 import numpy as np
@@ -19,11 +19,16 @@ SIZES = [(8, 2, 2, 1, 1), (12, 11, 6, 2, 2), (32, 9, 7, 3, 3), (28, 45, 5, 1, 2)
          (200, 5, 4, 1, 5), (256, 17, 5, 1, 3), (256, 40, 30, 2, 6), (64, 150, 40, 9, 2), (16, 8, 300, 1, 1)]
 
 
+MODES = [B.DN_NU_KL_GAUSS, B.DN_NU_KL_NODAL, B.DN_NU_NODAL]   # KL at the Gauss points / at the nodes (in the kernel), stored nodal field
+
+
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("nx,ny,nz,batch,m", SIZES)
-def test_strip3d_parity(nx, ny, nz, batch, m):
+def test_strip3d_parity(nx, ny, nz, batch, m, mode):
     inp = inputs.random_inputs(3, nx, ny, nz, batch, m, seed=11 + nx + 3 * ny + nz, f_const=0.6)
-    po, pg = make_problems(inp, B.DN_NU_KL_GAUSS)
-    expect = "strip3d" if (nx <= 128 or nx % 8 == 0) else "tiled3d"
+    nu = inputs.random_positive_field(inp.u.shape, 5) if mode == B.DN_NU_NODAL else None
+    po, pg = make_problems(inp, mode, nu=nu)
+    expect = "strip3d" if (nx <= 128 or nx % 8 == 0) else ("generic" if mode == B.DN_NU_KL_NODAL else "tiled3d")
     assert B.dn_path_name(pg) == expect
     Jo, _, _, ro = oracle.energy_grad(po, inp.u)
     Jg, rg = run_gpu(pg, inp.u)
@@ -31,13 +36,15 @@ def test_strip3d_parity(nx, ny, nz, batch, m):
     assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
 
 
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("nx,ny,nz", [(64, 9, 6), (24, 6, 5), (256, 7, 6), (128, 12, 9)])
-def test_strip3d_options(nx, ny, nz):
+def test_strip3d_options(nx, ny, nz, mode):
     inp = inputs.random_inputs(3, nx, ny, nz, 3, 3, seed=42, f_const=-0.4)
     u = inputs.random_field(inp.u.shape, 8)           # boundary values NOT satisfied
+    nu = inputs.random_positive_field(inp.u.shape, 6) if mode == B.DN_NU_NODAL else None
     gJ = np.array([1.5, -2.0, 0.25], dtype=np.float32)
     for flags in (0, B.DN_NO_MASK, B.DN_IMPOSE_BC_ON_LOAD, B.DN_IMPOSE_BC_ON_LOAD | B.DN_NO_MASK):
-        po, pg = make_problems(inp, B.DN_NU_KL_GAUSS, flags=flags, bc=(0.8, -0.3))
+        po, pg = make_problems(inp, mode, nu=nu, flags=flags, bc=(0.8, -0.3))
         assert B.dn_path_name(pg) == "strip3d"
         Jo, _, _, ro = oracle.energy_grad(po, u, gJ=gJ.astype(np.float64))
         Jg, rg = run_gpu(pg, u, gJ=gJ)
@@ -45,7 +52,7 @@ def test_strip3d_options(nx, ny, nz):
         if not (flags & B.DN_NO_MASK):
             assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
     # rectangular cells (hx != hy != hz take the scaled path), residual-only call, determinism with a stale workspace
-    po, pg = make_problems(inp, B.DN_NU_KL_GAUSS)
+    po, pg = make_problems(inp, mode, nu=nu)
     ws = B.new_workspace(pg)
     outs = []
     for it in range(3):
