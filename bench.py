@@ -120,7 +120,7 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def oracle_sample_run(cfg: int, mode: str, target_seconds: float = 12.0):
+def oracle_sample_run(cfg: int, mode: str, target_seconds: float = 12.0, want_results: bool = False):
     """Times the oracle (as it stands) on a bounded sample of the workload: whole samples of the batch."""
     import oracle
     wl = inputs.WORKLOADS[cfg]
@@ -134,15 +134,21 @@ def oracle_sample_run(cfg: int, mode: str, target_seconds: float = 12.0):
         p = oracle.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=nu_mode, nu=nu,
                            kl_modes=inp.kl_modes, kl_w=inp.kl_w, f_const=inp.f_const, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1)
         t = time.perf_counter()
-        oracle.energy_grad(p, inp.u)
-        return time.perf_counter() - t
+        res = oracle.energy_grad(p, inp.u)
+        return time.perf_counter() - t, res
 
-    t1 = run([0])
+    t1, res = run([0])
     n = int(max(1, min(wl.batch, round(target_seconds / max(t1, 1e-3)))))
-    t = run(list(range(n))) if n > 1 else t1
-    return {"value": wl.elements * n / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    if n > 1:
+        t, res = run(list(range(n)))
+    else:
+        t = t1
+    base = {"value": wl.elements * n / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"{n} of {wl.batch} samples of {wl.name} ({wl.elements * n} elements, energy + full residual), "
-                      f"{t:.2f} s wall"}, t, n
+                      f"{t:.2f} s wall"}
+    if want_results:
+        return base, t, n, res[0], res[3]
+    return base, t, n
 
 
 def run_reference(args):
@@ -381,7 +387,7 @@ def main_cg(args):
         peak, peak_kind = measured_peak()
         nodes = wl.nodes * inp.batch
         achieved = CG_BYTES_PER_NODE_ITER * nodes / (iter_ms * 1e-3) / 1e9
-        launches_per_iter = (2 if B.dn_path_name(prob) == "tiled3d" else 1) + 4    # fused kernel (3D: + seam fix-up) + 4 CG kernels
+        launches_per_iter = (2 if B.dn_path_name(prob) in ("tiled3d", "strip3d") else 1) + 4    # fused kernel (3D: + seam fix-up) + 4 CG kernels
         print(json.dumps({
             "metric": "PCG Gnode-iterations/s", "value": world * nodes * CG_ITERS / (step_ms * 1e-3) / 1e9,
             "unit": "Gnode-iterations/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
@@ -414,6 +420,8 @@ def main():
                          "cg: matrix-free preconditioned CG on the fused kernel (workload --config, KL at Gauss points)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="skip the device timing of the other target workloads and modes (default run only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference" and args.workload == "cg":
@@ -441,29 +449,94 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     B.lib()
 
-    wl = inputs.WORKLOADS[args.config]
-    # every rank draws its own contiguous piece of the global mini-batch (world * B samples of the same recipe)
-    inp = inputs.make_inputs(args.config, samples=sharding.minibatch_indices(world * wl.batch, world * wl.batch,
-                                                                           world, rank, 0))
-    u = torch.from_numpy(inp.u).cuda()
-    w = torch.from_numpy(inp.kl_w).cuda()
-    nu = None
-    mode = {"kl": B.DN_NU_KL_GAUSS, "nodal": B.DN_NU_NODAL, "klnodal": B.DN_NU_KL_NODAL}[args.nu_mode]
-    if mode == B.DN_NU_NODAL:
-        nu = torch.empty_like(u)
-        B.dn_kl_field(inp.dim, inp.nx, inp.ny, inp.nz, inp.batch, inp.kl_modes, w, nu)
-    prob = B.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=mode, nu=nu,
-                     kl_modes=inp.kl_modes, kl_w=w, f_const=inp.f_const, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1)
-    r = torch.empty_like(u)
-    J = torch.empty(inp.batch, device="cuda")
-    ws = B.new_workspace(prob)
-    cs = prob.c_struct()
-    field_bytes = u.numel() * 4
-    l2_bytes = torch.cuda.get_device_properties(local).L2_cache_size
-    traffic_bytes = 2 * field_bytes + (field_bytes if nu is not None else 0)
-    flush = None
-    if traffic_bytes < 2 * l2_bytes:
-        flush = torch.empty(max(2 * l2_bytes, 256 << 20), dtype=torch.uint8, device="cuda")
+    def device_run(cfg, nu_mode, K, warmup, sampler=None):
+        """K timed steps of one workload on this rank's device: the step time (plain calls) and, from K more steps, the
+        time of the fused kernel alone.  Returns the numbers and the tensors (for the parity check and the extras)."""
+        wl = inputs.WORKLOADS[cfg]
+        # every rank draws its own contiguous piece of the global mini-batch (world * B samples of the same recipe)
+        inp = inputs.make_inputs(cfg, samples=sharding.minibatch_indices(world * wl.batch, world * wl.batch, world, rank, 0))
+        u = torch.from_numpy(inp.u).cuda()
+        w = torch.from_numpy(inp.kl_w).cuda()
+        nu = None
+        mode = {"kl": B.DN_NU_KL_GAUSS, "nodal": B.DN_NU_NODAL, "klnodal": B.DN_NU_KL_NODAL}[nu_mode]
+        if mode == B.DN_NU_NODAL:
+            nu = torch.empty_like(u)
+            B.dn_kl_field(inp.dim, inp.nx, inp.ny, inp.nz, inp.batch, inp.kl_modes, w, nu)
+        prob = B.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=mode, nu=nu,
+                         kl_modes=inp.kl_modes, kl_w=w, f_const=inp.f_const, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1)
+        r = torch.empty_like(u)
+        J = torch.empty(inp.batch, device="cuda")
+        ws = B.new_workspace(prob)
+        cs = prob.c_struct()
+        field_bytes = u.numel() * 4
+        l2_bytes = torch.cuda.get_device_properties(local).L2_cache_size
+        traffic_bytes = 2 * field_bytes + (field_bytes if nu is not None else 0)
+        flush = None
+        if traffic_bytes < 2 * l2_bytes:
+            flush = torch.empty(max(2 * l2_bytes, 256 << 20), dtype=torch.uint8, device="cuda")
+        ev_step = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        ev_main = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for a, b_ in ev_step + ev_main:            # create the underlying CUDA events
+            a.record(); b_.record()
+        for _ in range(warmup):
+            if flush is not None:
+                flush.zero_()
+            B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
+        barrier()
+        if sampler is not None:
+            sampler.start()
+            time.sleep(0.15)
+        t0 = time.time()
+        # the K timed steps: the plain call a user makes (no events inside it).  Inputs larger than L2: one event pair
+        # around all K steps; otherwise one pair per step, so that the L2 flush between steps stays outside the timing.
+        if flush is None:
+            ev_step[0][0].record()
+            for k in range(K):
+                B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
+            ev_step[0][1].record()
+        else:
+            for k in range(K):
+                flush.zero_()
+                ev_step[k][0].record()
+                B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
+                ev_step[k][1].record()
+        barrier()
+        step_ms = (ev_step[0][0].elapsed_time(ev_step[0][1]) if flush is None
+                   else sum(a.elapsed_time(b_) for a, b_ in ev_step)) / K
+        # K more steps with events around the fused kernel alone (the roofline's kernel time)
+        for k in range(K):
+            if flush is not None:
+                flush.zero_()
+            B.dn_energy_grad_traced(prob, u, None, J, r, ws, ev_main[k][0], ev_main[k][1], _cstruct=cs)
+        barrier()
+        t1 = time.time()
+        clocks = sampler.stop(t0, t1) if sampler is not None else None
+        main_ms = sum(a.elapsed_time(b_) for a, b_ in ev_main) / K
+        return {"wl": wl, "inp": inp, "u": u, "w": w, "nu": nu, "mode": mode, "prob": prob, "r": r, "J": J, "ws": ws, "cs": cs,
+                "field_bytes": field_bytes, "flush": flush, "step_ms": step_ms, "main_ms": main_ms, "clocks": clocks,
+                "nu_mode": nu_mode}
+
+    def roofline_of(run, step_ms, main_ms):
+        """The roofline objects of one device run (rank 0): HBM (the metric's roof) and FP32 issue."""
+        wl, inp, mode = run["wl"], run["inp"], run["mode"]
+        peak, peak_kind = measured_peak()
+        elements = wl.elements * inp.batch
+        nodes = wl.nodes * inp.batch
+        alg_bytes = nodes * (12 if mode == B.DN_NU_NODAL else 8)
+        achieved = alg_bytes / (main_ms * 1e-3) / 1e9
+        path = B.dn_path_name(run["prob"])
+        cap = ncu_capture(f"{path}:{wl.name}:{run['nu_mode']}")
+        alu = None
+        if cap:
+            ops = cap["fp32_ops_per_element"] * elements / (main_ms * 1e-3)
+            alu = {"bound": "alu", "achieved": ops / 1e12, "peak": FP32_PEAK_LANE_OPS / 1e12, "unit": "T FP32 lane-ops/s",
+                   "frac": ops / FP32_PEAK_LANE_OPS, "fp32_ops_per_element": cap["fp32_ops_per_element"],
+                   "note": "executed FP32 operations (ncu) / kernel time, against SMs x 128 lanes x max clock"}
+        roof = {"bound": "hbm", "kernel": f"fused energy+residual ({path})", "achieved": achieved,
+                "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": main_ms,
+                "traffic": cap["traffic"] if cap else None}
+        return path, elements, roof, alu
 
     def barrier():
         if world > 1:
@@ -471,45 +544,10 @@ def main():
         torch.cuda.synchronize()
 
     K = args.steps
-    ev_step = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    ev_main = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    for a, b_ in ev_step + ev_main:            # create the underlying CUDA events
-        a.record(); b_.record()
-    for _ in range(args.warmup):
-        if flush is not None:
-            flush.zero_()
-        B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
-    barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.15)
-    t0 = time.time()
-    # the K timed steps: the plain call a user makes (no events inside it).  Inputs larger than L2: one event pair
-    # around all K steps; otherwise one pair per step, so that the L2 flush between steps stays outside the timing.
-    if flush is None:
-        ev_step[0][0].record()
-        for k in range(K):
-            B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
-        ev_step[0][1].record()
-    else:
-        for k in range(K):
-            flush.zero_()
-            ev_step[k][0].record()
-            B.dn_energy_grad_traced(prob, u, None, J, r, ws, None, None, _cstruct=cs)
-            ev_step[k][1].record()
-    barrier()
-    step_ms = (ev_step[0][0].elapsed_time(ev_step[0][1]) if flush is None
-               else sum(a.elapsed_time(b_) for a, b_ in ev_step)) / K
-    # K more steps with events around the fused kernel alone (the roofline's kernel time)
-    for k in range(K):
-        if flush is not None:
-            flush.zero_()
-        B.dn_energy_grad_traced(prob, u, None, J, r, ws, ev_main[k][0], ev_main[k][1], _cstruct=cs)
-    barrier()
-    t1 = time.time()
-    clocks = sampler.stop(t0, t1) if rank == 0 else None
-    main_ms = sum(a.elapsed_time(b_) for a, b_ in ev_main) / K
+    sampler = ClockSampler(local) if rank == 0 else None
+    run = device_run(args.config, args.nu_mode, K, args.warmup, sampler)
+    wl, inp, u, w, nu, mode, prob, r, J, ws, cs = (run[k] for k in ("wl", "inp", "u", "w", "nu", "mode", "prob", "r", "J", "ws", "cs"))
+    field_bytes, flush, step_ms, main_ms, clocks = (run[k] for k in ("field_bytes", "flush", "step_ms", "main_ms", "clocks"))
     Jsum = float(J.double().sum())
 
     # ---- the two small entry points of the path: diffusivity synthesis (4 B/node written) and the Dirichlet faces
@@ -589,21 +627,21 @@ def main():
     step_ms, main_ms, e2e_ms = sharding.max_over_ranks([step_ms, main_ms, e2e_ms])
     Jmean = sharding.mean_over_ranks(Jsum, inp.batch)          # the averaged loss of Algorithm 1 (one scalar all-reduce)
 
+    # ---- the other target workloads and modes, device-timed in this process (single-GPU default run only)
+    secondary = None
+    if world == 1 and not args.no_secondary and args.config == 2 and args.nu_mode == "kl":
+        secondary = []
+        for cfg2, mode2 in ((4, "kl"), (4, "nodal"), (2, "nodal"), (2, "klnodal")):
+            sub = device_run(cfg2, mode2, max(5, min(K, 20)), 3, ClockSampler(local))
+            path2, elements2, roof2, alu2 = roofline_of(sub, sub["step_ms"], sub["main_ms"])
+            secondary.append({"workload": sub["wl"].name, "nu_mode": mode2, "kernel_path": path2, "ms_per_step": sub["step_ms"],
+                              "value": elements2 / (sub["step_ms"] * 1e-3) / 1e9, "unit": UNIT, "roofline": roof2,
+                              "roofline_alu": alu2, "clocks": sub["clocks"], "checksum_J": float(sub["J"].double().sum())})
+            del sub
+            torch.cuda.empty_cache()
+
     if rank == 0:
-        peak, peak_kind = measured_peak()
-        elements = wl.elements * inp.batch
-        nodes = wl.nodes * inp.batch
-        alg_bytes = nodes * (12 if mode == B.DN_NU_NODAL else 8)
-        achieved = alg_bytes / (main_ms * 1e-3) / 1e9
-        path = B.dn_path_name(prob)
-        key = f"{path}:{wl.name}:{args.nu_mode}"
-        cap = ncu_capture(key)
-        alu = None
-        if cap:
-            ops = cap["fp32_ops_per_element"] * elements / (main_ms * 1e-3)
-            alu = {"bound": "alu", "achieved": ops / 1e12, "peak": FP32_PEAK_LANE_OPS / 1e12, "unit": "T FP32 lane-ops/s",
-                   "frac": ops / FP32_PEAK_LANE_OPS, "fp32_ops_per_element": cap["fp32_ops_per_element"],
-                   "note": "executed FP32 operations (ncu) / kernel time, against SMs x 128 lanes x max clock"}
+        path, elements, roof, alu = roofline_of(run, step_ms, main_ms)
         line = {
             "metric": METRIC, "value": world * elements / (step_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
@@ -616,15 +654,21 @@ def main():
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
                     "entry": "dn_energy_grad_host (pinned host buffers)"},
             "gpu_launches": K * B.dn_launches_per_call(prob),
-            "roofline": {"bound": "hbm", "kernel": f"fused energy+residual ({path})", "achieved": achieved,
-                         "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                         "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": main_ms,
-                         "traffic": cap["traffic"] if cap else None},
+            "roofline": roof,
             "roofline_alu": alu,
             "checksum_J": Jsum, "mean_J_all_ranks": Jmean, "l2_resident_extras": extras, "aux_kernels": aux,
+            "secondary": secondary,
         }
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = oracle_sample_run(args.config, args.nu_mode)[0]
+            base, _, n, Jo, ro = oracle_sample_run(args.config, args.nu_mode, want_results=True)
+            line["cpu_baseline"] = base
+            # the device results of the timed run against the oracle's, on the samples the baseline just computed
+            Jg = J[:n].cpu().numpy().astype(np.float64)
+            rerr = 0.0
+            for b_ in range(n):
+                rerr = max(rerr, float(np.abs(r[b_].cpu().numpy() - ro[b_]).max()))
+            line["parity"] = {"samples": n, "J_max_rel_err": float(np.max(np.abs(Jg - Jo) / np.abs(Jo))),
+                              "r_max_err_over_max_abs_r": rerr / float(np.abs(ro).max()), "tolerance": 1e-5}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -46,11 +46,17 @@ __device__ void rowpoly_entry(const TableArgs& A, long long idx) {
     const double ga = 0.5 * (1.0 - 0.57735026918962576451);
     const double gb = 0.5 * (1.0 + 0.57735026918962576451);
     const double y = ((double)j + (q ? gb : ga)) / (double)(ny - 1);
+    // cos(jj pi y) from cos(pi y) by the Chebyshev recurrence in double, rounded to float as the cosine tables are
     double cy[MX], g[MX];
+    {
+        const double c1 = cospi(A.rp_nodes ? (double)j / (double)(ny - 1) : y);
+        double tm = 1.0, tc = c1;
 #pragma unroll
-    for (int jj = 0; jj < MX; ++jj) {
-        const double arg = A.rp_nodes ? (double)(jj + 1) * (double)j / (double)(ny - 1) : (double)(jj + 1) * y;   // as the tables
-        cy[jj] = (jj < m) ? (double)(float)cospi(arg) : 0.0;
+        for (int jj = 0; jj < MX; ++jj) {
+            cy[jj] = (jj < m) ? (double)(float)tc : 0.0;
+            const double tn = 2.0 * c1 * tc - tm;
+            tm = tc; tc = tn;
+        }
     }
     const float* w = A.kl_w + b * m * m;
 #pragma unroll
@@ -87,6 +93,7 @@ __device__ void rowpoly_entry(const TableArgs& A, long long idx) {
 }
 
 __global__ void tables_kernel(TableArgs A) {
+    dep_release();
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int m = A.m;
     long long mpow = 1;
@@ -137,6 +144,7 @@ __global__ void tables_kernel(TableArgs A) {
 // in a fixed order in double, rounded once to float.
 // ---------------------------------------------------------------------------------------
 __global__ void finalize_kernel(const double* __restrict__ partials, int nblk, float* __restrict__ J) {
+    dep_wait();
     const int b = blockIdx.x;
     const double* p = partials + 2ll * b * nblk;
     double d = 0.0, l = 0.0;
@@ -326,8 +334,7 @@ cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float*
 }
 
 cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s) {
-    finalize_kernel<<<batch, 256, 0, s>>>(partials, nblk, J);
-    return cudaGetLastError();
+    return launch_dependent(finalize_kernel, dim3((unsigned)batch), dim3(256), 0, s, partials, nblk, J);
 }
 
 cudaError_t launch_kl_field(const dn_grid& g, int batch, int m, const float* kl_w, float* nu, cudaStream_t s) {

@@ -147,7 +147,28 @@ struct HostPipe {
     }
 };
 
+// Launch of a kernel that may start before the kernel ahead of it in the stream has finished (programmatic
+// dependent launch): its blocks become resident as the blocks of that kernel retire, and it must not touch anything
+// that kernel writes, nor write anything it reads, before dep_wait() has returned.  Hides the launch latency and the
+// tail of the kernel ahead.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 #ifdef __CUDACC__
+// dep_wait(): everything the kernels ahead in the stream wrote is complete and visible (a no-op in a kernel that was
+// launched the ordinary way).  dep_release(): kernels launched behind this one with launch_dependent may become
+// resident from now on (they still wait in dep_wait() for this kernel to finish).
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Sum (d, l) over the block in a fixed order and let thread 0 store the pair.
 // Every thread of the block must call this.  blockDim.x * blockDim.y <= 1024.
 __device__ __forceinline__ void block_reduce_store(double d, double l, double* slot) {

@@ -77,6 +77,8 @@ template <int M, int BPS, int MODE>
 __global__ void __launch_bounds__(S2_WARPS * 32, BPS)
 strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, const int nchunk, const int nstrip) {
     extern __shared__ __align__(16) float smem[];
+    dep_wait();                                         // the tables of this call are complete
+    dep_release();                                      // the finaliser may move in behind the last wave
     constexpr int NE = S2_NE;
     constexpr int GS = s2_gs(M);
     // MODE 0: KL at the Gauss points; 1 (KN): KL at the nodes, then Q1 interpolation; 2 (ND): stored nodal field
@@ -429,8 +431,8 @@ cudaError_t launch_mk(const Params& P, const float* rowpoly, const GeoS& g, cuda
     const unsigned blocks = (unsigned)((units + S2_WARPS - 1) / S2_WARPS);
     const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    strip2d_kernel<M, 2, MODE><<<blocks, S2_WARPS * 32, smem, s>>>(P, rowpoly, g.R, g.nchunk, g.nstrip);
-    return cudaGetLastError();
+    return launch_dependent(strip2d_kernel<M, 2, MODE>, dim3(blocks), dim3(S2_WARPS * 32), smem, s, P, rowpoly, g.R, g.nchunk,
+                            g.nstrip);
 }
 
 template <int M>

@@ -198,6 +198,8 @@ template <int NX, int M, int MODE, int MINB>
 __global__ void __launch_bounds__(S3_WARPS * 32, MINB)
 strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G) {
     extern __shared__ __align__(16) float smem[];
+    dep_wait();                                         // the tables of this call are complete
+    dep_release();                                      // the fix-up kernel may move in as units finish
     constexpr bool KG = (MODE == 0), KN = (MODE == 1), ND = (MODE == 2);
     constexpr int GS = s3_gs(M);
     constexpr int CF = KG ? 2 * GS : KN ? GS : 0;       // coefficient floats per slot (KG: Gauss rows q = a, b of an element row)
@@ -600,6 +602,8 @@ template <int M>
 __global__ void __launch_bounds__(128) linepoly3d_kernel(const Params P, float* __restrict__ out) {
     constexpr int GS = s3_gs(M);
     __shared__ double h[2][M][M];                       // h[s][i][j] = sum_k ckl[i][j][k] cos(k pi z_s)
+    dep_wait();                                         // the scaled weights and cosine tables are complete
+    dep_release();
     const int ez = blockIdx.y, b = blockIdx.z;
     const float* w = P.ckl + (size_t)b * M * M * M;
     for (int t = threadIdx.x; t < 2 * M * M; t += blockDim.x) {
@@ -656,6 +660,8 @@ template <int M>
 __global__ void __launch_bounds__(128) nodepoly3d_kernel(const Params P, float* __restrict__ out) {
     constexpr int GS = s3_gs(M);
     __shared__ double h[M][M];                          // h[i][j] = sum_k ckl[i][j][k] cos(k pi z)
+    dep_wait();                                         // the scaled weights and cosine tables are complete
+    dep_release();
     const int iz = blockIdx.y, b = blockIdx.z;
     const float* w = P.ckl + (size_t)b * M * M * M;
     for (int t = threadIdx.x; t < M * M; t += blockDim.x) {
@@ -702,6 +708,8 @@ __global__ void __launch_bounds__(128) nodepoly3d_kernel(const Params P, float* 
 __global__ void seam_fixup3_kernel(float* __restrict__ r, const float* __restrict__ yseam, const float* __restrict__ zseam,
                                    int nx, int ny, int nz, int batch, int Ry, int ntile, int Z, int nchunk,
                                    long long nA, long long nB) {
+    dep_wait();                                         // the fused kernel has finished
+    dep_release();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int nx4 = nx / 4;
     const float4* zy = reinterpret_cast<const float4*>(zseam + (size_t)batch * (nchunk - 1) * ny * nx);
@@ -807,8 +815,7 @@ cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cu
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
     const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    strip3d_kernel<NX, M, MODE, MINB><<<blocks, S3_WARPS * 32, smem, s>>>(P, linepoly, g);
-    return cudaGetLastError();
+    return launch_dependent(strip3d_kernel<NX, M, MODE, MINB>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
 }
 
 template <int M>
@@ -871,12 +878,11 @@ template <int M>
 static cudaError_t launch_linepoly3d_m(const Params& P, float* linepoly, cudaStream_t s) {
     if (P.nu_mode == DN_NU_KL_NODAL) {
         const dim3 grid((unsigned)((P.ny + 127) / 128), (unsigned)P.nz, (unsigned)P.batch);
-        nodepoly3d_kernel<M><<<grid, 128, 0, s>>>(P, linepoly);
+        return launch_dependent(nodepoly3d_kernel<M>, grid, dim3(128), 0, s, P, linepoly);
     } else {
         const dim3 grid((unsigned)((P.ny - 1 + 127) / 128), (unsigned)(P.nz - 1), (unsigned)P.batch);
-        linepoly3d_kernel<M><<<grid, 128, 0, s>>>(P, linepoly);
+        return launch_dependent(linepoly3d_kernel<M>, grid, dim3(128), 0, s, P, linepoly);
     }
-    return cudaGetLastError();
 }
 
 cudaError_t launch_linepoly3d(const Params& P, float* linepoly, cudaStream_t s) {
@@ -912,9 +918,9 @@ cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t 
     const long long nA = (long long)P.batch * (g.ntile - 1) * P.nz * (P.nx / 4);
     const long long nB = (long long)P.batch * (g.nchunk - 1) * P.ny * (P.nx / 4);
     if (nA + nB > 0) {
-        seam_fixup3_kernel<<<(unsigned)((nA + nB + 255) / 256), 256, 0, s>>>(P.r, P.seam, P.zseam, P.nx, P.ny, P.nz, P.batch,
-                                                                            g.Ry, g.ntile, g.Z, g.nchunk, nA, nB);
-        return cudaGetLastError();
+        return launch_dependent(seam_fixup3_kernel, dim3((unsigned)((nA + nB + 255) / 256)), dim3(256), 0, s, P.r,
+                                (const float*)P.seam, (const float*)P.zseam, P.nx, P.ny, P.nz, P.batch, g.Ry, g.ntile, g.Z,
+                                g.nchunk, nA, nB);
     }
     return cudaSuccess;
 }
