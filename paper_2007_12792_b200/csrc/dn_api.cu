@@ -39,12 +39,14 @@ static long long nodes_per_sample(const dn_grid& g) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 Launch choose_launch(const dn_problem& p, const float* u, const float* r) {
-    const bool vec_ok = aligned16(u) && aligned16(r) && (p.nu_mode != DN_NU_NODAL || aligned16(p.nu));
-    if (!(p.flags & DN_FORCE_GENERIC) && vec_ok && p.f == nullptr) {
-        if (r && strip2d_applicable(p)) return strip2d_geometry(p);
-        if (r && strip3d_applicable(p)) return strip3d_geometry(p);
-        if (tiled2d_applicable(p)) return tiled2d_geometry(p);
-        if (tiled3d_applicable(p)) return tiled3d_geometry(p);
+    const bool vec_ok = aligned16(u) && aligned16(r) && (p.nu_mode != DN_NU_NODAL || aligned16(p.nu)) && aligned16(p.f);
+    if (!(p.flags & DN_FORCE_GENERIC) && vec_ok) {
+        if (r && strip2d_applicable(p)) return strip2d_geometry(p);      // also with nodal forcing
+        if (p.f == nullptr) {
+            if (r && strip3d_applicable(p)) return strip3d_geometry(p);
+            if (tiled2d_applicable(p)) return tiled2d_geometry(p);
+            if (tiled3d_applicable(p)) return tiled3d_geometry(p);
+        }
     }
     Launch l{};
     l.path = PATH_GENERIC;
@@ -425,8 +427,9 @@ int32_t dn_launches_per_call(const dn_problem* p) {
 
 const char* dn_path_name(const dn_problem* p) {
     if (validate(p) != DN_OK) return "invalid";
+    if (!(p->flags & DN_FORCE_GENERIC) && strip2d_applicable(*p))
+        return "strip2d";   // the fused call (also with nodal forcing); the energy-only call of such a problem runs tiled2d or, with nodal forcing, the any-size kernel
     if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr) {
-        if (strip2d_applicable(*p)) return "strip2d";      // the fused call; the energy-only call of such a problem runs tiled2d
         if (tiled2d_applicable(*p)) return "tiled2d";
         if (strip3d_applicable(*p)) return "strip3d";      // the fused call; the energy-only call runs tiled3d
         if (tiled3d_applicable(*p)) return "tiled3d";

@@ -73,7 +73,10 @@ template <int N> __device__ __forceinline__ void s2_wait() { asm volatile("cp.as
 // Floats per element row in the coefficient table: (row a, row b) pairs for k = 0..M, padded to a multiple of 4.
 __host__ __device__ constexpr int s2_gs(int m) { return (2 * (m + 1) + 3) / 4 * 4; }
 
-template <int M, int BPS, int MODE>
+// NF: nodal forcing.  The f row rides in the ring next to the u row; the load vector is the consistent mass matrix
+// applied to f, a 3 x 3 stencil that separates into a smoothing along x (neighbours by shuffle) and one along y (the row
+// below carried, the row above arriving), with the one-sided weights on the boundary nodes.
+template <int M, int BPS, int MODE, bool NF>
 __global__ void __launch_bounds__(S2_WARPS * 32, BPS)
 strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, const int nchunk, const int nstrip) {
     extern __shared__ __align__(16) float smem[];
@@ -83,10 +86,13 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
     constexpr int GS = s2_gs(M);
     // MODE 0: KL at the Gauss points; 1 (KN): KL at the nodes, then Q1 interpolation; 2 (ND): stored nodal field
     constexpr bool KN = (MODE == 1), ND = (MODE == 2);
-    // ring slot: node row of u, the 4 nodes right of it, then the coefficient row - or (ND) the same two pieces of nu
-    constexpr int S2_SLOT = ND ? 2 * S2_SLOT0 : S2_SLOT0, S2_DEPTH = ND ? S2_DEPTH0 / 2 : S2_DEPTH0;
+    // ring slot: node row of u, the 4 nodes right of it, then the coefficient row - or (ND) the same two pieces of nu;
+    // with nodal forcing the f row and the 4 nodes right of it follow
+    constexpr bool BIG = ND || NF;
+    constexpr int S2_SLOT = BIG ? 2 * S2_SLOT0 : S2_SLOT0, S2_DEPTH = BIG ? S2_DEPTH0 / 2 : S2_DEPTH0;
     constexpr int NUOFF = S2_COLS + 4;                  // ND: where the nu row starts inside a slot
-    static_assert(S2_COLS + 4 + GS <= S2_SLOT && 2 * (S2_COLS + 4) <= 2 * S2_SLOT0, "ring slot too small");
+    constexpr int FOFF = ND ? 2 * (S2_COLS + 4) : S2_COLS + 4 + GS;      // NF: where the f row starts
+    static_assert(S2_COLS + 4 + GS <= S2_SLOT0 && FOFF + S2_COLS + 4 <= 2 * S2_SLOT0, "ring slot too small");
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     float* ring = smem + (size_t)warp * S2_DEPTH * S2_SLOT;
@@ -121,8 +127,8 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
     }
     const float kx = 0.25f * P.hy / P.hx, ky = 0.25f * P.hx / P.hy;
     const float kxa = kx * DN_GA, kxb = kx * DN_GB, kya = ky * DN_GA, kyb = ky * DN_GB;
-    const float fw = P.f_const * P.hx * P.hy;           // nodal load of an interior node
-    const bool hasf = (P.f_const != 0.f);
+    const float fw = NF ? 0.f : P.f_const * P.hx * P.hy;   // nodal load of an interior node (constant forcing)
+    const bool hasf = !NF && (P.f_const != 0.f);
     const float gs = P.gJ ? __ldg(P.gJ + b) : 1.f;
 
     // Lane constants that make the march branch-free:
@@ -161,6 +167,7 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
     const float* usrc = ub + (size_t)(jbeg + 1) * nx;
     const bool xcoef = !ND && (lane < GS / 4), xhalo = (lane == 31) && has_halo;
     const float* nsrc = ND ? P.nu + (size_t)b * P.nodes + x0c + (size_t)(jbeg + 1) * nx : nullptr;
+    const float* fsrc = NF ? P.f + (size_t)b * P.nodes + x0c + (size_t)(jbeg + 1) * nx : nullptr;
     const int xp = (xcoef || xhalo) ? 1 : 0;            // this lane makes a second copy per row
     // coefficient rows: per element row (its two Gauss rows), or with KN per node row (the row that arrives with it)
     const float* polyb = rowpoly + (size_t)b * (KN ? ny : ny - 1) * GS;
@@ -175,10 +182,15 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
                 s2_cp16(slot + NUOFF + NE * lane, nsrc);
                 s2_cp16_if(slot + NUOFF + S2_COLS, nsrc + NE, xp);
             }
+            if constexpr (NF) {
+                s2_cp16(slot + FOFF + NE * lane, fsrc);
+                s2_cp16_if(slot + FOFF + S2_COLS, fsrc + NE, xhalo ? 1 : 0);
+            }
         }
         s2_commit();                                    // one group per step, possibly empty
         ++fetch; usrc += nx; xsrc += xstep;
         if constexpr (ND) nsrc += nx;
+        if constexpr (NF) fsrc += nx;
     };
 #pragma unroll
     for (int d = 0; d < S2_DEPTH - 1; ++d) issue(ring + d * S2_SLOT);
@@ -240,6 +252,39 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         for (int k = 0; k < NE; ++k) hnu[k] = nlo[k] + nlo[k + 1];
     }
 
+    // NF: x-smoothed forcing (hx/6) (f[k-1] + 4 f[k] + f[k+1]) of a node row, one-sided on the Dirichlet columns
+    const float m6x = P.hx * (1.f / 6.f), m6y = P.hy * (1.f / 6.f);
+    const float mxl = has_first ? 0.f : m6x, mxc0 = has_first ? 2.f * m6x : 4.f * m6x;     // node 0 of the lane
+    const float mxr = has_last ? 0.f : m6x, mxc3 = has_last ? 2.f * m6x : 4.f * m6x;       // node 3 of the lane
+    auto smooth_x = [&](const float (&f)[NE], const float fright, float (&g)[NE]) {
+        const float fleft = __shfl_up_sync(0xffffffffu, f[NE - 1], 1);   // lane 0: its own value, unused (mxl = 0 or a lane that stores nothing)
+        g[0] = fmaf(mxl, fleft, fmaf(mxc0, f[0], m6x * f[1]));
+        g[1] = m6x * (fmaf(4.f, f[1], f[0]) + f[2]);
+        g[2] = m6x * (fmaf(4.f, f[2], f[1]) + f[3]);
+        g[3] = fmaf(mxr, fright, fmaf(mxc3, f[3], m6x * f[2]));
+    };
+    float gf_lo[NE], gf_mid[NE];                        // smoothed f of the row below the current node row, and of that row
+#pragma unroll
+    for (int k = 0; k < NE; ++k) { gf_lo[k] = 0.f; gf_mid[k] = 0.f; }
+    if constexpr (NF) {
+        const float* fp = P.f + (size_t)b * P.nodes + x0c + (size_t)jbeg * nx;
+        const float4 q = __ldg(reinterpret_cast<const float4*>(fp));
+        const float f0[NE] = {q.x, q.y, q.z, q.w};
+        float halo = 0.f;
+        if (xhalo) halo = __ldg(fp + NE);
+        float fr = __shfl_down_sync(0xffffffffu, f0[0], 1);
+        if (lane == 31) fr = halo;
+        smooth_x(f0, fr, gf_mid);
+        if (jbeg > 0) {                                 // the row below the unit's first row (uniform)
+            const float4 q1 = __ldg(reinterpret_cast<const float4*>(fp - nx));
+            const float f1[NE] = {q1.x, q1.y, q1.z, q1.w};
+            float h1 = 0.f;
+            if (xhalo) h1 = __ldg(fp - nx + NE);
+            float fr1 = __shfl_down_sync(0xffffffffu, f1[0], 1);
+            if (lane == 31) fr1 = h1;
+            smooth_x(f1, fr1, gf_lo);
+        }
+    }
     float en = 0.f, ell = 0.f;                          // sum u (K u) and sum w u of the rows this lane went over
     float* rrow = rb + (size_t)jbeg * nx;
     int rd = 0;                                         // float offset of the slot to read; the one before it is refilled
@@ -331,12 +376,32 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         const float tl = __shfl_up_sync(0xffffffffu, Tp, 1);
         rout[0] = fmaf(-ky, SY0, fmaf(ql, lm, -Q0)) + U[0];
         U[0] = fmaf(tl, lm, R0);
+        float gf_up[NE];                                // NF: smoothed f of node row j + 1
+        if constexpr (NF) {
+            const float4 q = *reinterpret_cast<const float4*>(slot + FOFF + NE * lane);
+            const float fu[NE] = {q.x, q.y, q.z, q.w};
+            const float fh = slot[FOFF + S2_COLS];
+            float fr = __shfl_down_sync(0xffffffffu, fu[0], 1);
+            if (lane == 31) fr = has_halo ? fh : 0.f;
+            smooth_x(fu, fr, gf_up);
+        }
         if (j >= n0) {                                  // uniform: this unit owns node row j
             // rout is (K u) of node row j: Euler's identity gives the diffusion energy
 #pragma unroll
             for (int k = 0; k < NE; ++k) en = fmaf(a[k], rout[k], en);
             float4 o;
-            if (hasf) {
+            if constexpr (NF) {
+                // load of node row j: the y-smoothing of the three smoothed rows (row 0 has no row below)
+                const float wc = (j == 0) ? 2.f * m6y : 4.f * m6y;
+                float F[NE];
+#pragma unroll
+                for (int k = 0; k < NE; ++k) {
+                    F[k] = fmaf(m6y, gf_lo[k] + gf_up[k], wc * gf_mid[k]);
+                    ell = fmaf(a[k], F[k], ell);
+                }
+                o.x = gsf * (rout[0] - F[0]); o.y = gs * (rout[1] - F[1]);
+                o.z = gs * (rout[2] - F[2]); o.w = gsl * (rout[3] - F[3]);
+            } else if (hasf) {
                 const float wrow = (j == 0) ? 0.5f : 1.f;
                 ell = fmaf(wrow, fmaf(a[0], wf, a[1]) + fmaf(a[NE - 1], wl, a[2]), ell);
                 o.x = fmaf(gsf, rout[0], wrow * nlf); o.y = fmaf(gs, rout[1], wrow * nl);
@@ -347,6 +412,10 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             if (owner) *reinterpret_cast<float4*>(rrow) = o;
         }
         rrow += nx;
+        if constexpr (NF) {
+#pragma unroll
+            for (int k = 0; k < NE; ++k) { gf_lo[k] = gf_mid[k]; gf_mid[k] = gf_up[k]; }
+        }
         if constexpr (KN || ND) {
 #pragma unroll
             for (int k = 0; k <= NE; ++k) nlo[k] = ncur[k];
@@ -372,15 +441,26 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
     if (n1 == ny) {
 #pragma unroll
         for (int k = 0; k < NE; ++k) en = fmaf(lo[k], U[k], en);
-        ell = fmaf(0.5f, fmaf(lo[0], wf, lo[1]) + fmaf(lo[NE - 1], wl, lo[2]), ell);
         float4 o;
-        o.x = fmaf(gsf, U[0], 0.5f * nlf); o.y = fmaf(gs, U[1], 0.5f * nl);
-        o.z = fmaf(gs, U[2], 0.5f * nl); o.w = fmaf(gsl, U[3], 0.5f * nll);
+        if constexpr (NF) {
+            float F[NE];
+#pragma unroll
+            for (int k = 0; k < NE; ++k) {              // the top row: one-sided in y
+                F[k] = m6y * fmaf(2.f, gf_mid[k], gf_lo[k]);
+                ell = fmaf(lo[k], F[k], ell);
+            }
+            o.x = gsf * (U[0] - F[0]); o.y = gs * (U[1] - F[1]); o.z = gs * (U[2] - F[2]); o.w = gsl * (U[3] - F[3]);
+        } else {
+            ell = fmaf(0.5f, fmaf(lo[0], wf, lo[1]) + fmaf(lo[NE - 1], wl, lo[2]), ell);
+            o.x = fmaf(gsf, U[0], 0.5f * nlf); o.y = fmaf(gs, U[1], 0.5f * nl);
+            o.z = fmaf(gs, U[2], 0.5f * nl); o.w = fmaf(gsl, U[3], 0.5f * nll);
+        }
         if (owner) *reinterpret_cast<float4*>(rb + (size_t)(ny - 1) * nx) = o;
     }
 
     // ---- energy partial of this unit: owning lanes summed in a fixed order in double
-    double d = owner ? 0.5 * (double)en : 0.0, l = (owner && hasf) ? (double)fw * (double)ell : 0.0;
+    double d = owner ? 0.5 * (double)en : 0.0;
+    double l = !owner ? 0.0 : NF ? (double)ell : hasf ? (double)fw * (double)ell : 0.0;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         d += __shfl_down_sync(0xffffffffu, d, o);
@@ -424,15 +504,20 @@ GeoS geometry_s(const dn_problem& p) {
     return g;
 }
 
-template <int M, int MODE>
-cudaError_t launch_mk(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
+template <int M, int MODE, bool NF>
+cudaError_t launch_mkf(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
     const size_t smem = sizeof(float) * S2_WARPS * S2_DEPTH0 * S2_SLOT0;
     const long long units = (long long)P.batch * g.nchunk * g.nstrip;
     const unsigned blocks = (unsigned)((units + S2_WARPS - 1) / S2_WARPS);
-    const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2, MODE, NF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(strip2d_kernel<M, 2, MODE>, dim3(blocks), dim3(S2_WARPS * 32), smem, s, P, rowpoly, g.R, g.nchunk,
-                            g.nstrip);
+    return launch_dependent(strip2d_kernel<M, 2, MODE, NF>, dim3(blocks), dim3(S2_WARPS * 32), smem, s, P, rowpoly, g.R,
+                            g.nchunk, g.nstrip);
+}
+
+template <int M, int MODE>
+cudaError_t launch_mk(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
+    return P.f ? launch_mkf<M, MODE, true>(P, rowpoly, g, s) : launch_mkf<M, MODE, false>(P, rowpoly, g, s);
 }
 
 template <int M>
@@ -446,7 +531,7 @@ cudaError_t launch_m(const Params& P, const float* rowpoly, const GeoS& g, cudaS
 // row takes 3 strips of 128).  The tiled kernel is about 1.16 times slower per element in this mode: the strip
 // kernel takes over where its lanes are at most 15 % more than the row, and wherever the tiled kernel cannot run.
 bool strip2d_applicable(const dn_problem& p) {
-    if (!(p.grid.dim == 2 && p.f == nullptr && p.grid.nx % 4 == 0 &&
+    if (!(p.grid.dim == 2 && p.grid.nx % 4 == 0 &&
           p.grid.nx >= 2 * S2_COLS && p.grid.ny >= 16))
         return false;
     const long long lanes = (long long)((p.grid.nx - S2_COLS + S2_STRIDE - 1) / S2_STRIDE + 1) * S2_COLS;

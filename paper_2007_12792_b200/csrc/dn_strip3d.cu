@@ -205,8 +205,9 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     constexpr int CF = KG ? 2 * GS : KN ? GS : 0;       // coefficient floats per slot (KG: Gauss rows q = a, b of an element row)
     constexpr int CFQ = CF / 4;                         // ... in 16-byte pieces
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int LW = G.LW, SUBS = 32 >> G.lwsh;
-    const int sub = lane >> G.lwsh, lx = lane & (LW - 1);
+    // 8 nodes per lane are used on rows of more than 128 nodes only: then a unit is a whole warp
+    const int LW = (NX == 8) ? 32 : G.LW, lwsh = (NX == 8) ? 5 : G.lwsh, SUBS = 32 >> lwsh;
+    const int sub = lane >> lwsh, lx = lane & (LW - 1);
     const unsigned submask = (LW == 32) ? 0xffffffffu : (((1u << LW) - 1u) << (sub * LW));
     const int nx = P.nx, ny = P.ny, nz = P.nz;
     const int x0 = NX * lx;
@@ -218,7 +219,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     float4* cps = reinterpret_cast<float4*>(smem);
     if constexpr (KG) {
         for (int i = threadIdx.x; i < NX * LW; i += blockDim.x) {
-            const int c = i >> G.lwsh, l = i & (LW - 1);
+            const int c = i >> lwsh, l = i & (LW - 1);
             const int xe = min(NX * l, nx - NX) + c;    // element index = index of its left node
             const float ca = __ldg(P.cg[0] + 2 * xe), cb = __ldg(P.cg[0] + 2 * xe + 1);
             cps[i] = make_float4(ca, ca, cb, cb);

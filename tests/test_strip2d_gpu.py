@@ -95,3 +95,23 @@ def test_strip2d_determinism_and_stale_workspace():
         outs.append((J.cpu().numpy().copy(), r.cpu().numpy().copy()))
     for J, r in outs[1:]:
         assert J.tobytes() == outs[0][0].tobytes() and r.tobytes() == outs[0][1].tobytes()
+
+
+@pytest.mark.parametrize("mode", KL_MODES)
+@pytest.mark.parametrize("nx,ny,batch,m", [(1024, 40, 2, 4), (1120, 16, 2, 2), (1124, 21, 1, 3), (2052, 37, 1, 7), (1024, 300, 5, 2)])
+def test_strip2d_nodal_forcing(nx, ny, batch, m, mode):
+    """Nodal forcing on the strip kernel: the load vector is the consistent mass matrix applied to f (the f row rides in the
+    ring with the u row).  All flag combinations, because the Dirichlet columns take the one-sided mass weights."""
+    inp = inputs.random_inputs(2, nx, ny, 1, batch, m, seed=17 + nx + ny)
+    u = inputs.random_field(inp.u.shape, 4)
+    f = inputs.random_field(inp.u.shape, 9, scale=3.0)
+    nu = inputs.random_positive_field(inp.u.shape, 5) if mode == B.DN_NU_NODAL else None
+    gJ = np.linspace(-1.5, 2.0, batch).astype(np.float32)
+    for flags in (0, B.DN_NO_MASK, B.DN_IMPOSE_BC_ON_LOAD):
+        po, pg = make_problems(inp, mode, nu=nu, f=f, flags=flags, bc=(0.8, -0.3))
+        assert B.dn_path_name(pg) == "strip2d"
+        Jo, _, _, ro = oracle.energy_grad(po, u, gJ=gJ.astype(np.float64))
+        Jg, rg = run_gpu(pg, u, gJ=gJ)
+        check(Jg, rg, Jo, ro, f"nodal f, flags={flags}")
+        if not (flags & B.DN_NO_MASK):
+            assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
