@@ -240,7 +240,13 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     if (su >= G.units) return;                          // the other units of the warp synchronise among themselves only
     const int C = G.C, RS = G.RS;
     const unsigned RSB = (unsigned)RS * 4u, RINGB = (unsigned)C * RSB;
-    float* ring = smem + (KG ? 4 * NX * LW : 0) + (size_t)(warp * SUBS + sub) * C * RS;
+    // PREF (wide rows): the parked sums of a node row come back through shared memory, copied one step ahead of their
+    // use; narrow rows load them directly (the copy cost more than it hid there: 83 against 77 us on 64^3 x 32)
+    constexpr bool PREF = (NX == 8);
+    float* ring = smem + (KG ? 4 * NX * LW : 0) + (size_t)(warp * SUBS + sub) * (C * RS + (PREF ? NX * LW : 0));
+    // behind the ring: one row of parked sums (each lane its own pieces)
+    float* cbuf = ring + (size_t)C * RS + 4 * lx;
+    const unsigned cbuf_s = (unsigned)__cvta_generic_to_shared(cbuf);
     const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring);
     const int UROW = NX * LW + 4;                       // floats of a node row in a slot (with the 4 floats of padding)
     const int COEF = KG ? UROW : 2 * UROW;              // offset of the coefficient row inside a slot
@@ -413,14 +419,38 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
         for (int c = 0; c < NX; ++c) { pendL1[c] = 0.f; pendU1[c] = 0.f; }
         float* rlo = rb + ((size_t)k * ny + y0) * nx;
         float* rup = last ? ztop : rlo + plane;
+        float* ptoplo = lasttile ? rlo + (size_t)(T - 1) * nx : sb + (size_t)k * nx;   // where the tile's top row is finished
+        // The sums parked for a node row one plane ago come back through shared memory, copied one step ahead (this
+        // thread stored them long ago; the copy reads them from L2 while the elements of the row before are computed).
+        auto fetch_parked = [&](const float* p) {
+            s3_cp16s(cbuf_s, p);
+            if constexpr (NX == 8) s3_cp16s(cbuf_s + 16u * LW, p + 4);
+            s3_commit();
+        };
+        auto read_parked = [&](float (&v)[NX]) {
+            const float4 q = *reinterpret_cast<const float4*>(cbuf);
+            v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+            if constexpr (NX == 8) {
+                const float4 q1 = *reinterpret_cast<const float4*>(cbuf + 4 * LW);
+                v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+            }
+        };
+        if (PREF && hascarry) fetch_parked(rlo);
         for (int jj = 0; jj + 1 < T; ++jj) {
             s3_wait<0>();                               // everything issued up to the previous step has landed ...
             __syncwarp(submask);                        // ... is visible to the unit, and the rows it retired are free
-            while (pf < n + C) issue();
             float cin[NX];
 #pragma unroll
             for (int c = 0; c < NX; ++c) cin[c] = 0.f;
-            if (hascarry) ld4(rlo, cin);
+            if (hascarry) {
+                if constexpr (PREF) {
+                    read_parked(cin);
+                    fetch_parked((jj + 2 < T) ? rlo + nx : ptoplo);
+                } else {
+                    ld4(rlo, cin);
+                }
+            }
+            while (pf < n + C) issue();
             const unsigned oB = wrapb(oA + RSB), oC = wrapb(oA + TB), oD = wrapb(oC + RSB);
             const float wy = (y0 + jj == 0) ? 0.5f : 1.f;
             float uA[NX + 1], uB[NX + 1], uC[NX + 1], uD[NX + 1];
@@ -515,14 +545,21 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
         {
             float uA[NX + 1];
             ldrow(oA, uA);
-            float* plo = lasttile ? rlo : sb + (size_t)k * nx;
+            float* plo = ptoplo;
             float* pup = lasttile ? rup : last ? zstop : plo + nx;
             const float wy = lasttile ? 0.5f : 0.f;
             const float nlrow = nllo * wy;
             float cin[NX], olo[NX];
 #pragma unroll
             for (int c = 0; c < NX; ++c) cin[c] = 0.f;
-            if (hascarry) ld4(plo, cin);
+            if (hascarry) {
+                if constexpr (PREF) {
+                    s3_wait<0>();
+                    read_parked(cin);
+                } else {
+                    ld4(plo, cin);
+                }
+            }
 #pragma unroll
             for (int c = 0; c < NX; ++c) {
                 const float raw = pendL1[c] + cin[c];
@@ -782,6 +819,7 @@ S3Geo geometry3s(const dn_problem& p) {
     size_t per_block = (S3_SMEM_SM - (size_t)minb * 1024) / minb;
     if (per_block > S3_SMEM_BLOCK) per_block = S3_SMEM_BLOCK;
     if (p.nu_mode == DN_NU_KL_GAUSS) per_block -= sizeof(float) * 4 * NX * g.LW;      // the block's table of cosine pairs
+    if (NX == 8) per_block -= sizeof(float) * S3_WARPS * subs * NX * g.LW;   // one row of parked sums per unit
     const int cmax = (int)(per_block / ((size_t)S3_WARPS * subs * g.RS * sizeof(float)));
     int ry_max = cmax - 2 - S3_D;
     if (ry_max > ny - 1) ry_max = ny - 1;
@@ -811,7 +849,7 @@ S3Geo geometry3s(const dn_problem& p) {
 template <int NX, int M, int MODE, int MINB>
 cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
     const int subs = 32 / g.LW;
-    const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * g.C * g.RS + (MODE == 0 ? 4 * NX * g.LW : 0));
+    const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * (g.C * g.RS + (NX == 8 ? NX * g.LW : 0)) + (MODE == 0 ? 4 * NX * g.LW : 0));
     const long long per_block = (long long)S3_WARPS * subs;
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
     const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
