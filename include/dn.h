@@ -94,8 +94,9 @@ typedef struct {
 } dn_problem;
 
 /* Bytes of device scratch that dn_energy / dn_energy_grad need for this problem (per-block
- * energy partials, cosine tables and, for 3D grids, the contributions exchanged across tile seams:
- * about 1/4 of one field).  0 if the problem is invalid.  The workspace must be
+ * energy partials, cosine and coefficient tables and, for 3D grids, the contributions exchanged across
+ * tile and chunk seams: up to about 1/3 of one field, plus 16 floats per element row of the grid for the
+ * coefficient table of the KL modes).  0 if the problem is invalid.  The workspace must be
  * 256-byte aligned; its contents need not be preserved between calls, and two calls that
  * may overlap on the device need separate workspaces. */
 size_t dn_workspace_bytes(const dn_problem* problem);
@@ -124,7 +125,8 @@ dn_status dn_energy(const dn_problem* problem, const float* u, float* J, void* w
  * Errors found before anything is enqueued come back as a status and leave the outputs untouched.
  * The kernels contain no unbounded wait: where warps of the tiled 2D kernel hand values to one
  * another, the wait has an iteration limit, and should it ever run out the energy J[b] of that
- * sample is returned as NaN (its residual is then not to be trusted either). */
+ * sample is returned as NaN (its residual is then not to be trusted either; a residual-only call, J == NULL,
+ * cannot report it: pass J where that check matters). */
 dn_status dn_energy_grad(const dn_problem* problem, const float* u, const float* gJ, float* J, float* r,
                          void* workspace, size_t workspace_bytes, void* stream);
 
@@ -254,7 +256,7 @@ const char* dn_burgers_path_name(const dn_burgers* problem, const float* u, cons
  * dn_energy_grad call (for launch accounting); 0 if the problem is invalid. */
 int32_t dn_launches_per_call(const dn_problem* problem);
 
-/* Name of the kernel family that dn_energy_grad would use ("strip2d", "tiled2d", "tiled3d", "generic"). */
+/* Name of the kernel family that dn_energy_grad would use ("strip2d", "strip3d", "tiled2d", "tiled3d", "generic"). */
 const char* dn_path_name(const dn_problem* problem);
 
 const char* dn_status_string(dn_status status);
