@@ -192,7 +192,7 @@ dn_status dn_energy_grad_host(const dn_problem* problem, const float* u_host, co
  *    fallen to rtol times its initial value stops changing.  relres_out: [B] floats = |r| / |r0| reached,
  *    iters_out: [B] int32 = iterations a sample took part in; either may be NULL.
  *  - problem->flags: DN_FORCE_GENERIC is honoured, the other flags are ignored.
- *  - workspace: dn_cg_workspace_bytes(problem) bytes (four fields + dn_workspace_bytes), 256-byte aligned. */
+ *  - workspace: dn_cg_workspace_bytes(problem) bytes (four fields + two fused-kernel workspaces), 256-byte aligned. */
 size_t dn_cg_workspace_bytes(const dn_problem* problem);
 dn_status dn_cg_solve(const dn_problem* problem, float* u_inout, int32_t max_iters, float rtol,
                       float* relres_out, int32_t* iters_out, void* workspace, size_t workspace_bytes,

@@ -41,9 +41,9 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 Launch choose_launch(const dn_problem& p, const float* u, const float* r) {
     const bool vec_ok = aligned16(u) && aligned16(r) && (p.nu_mode != DN_NU_NODAL || aligned16(p.nu)) && aligned16(p.f);
     if (!(p.flags & DN_FORCE_GENERIC) && vec_ok) {
-        if (r && strip2d_applicable(p)) return strip2d_geometry(p);      // also with nodal forcing
+        if (r && strip2d_applicable(p)) return strip2d_geometry(p);      // the strip kernels also take nodal forcing
+        if (r && strip3d_applicable(p)) return strip3d_geometry(p);
         if (p.f == nullptr) {
-            if (r && strip3d_applicable(p)) return strip3d_geometry(p);
             if (tiled2d_applicable(p)) return tiled2d_geometry(p);
             if (tiled3d_applicable(p)) return tiled3d_geometry(p);
         }
@@ -419,7 +419,7 @@ dn_status dn_energy_grad_host(const dn_problem* p, const float* u_host, const fl
 int32_t dn_launches_per_call(const dn_problem* p) {
     if (validate(p) != DN_OK) return 0;
     const bool fast = !(p->flags & DN_FORCE_GENERIC) && p->f == nullptr;
-    if (fast && strip3d_applicable(*p))                 // (tables, line polynomials,) fused kernel, seam fix-up, finaliser
+    if (!(p->flags & DN_FORCE_GENERIC) && strip3d_applicable(*p))                 // (tables, line polynomials,) fused kernel, seam fix-up, finaliser
         return 2 + (p->nu_mode != DN_NU_NODAL ? 2 : 0) + ((strip3d_seam_floats(*p) + strip3d_zseam_floats(*p)) > 0 ? 1 : 0);
     const bool t3 = fast && !tiled2d_applicable(*p) && tiled3d_applicable(*p);
     return 2 + (p->nu_mode != DN_NU_NODAL ? 1 : 0) + ((t3 && tiled3d_seam_floats(*p) > 0) ? 1 : 0);
@@ -427,13 +427,12 @@ int32_t dn_launches_per_call(const dn_problem* p) {
 
 const char* dn_path_name(const dn_problem* p) {
     if (validate(p) != DN_OK) return "invalid";
-    if (!(p->flags & DN_FORCE_GENERIC) && strip2d_applicable(*p))
-        return "strip2d";   // the fused call (also with nodal forcing); the energy-only call of such a problem runs tiled2d or, with nodal forcing, the any-size kernel
-    if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr) {
-        if (tiled2d_applicable(*p)) return "tiled2d";
-        if (strip3d_applicable(*p)) return "strip3d";      // the fused call; the energy-only call runs tiled3d
-        if (tiled3d_applicable(*p)) return "tiled3d";
-    }
+    // the fused call (the strip kernels also with nodal forcing); the energy-only call of such a problem runs the tiled
+    // kernel of its dimension or, with nodal forcing, the any-size kernel
+    if (!(p->flags & DN_FORCE_GENERIC) && strip2d_applicable(*p)) return "strip2d";
+    if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && tiled2d_applicable(*p)) return "tiled2d";
+    if (!(p->flags & DN_FORCE_GENERIC) && strip3d_applicable(*p)) return "strip3d";
+    if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && tiled3d_applicable(*p)) return "tiled3d";
     return "generic";
 }
 

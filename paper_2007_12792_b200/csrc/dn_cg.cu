@@ -198,7 +198,7 @@ __global__ void cg_report_kernel(const CgScalars* __restrict__ sc, int batch, fl
 long long nodes_of(const dn_problem& p) { return (long long)p.grid.nx * p.grid.ny * (p.grid.dim == 3 ? p.grid.nz : 1); }
 int vec_blocks(long long nodes) { return (int)((nodes + CG_BLOCK_NODES - 1) / CG_BLOCK_NODES); }
 
-struct CgLayout { size_t r, q, p, dinv, partials, scalars, op, total; };
+struct CgLayout { size_t r, q, p, dinv, partials, scalars, op, op_bytes, op1, op1_bytes, total; };
 
 CgLayout cg_layout(const dn_problem& p) {
     CgLayout L{};
@@ -210,10 +210,14 @@ CgLayout cg_layout(const dn_problem& p) {
     L.dinv = off; off += field;
     L.partials = off; off += align_up(sizeof(double) * 2 * (size_t)p.batch * vec_blocks(nodes_of(p)));
     L.scalars = off; off += align_up(sizeof(CgScalars) * (size_t)p.batch);
-    dn_problem pop = p;                      // the operator on directions has no nodal forcing and may take a kernel
-    pop.f = nullptr;                         // family with a larger workspace than the caller's problem
-    const size_t a = dn_workspace_bytes(&p), b = dn_workspace_bytes(&pop);
-    L.op = off; off += (a > b) ? a : b;
+    // Two fused-kernel workspaces: one for the operator on directions (no nodal forcing, aligned scratch fields) and one
+    // for the caller's problem (initial residual), which may take another kernel family with another layout.
+    dn_problem pop = p;
+    pop.f = nullptr;
+    L.op_bytes = dn_workspace_bytes(&pop);
+    L.op = off; off += align_up(L.op_bytes);
+    L.op1_bytes = dn_workspace_bytes(&p);
+    L.op1 = off; off += align_up(L.op1_bytes);
     L.total = off;
     return L;
 }
@@ -249,7 +253,9 @@ dn_status dn_cg_solve(const dn_problem* p, float* u, int32_t max_iters, float rt
     double* partials = reinterpret_cast<double*>(base + L.partials);
     CgScalars* sc = reinterpret_cast<CgScalars*>(base + L.scalars);
     void* op_ws = base + L.op;
-    const size_t op_bytes = ws_bytes - L.op;
+    const size_t op_bytes = L.op_bytes;
+    void* op1_ws = base + L.op1;
+    const size_t op1_bytes = L.op1_bytes;
     const long long nodes = nodes_of(*p);
     const int nvb = vec_blocks(nodes);
     const dim3 vgrid((unsigned)nvb, (unsigned)p->batch);
@@ -263,12 +269,11 @@ dn_status dn_cg_solve(const dn_problem* p, float* u, int32_t max_iters, float rt
     // the operator on directions: zero forcing, zero boundary values, same diffusivity
     dn_problem p0 = p1;
     p0.f = nullptr; p0.f_const = 0.0f; p0.bc_x0 = 0.0f; p0.bc_x1 = 0.0f; p0.bc_x0_b = nullptr; p0.bc_x1_b = nullptr;
-    // The KL tables are built once, for the kernel family the direction operator takes (aligned scratch fields, no
-    // nodal forcing: the family that needs the most, e.g. the strip kernel's per-row polynomials); the caller's
-    // problem may run on another family (nodal forcing, unaligned u), which reads a subset of the same tables.
+    // The KL tables are built once per solve for the direction operator (aligned scratch fields, no nodal forcing); the
+    // caller's problem is applied once, in a workspace of its own with its own tables (it may take another family).
     st = build_tables(&p0, pd, q, op_ws, op_bytes, s);
     if (st != DN_OK) return st;
-    st = run_operator(&p1, u, r, op_ws, op_bytes, s, false, nullptr, nullptr);
+    st = run_operator(&p1, u, r, op1_ws, op1_bytes, s, true, nullptr, nullptr);
     if (st != DN_OK) return st;
     {   // Jacobi preconditioner: the diagonal of K, one colour class per application (p and q serve as scratch)
         const int nz = p->grid.dim == 3 ? p->grid.nz : 1;

@@ -535,7 +535,7 @@ bool strip2d_applicable(const dn_problem& p) {
           p.grid.nx >= 2 * S2_COLS && p.grid.ny >= 16))
         return false;
     const long long lanes = (long long)((p.grid.nx - S2_COLS + S2_STRIDE - 1) / S2_STRIDE + 1) * S2_COLS;
-    return !tiled2d_applicable(p) || 100 * lanes <= 115ll * p.grid.nx;
+    return !tiled2d_applicable(p) || 100 * lanes <= 115ll * p.grid.nx || p.f != nullptr;   // nodal forcing: the only fast kernel
 }
 
 Launch strip2d_geometry(const dn_problem& p) {

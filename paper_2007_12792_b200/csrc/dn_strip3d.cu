@@ -140,6 +140,18 @@ __device__ __forceinline__ void s3_bilerp(const float h00, const float h10, cons
     out[2] = fmaf(DN_GA, db, mb0); out[3] = fmaf(DN_GB, db, mb0);
 }
 
+// Nodal forcing: the element mass matrix applied to the 8 corner values of f, by sum factorisation (per axis the
+// matrix [[2, 1], [1, 2]]; the factor hx hy hz / 216 is applied by the caller).  f and m are indexed i + 2j + 4k.
+__device__ __forceinline__ void s3_mass(const float (&f)[8], float (&m)[8]) {
+    float g[8], h[8];
+#pragma unroll
+    for (int t = 0; t < 8; t += 2) { g[t] = fmaf(2.f, f[t], f[t + 1]); g[t + 1] = fmaf(2.f, f[t + 1], f[t]); }          // x
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { if (t & 2) continue; h[t] = fmaf(2.f, g[t], g[t + 2]); h[t + 2] = fmaf(2.f, g[t + 2], g[t]); }   // y
+#pragma unroll
+    for (int t = 0; t < 4; ++t) { m[t] = fmaf(2.f, h[t], h[t + 4]); m[t + 4] = fmaf(2.f, h[t + 4], h[t]); }               // z
+}
+
 // The element: from the 12 sums of nu and the 7 hierarchical coordinates of u to the 8 corner contributions
 // r[i + 2j + 4k] (i, j, k the x, y, z bits of the corner), all in units of kap = hx hy hz / (8 h^2) on isotropic cells
 // (iso), else scaled by kx, ky, kz here.
@@ -194,7 +206,10 @@ __device__ __forceinline__ void s3_element(const float (&Nx)[4], const float (&N
 // In the nodal modes a slot of the ring holds the nu row next to the u row: copied from the field (ND), or computed
 // from the polynomial of that node line when the row is first used (KN: the table then holds one polynomial per node
 // line, every coefficient twice, and travels with the row itself).
-template <int NX, int M, int MODE, int MINB>
+// NF: nodal forcing.  The f row sits in the slot as well; the load is taken element by element (mass matrix applied
+// to the corner values of f) and joins the corner contributions before they are gathered, so it needs no other
+// treatment at the boundary of the domain, a tile or a chunk than the stiffness part.
+template <int NX, int M, int MODE, bool NF, int MINB>
 __global__ void __launch_bounds__(S3_WARPS * 32, MINB)
 strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G) {
     extern __shared__ __align__(16) float smem[];
@@ -249,7 +264,8 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const unsigned cbuf_s = (unsigned)__cvta_generic_to_shared(cbuf);
     const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring);
     const int UROW = NX * LW + 4;                       // floats of a node row in a slot (with the 4 floats of padding)
-    const int COEF = KG ? UROW : 2 * UROW;              // offset of the coefficient row inside a slot
+    const int FOFF = KG ? UROW : 2 * UROW;              // offset of the f row (nodal forcing)
+    const int COEF = FOFF + (NF ? UROW : 0);            // offset of the coefficient row inside a slot
     const int H1 = 4 * LW + 4;                          // NX = 8: offset of the second 16 bytes of every lane
 
     const int b = (int)(su % P.batch);
@@ -289,8 +305,10 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const float kx = W8 / (P.hx * P.hx), ky = W8 / (P.hy * P.hy), kz = W8 / (P.hz * P.hz);
     const float kap = iso ? kx : 1.f;                   // isotropic cells: one scale applied at the end
     const float gs = P.gJ ? __ldg(P.gJ + b) : 1.f;
-    const float fw = P.f_const * P.hx * P.hy * P.hz;    // nodal load of an interior node
-    const bool hasf = (P.f_const != 0.f);
+    const float fw = NF ? 0.f : P.f_const * P.hx * P.hy * P.hz;    // nodal load of an interior node (constant forcing)
+    const bool hasf = !NF && (P.f_const != 0.f);
+    const float fsabs = P.hx * P.hy * P.hz * (1.f / 216.f);        // NF: scale of the element mass matrix ...
+    const float fs = fsabs / kap;                                   // ... in the units the corner contributions are kept in
     // Lane constants that keep the finish of a node row branch-free: output scale, share of the nodal load and
     // weight in the load energy of the lane's first / last node (Dirichlet columns: masked, or with DN_NO_MASK
     // carrying half a load); g3 = 0 in the lane whose last element lies right of node nx-1 (it does not exist).
@@ -306,6 +324,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     for (int s = lx; s < C; s += LW) {                  // the 4 floats right of the last lane's nodes stay zero
         *reinterpret_cast<float4*>(ring + (size_t)s * RS + 4 * LW) = make_float4(0.f, 0.f, 0.f, 0.f);
         if constexpr (!KG) *reinterpret_cast<float4*>(ring + (size_t)s * RS + UROW + 4 * LW) = make_float4(0.f, 0.f, 0.f, 0.f);
+        if constexpr (NF) *reinterpret_cast<float4*>(ring + (size_t)s * RS + FOFF + 4 * LW) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     int pf = 0, pfj = 0, pfk = 0;
     unsigned pfo = 0;                                   // byte offset of the slot the next entry goes to
@@ -316,6 +335,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const float* csrc = KG ? linepoly + (((size_t)b * (nz - 1) + kbeg) * (ny - 1) + y0) * CF - ((size_t)(ny - 1) + 1) * CF + 4 * clx
                            : linepoly + (((size_t)b * nz + kbeg) * ny + y0) * CF + 4 * clx;
     const float* nsrc = ND ? P.nu + (size_t)b * P.nodes + x0c + (size_t)kbeg * plane + (size_t)y0 * nx : nullptr;
+    const float* fsrc = NF ? P.f + (size_t)b * P.nodes + x0c + (size_t)kbeg * plane + (size_t)y0 * nx : nullptr;
     const long long uwrap = (long long)plane - (long long)T * nx, cwrap = ((long long)(KG ? ny - 1 : ny) - T) * CF;
     const unsigned d0 = ring_s + 16u * lx, d1 = ring_s + 4u * H1 + 16u * lx, dc = ring_s + 4u * COEF + 16u * clx;
     auto issue = [&]() {
@@ -326,6 +346,10 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                 s3_cp16s(d0 + 4u * UROW + pfo, nsrc);
                 if constexpr (NX == 8) s3_cp16s(d1 + 4u * UROW + pfo, nsrc + 4);
             }
+            if constexpr (NF) {
+                s3_cp16s(d0 + 4u * FOFF + pfo, fsrc);
+                if constexpr (NX == 8) s3_cp16s(d1 + 4u * FOFF + pfo, fsrc + 4);
+            }
             if constexpr (CF > 0) {
                 const int cok = (KN || (pfk >= 1 && pfj >= 1)) ? 1 : 0;
                 s3_cp16s_if(dc + pfo, csrc, (lx < CFQ) ? cok : 0);
@@ -335,9 +359,11 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
         s3_commit();                                    // one group per entry, possibly empty
         ++pf; ++pfj; usrc += nx; csrc += CF;
         if constexpr (ND) nsrc += nx;
+        if constexpr (NF) fsrc += nx;
         if (pfj == T) {
             pfj = 0; ++pfk; usrc += uwrap; csrc += cwrap;
             if constexpr (ND) nsrc += uwrap;
+            if constexpr (NF) fsrc += uwrap;
         }
         pfo += RSB;
         if (pfo == RINGB) pfo = 0;
@@ -358,8 +384,8 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
             if (last_col) v[NX - 1] = bc1;
         }
     };
-    auto ldnu = [&](const unsigned off, float (&v)[NX + 1]) {      // nodal modes: the nu row of a slot
-        const float* slot = reinterpret_cast<const float*>(reinterpret_cast<const char*>(ring) + off) + UROW;
+    auto ldnu = [&](const unsigned off, float (&v)[NX + 1], const int rowoff) {      // the nu (or f) row of a slot
+        const float* slot = reinterpret_cast<const float*>(reinterpret_cast<const char*>(ring) + off) + rowoff;
         const float4 q = *reinterpret_cast<const float4*>(slot + 4 * lx);
         v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
         if constexpr (NX == 8) {
@@ -414,7 +440,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
         const bool last = (k + 1 == ke);                // the sums of plane k + 1 are parked (plane ke: finished after the march)
         const float wzlo = (k == 0) ? 0.5f : 1.f;
         const float nllo = -gs * fw * wzlo;
-        float enlo = 0.f, ello = 0.f;
+        float enlo = 0.f, ello = 0.f, elnf = 0.f;
 #pragma unroll
         for (int c = 0; c < NX; ++c) { pendL1[c] = 0.f; pendU1[c] = 0.f; }
         float* rlo = rb + ((size_t)k * ny + y0) * nx;
@@ -468,13 +494,15 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                 __syncwarp(submask);                    // the node right of a lane's last is the next lane's
             }
             if constexpr (!KG) {
-                ldnu(oA, nA); ldnu(oB, nB); ldnu(oC, nC); ldnu(oD, nD);
+                ldnu(oA, nA, UROW); ldnu(oB, nB, UROW); ldnu(oC, nC, UROW); ldnu(oD, nD, UROW);
 #pragma unroll
                 for (int c = 0; c <= NX; ++c) {
                     yA[c] = nA[c] + nB[c]; yC[c] = nC[c] + nD[c];
                     zA[c] = nA[c] + nC[c]; zB[c] = nB[c] + nD[c];
                 }
             }
+            float fA[NX + 1], fB[NX + 1], fC[NX + 1], fD[NX + 1];      // nodal forcing on the four node rows
+            if constexpr (NF) { ldnu(oA, fA, FOFF); ldnu(oB, fB, FOFF); ldnu(oC, fC, FOFF); ldnu(oD, fD, FOFF); }
             if constexpr (KG) {
                 const ulonglong2* gp = reinterpret_cast<const ulonglong2*>(reinterpret_cast<const char*>(ring) + oD) + COEF / 4;
 #pragma unroll
@@ -517,6 +545,15 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                     s3_bilerp(zA[c], zA[c + 1], zB[c], zB[c + 1], Nz);                                           // (p, q)
                 }
                 s3_element(Nx, Ny, Nz, eA, slo, w0, txy, txz, tyz, txyz, iso, kx, ky, kz, r);
+                if constexpr (NF) {
+                    const float fc[8] = {fA[c], fA[c + 1], fB[c], fB[c + 1], fC[c], fC[c + 1], fD[c], fD[c + 1]};
+                    const float uc[8] = {uA[c], uA[c + 1], uB[c], uB[c + 1], uC[c], uC[c + 1], uD[c], uD[c + 1]};
+                    float m[8], e = 0.f;
+                    s3_mass(fc, m);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) { r[t] = fmaf(-fs, m[t], r[t]); e = fmaf(uc[t], m[t], e); }
+                    elnf += (c == NX - 1) ? e * g3 : e;
+                }
                 if (c == NX - 1) {
                     // the lane's last element: its right-hand corners belong to the next lane; in the lane that ends the
                     // row it does not exist (g3 = 0)
@@ -577,7 +614,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
             if (act) { st4(plo, olo); st4(pup, pendU1); }
             oA = wrapb(oA + RSB); ++n;
         }
-        end += (double)enlo; eld += (double)(wzlo * ello);   // per-plane sums go to double
+        end += (double)enlo; eld += NF ? (double)elnf : (double)(wzlo * ello);   // per-plane sums go to double
     }
     s3_wait<0>();
 
@@ -614,11 +651,15 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
             ptop += nx;
             oA = wrapb(oA + RSB);
         }
-        end += (double)entop; eld += (double)(0.5f * eltop);
+        end += (double)entop;
+        if constexpr (!NF) eld += (double)(0.5f * eltop);
     }
 
     // ---- energy partial of this unit: its lanes summed in a fixed order in double
-    double d = act ? 0.5 * (double)kap * end : 0.0, l = (act && hasf) ? (double)fw * eld : 0.0;
+    // NF: `end` holds sum u (K u - F) in units of kap and `eld` sum u_corner (M_e f_e)_corner, so that
+    // the load part is fsabs * eld and the diffusion part half of (kap * end + load part)
+    double l = !act ? 0.0 : NF ? (double)fsabs * eld : hasf ? (double)fw * eld : 0.0;
+    double d = !act ? 0.0 : NF ? 0.5 * ((double)kap * end + l) : 0.5 * (double)kap * end;
     for (int off = LW >> 1; off > 0; off >>= 1) {
         d += __shfl_down_sync(submask, d, off, LW);
         l += __shfl_down_sync(submask, l, off, LW);
@@ -802,20 +843,21 @@ constexpr size_t S3_SMEM_BLOCK = 232448;           // most a block can ask for
 int s3_nxl(int nx) { return (nx > 128) ? 8 : 4; }  // nodes per lane (8 on narrow rows was slower: 89 against 79 us on 64^3 x 32)
 // resident blocks of 4 warps per SM the kernel is compiled for: the nodal modes keep two rows per slot and trade
 // warps for taller tiles on wide rows
-int s3_minb(int nxl, int mode) { return (nxl == 8) ? (mode == DN_NU_KL_GAUSS ? 3 : 2) : 4; }
-int s3_slot_floats(int nxl, int lw, int mode, int m) {
+int s3_minb(int nxl, int mode, bool nf) { return (nxl == 8) ? ((mode == DN_NU_KL_GAUSS && !nf) ? 3 : 2) : 4; }
+int s3_slot_floats(int nxl, int lw, int mode, int m, bool nf) {
     const int urow = nxl * lw + 4;
-    return (mode == DN_NU_KL_GAUSS) ? urow + 2 * s3_gs(m) : (mode == DN_NU_KL_NODAL) ? 2 * urow + s3_gs(m) : 2 * urow;
+    const int rows = (mode == DN_NU_KL_GAUSS ? 1 : 2) + (nf ? 1 : 0);
+    return rows * urow + (mode == DN_NU_KL_GAUSS ? 2 * s3_gs(m) : mode == DN_NU_KL_NODAL ? s3_gs(m) : 0);
 }
 
 S3Geo geometry3s(const dn_problem& p) {
     S3Geo g{};
     const int nx = p.grid.nx, ny = p.grid.ny, nz = p.grid.nz;
-    const int NX = s3_nxl(nx), minb = s3_minb(NX, p.nu_mode);
+    const int NX = s3_nxl(nx), minb = s3_minb(NX, p.nu_mode, p.f != nullptr);
     g.LW = 8; g.lwsh = 3;
     while (g.LW * NX < nx) { g.LW *= 2; ++g.lwsh; }
     const int subs = 32 / g.LW;
-    g.RS = s3_slot_floats(NX, g.LW, p.nu_mode, p.kl_modes);
+    g.RS = s3_slot_floats(NX, g.LW, p.nu_mode, p.kl_modes, p.f != nullptr);
     size_t per_block = (S3_SMEM_SM - (size_t)minb * 1024) / minb;
     if (per_block > S3_SMEM_BLOCK) per_block = S3_SMEM_BLOCK;
     if (p.nu_mode == DN_NU_KL_GAUSS) per_block -= sizeof(float) * 4 * NX * g.LW;      // the block's table of cosine pairs
@@ -846,15 +888,22 @@ S3Geo geometry3s(const dn_problem& p) {
     return g;
 }
 
-template <int NX, int M, int MODE, int MINB>
-cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+template <int NX, int M, int MODE, bool NF, int MINB>
+cudaError_t launch_nmf(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
     const int subs = 32 / g.LW;
     const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * (g.C * g.RS + (NX == 8 ? NX * g.LW : 0)) + (MODE == 0 ? 4 * NX * g.LW : 0));
     const long long per_block = (long long)S3_WARPS * subs;
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
-    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, NF, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(strip3d_kernel<NX, M, MODE, MINB>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
+    return launch_dependent(strip3d_kernel<NX, M, MODE, NF, MINB>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
+}
+
+// MINB: blocks per SM without nodal forcing; with it, wide rows run two blocks per SM in every mode (s3_minb)
+template <int NX, int M, int MODE, int MINB>
+cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+    if (P.f) return launch_nmf<NX, M, MODE, true, (NX == 8 ? 2 : 4)>(P, linepoly, g, s);
+    return launch_nmf<NX, M, MODE, false, MINB>(P, linepoly, g, s);
 }
 
 template <int M>
@@ -868,7 +917,7 @@ cudaError_t launch_m3(const Params& P, const float* linepoly, const S3Geo& g, cu
 dn_problem s3_problem_of(const Params& P) {
     dn_problem p{};
     p.grid.dim = 3; p.grid.nx = P.nx; p.grid.ny = P.ny; p.grid.nz = P.nz; p.batch = P.batch;
-    p.nu_mode = P.nu_mode; p.kl_modes = P.m;
+    p.nu_mode = P.nu_mode; p.kl_modes = P.m; p.f = P.f;
     return p;
 }
 
@@ -877,7 +926,7 @@ dn_problem s3_problem_of(const Params& P) {
 // Rows of at most 128 nodes take 4 nodes per lane, rows of at most 256 nodes 8 (then nx must be a multiple of 8,
 // so that only the last element of the last lane falls outside the grid).
 bool strip3d_applicable(const dn_problem& p) {
-    if (!(p.grid.dim == 3 && p.f == nullptr && p.grid.nx % 4 == 0 && p.grid.nx >= 8 &&
+    if (!(p.grid.dim == 3 && p.grid.nx % 4 == 0 && p.grid.nx >= 8 &&
           p.grid.nx <= 256 && p.grid.ny >= 2 && p.grid.nz >= 2))
         return false;
     return p.grid.nx <= 128 || p.grid.nx % 8 == 0;

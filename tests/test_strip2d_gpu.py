@@ -98,7 +98,8 @@ def test_strip2d_determinism_and_stale_workspace():
 
 
 @pytest.mark.parametrize("mode", KL_MODES)
-@pytest.mark.parametrize("nx,ny,batch,m", [(1024, 40, 2, 4), (1120, 16, 2, 2), (1124, 21, 1, 3), (2052, 37, 1, 7), (1024, 300, 5, 2)])
+@pytest.mark.parametrize("nx,ny,batch,m", [(1024, 40, 2, 4), (1120, 16, 2, 2), (1124, 21, 1, 3), (2052, 37, 1, 7), (1024, 300, 5, 2),
+                                           (256, 64, 3, 4), (380, 33, 2, 2)])     # with nodal forcing also rows from 256 nodes on
 def test_strip2d_nodal_forcing(nx, ny, batch, m, mode):
     """Nodal forcing on the strip kernel: the load vector is the consistent mass matrix applied to f (the f row rides in the
     ring with the u row).  All flag combinations, because the Dirichlet columns take the one-sided mass weights."""

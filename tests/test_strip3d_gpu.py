@@ -78,3 +78,33 @@ def test_strip3d_isotropic_cells_and_closed_form():
     Jg, rg = run_gpu(pg, u)
     assert np.allclose(Jg, 0.5, rtol=1e-5)
     assert np.abs(rg).max() < 1e-5 / n
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("nx,ny,nz,batch,m", [(64, 20, 9, 3, 2), (24, 7, 6, 2, 3), (256, 12, 7, 1, 3), (128, 9, 13, 2, 4), (136, 6, 5, 1, 2)])
+def test_strip3d_nodal_forcing(nx, ny, nz, batch, m, mode):
+    """Nodal forcing on the 3D strip kernel: the load is taken element by element (mass matrix applied to the corner values
+    of f) and gathered with the stiffness contributions, across tile and chunk seams; anisotropic cells; every flag."""
+    inp = inputs.random_inputs(3, nx, ny, nz, batch, m, seed=23 + nx + ny)
+    u = inputs.random_field(inp.u.shape, 4)
+    f = inputs.random_field(inp.u.shape, 9, scale=3.0)
+    nu = inputs.random_positive_field(inp.u.shape, 5) if mode == B.DN_NU_NODAL else None
+    gJ = np.linspace(-1.5, 2.0, batch).astype(np.float32)
+    for flags in (0, B.DN_NO_MASK, B.DN_IMPOSE_BC_ON_LOAD):
+        po, pg = make_problems(inp, mode, nu=nu, f=f, flags=flags, bc=(0.8, -0.3))
+        assert B.dn_path_name(pg) == "strip3d"
+        Jo, _, _, ro = oracle.energy_grad(po, u, gJ=gJ.astype(np.float64))
+        Jg, rg = run_gpu(pg, u, gJ=gJ)
+        check(Jg, rg, Jo, ro, f"nodal f, flags={flags}")
+        if not (flags & B.DN_NO_MASK):
+            assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
+
+
+def test_strip3d_nodal_forcing_on_cubic_cells():
+    inp = inputs.random_inputs(3, 40, 40, 40, 2, 2, seed=5)
+    f = inputs.random_field(inp.u.shape, 3)
+    po, pg = make_problems(inp, B.DN_NU_KL_GAUSS, f=f)
+    assert B.dn_path_name(pg) == "strip3d"
+    Jo, _, _, ro = oracle.energy_grad(po, inp.u)
+    Jg, rg = run_gpu(pg, inp.u)
+    check(Jg, rg, Jo, ro, "nodal f, cubic cells")
