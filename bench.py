@@ -173,7 +173,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "nu_mode": args.nu_mode, "step": f"oracle pass over {n} sample(s)"},
+            "config": {"workload": wl.name, "nu_mode": args.nu_mode},
+            "detail": {"step": f"oracle pass over {n} sample(s)"},
             "cpu_baseline": base,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -218,7 +219,7 @@ def run_reference_burgers(args):
     print(json.dumps({"impl": "reference", "metric": BURGERS_METRIC, "value": value, "unit": BURGERS_UNIT,
                       "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
                       "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-                      "config": {"workload": BURGERS_NAME, "step": f"oracle pass over {n} sample(s)"},
+                      "config": {"workload": BURGERS_NAME}, "detail": {"step": f"oracle pass over {n} sample(s)"},
                       "cpu_baseline": base,
                       "e2e": {"value": value, "unit": BURGERS_UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
@@ -308,9 +309,9 @@ def main_burgers(args):
             "metric": BURGERS_METRIC, "value": world * nodes / (step_ms * 1e-3) / 1e9, "unit": BURGERS_UNIT, "n_gpus": world,
             "steps": K, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": BURGERS_NAME, "kernel_path": B.dn_burgers_path_name(prob, u, g),
-                       "nodes_per_step_per_gpu": nodes, "sharding": "independent batches per rank",
-                       "l2": "inputs larger than L2"},
+            "config": {"workload": BURGERS_NAME},
+            "detail": {"kernel_path": B.dn_burgers_path_name(prob, u, g), "nodes_per_step_per_gpu": nodes,
+                       "sharding": "independent batches per rank", "l2": "inputs larger than L2"},
             "clocks": clocks,
             "e2e": {"value": world * nodes / (e2e_ms * 1e-3) / 1e9, "unit": BURGERS_UNIT,
                     "h2d_bytes_per_step": field_bytes + 8 * bs, "d2h_bytes_per_step": field_bytes + 4 * bs,
@@ -650,8 +651,8 @@ def main():
             "metric": METRIC, "value": world * elements / (step_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "nu_mode": args.nu_mode, "kernel_path": path,
-                       "elements_per_step_per_gpu": elements, "sharding": "independent batches per rank",
+            "config": {"workload": wl.name, "nu_mode": args.nu_mode},        # the same keys in the reference arm's line
+            "detail": {"kernel_path": path, "elements_per_step_per_gpu": elements, "sharding": "independent batches per rank",
                        "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps"},
             "clocks": clocks,
             "e2e": {"value": world * elements / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
