@@ -66,7 +66,7 @@ __device__ void rowpoly_entry(const TableArgs& A, long long idx) {
         for (int jj = 0; jj < MX; ++jj) {
             if (i < m && jj < m) {
                 const double den = 1.0 + (double)((i + 1) * (i + 1)) + (double)((jj + 1) * (jj + 1));
-                a += (double)(float)((double)w[i * m + jj] * kLog2e / den) * cy[jj];
+                a += (double)(float)((double)w[i * m + jj] * (kLog2e / den)) * cy[jj];     // the constant folds: no division
             }
         }
         g[i] = a;
@@ -106,7 +106,7 @@ __global__ void tables_kernel(TableArgs A) {
         j = (int)(c % m) + 1;
         i = (int)(c / m) + 1;
         const double den = 1.0 + (double)i * i + (double)j * j + (double)k * k;
-        A.ckl[idx] = (float)((double)A.kl_w[idx] * kLog2e / den);
+        A.ckl[idx] = (float)((double)A.kl_w[idx] * (kLog2e / den));      // the same product the row polynomials form
         return;
     }
     idx -= ncoef;
