@@ -38,18 +38,18 @@ FP32_PEAK_LANE_OPS = 148 * 128 * 1.965e9     # SMs x FP32 lanes x max SM clock: 
 # (FADD + FMUL + FFMA + 2 FFMA2).  Each entry names the kernel source it was taken from and the first 16
 # hex digits of its sha256: once that file changes the entry no longer applies and null is reported.
 NCU_CAPTURES = {
-    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 499726848, "fp32_ops_per_element": 57.7,
-                                          "src": "dn_strip2d.cu", "sha": "2756d5fb6f39c161"},
-    "strip2d:cfg2_2d_2048^2_b16_m6:klnodal": {"traffic": 502524160, "fp32_ops_per_element": 44.0,
-                                               "src": "dn_strip2d.cu", "sha": "2756d5fb6f39c161"},
-    "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 789649408, "fp32_ops_per_element": 35.9,
-                                             "src": "dn_strip2d.cu", "sha": "2756d5fb6f39c161"},
-    "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 610945279, "fp32_ops_per_element": 133.8,
-                                        "src": "dn_strip3d.cu", "sha": "6ead4793590ff495"},
-    "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 839546880, "fp32_ops_per_element": 142.2,
-                                           "src": "dn_strip3d.cu", "sha": "6ead4793590ff495"},
-    "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 556759296, "fp32_ops_per_element": 145.9,
-                                             "src": "dn_strip3d.cu", "sha": "6ead4793590ff495"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 500348160, "fp32_ops_per_element": 57.7,
+                                          "src": "dn_strip2d.cu", "sha": "20e9f8b91a7ab7a5"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:klnodal": {"traffic": 500662784, "fp32_ops_per_element": 44.0,
+                                               "src": "dn_strip2d.cu", "sha": "20e9f8b91a7ab7a5"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 789951488, "fp32_ops_per_element": 35.9,
+                                             "src": "dn_strip2d.cu", "sha": "20e9f8b91a7ab7a5"},
+    "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 610791424, "fp32_ops_per_element": 133.8,
+                                        "src": "dn_strip3d.cu", "sha": "8ed5fe52383281c8"},
+    "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 835259904, "fp32_ops_per_element": 142.2,
+                                           "src": "dn_strip3d.cu", "sha": "8ed5fe52383281c8"},
+    "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 556080384, "fp32_ops_per_element": 145.9,
+                                             "src": "dn_strip3d.cu", "sha": "8ed5fe52383281c8"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
                                     "src": "dn_burgers.cu", "sha": "baf4524ba7aede8d"},
 }
