@@ -119,6 +119,39 @@ def test_entry_point_without_workspace_refuses_on_the_host(L):
     assert L.dn_energy_grad_static(C.byref(prob(64, 64, 2, 2)), fake, None, None, None, None) == B.DN_ERR_NULL
 
 
+def test_kernel_family_and_launch_count_by_shape(L):
+    """Which kernel family the fused call takes is decided on the host from the shape alone (pointer alignment aside)."""
+    from paper_2007_12792_b200 import binding as B
+    fake = 0x100000
+
+    def prob(dim, nx, ny, nz, mode=B.DN_NU_KL_GAUSS, f=None, flags=0, batch=4, m=3):
+        p = B.DnProblem()
+        p.grid = B.DnGrid(dim, nx, ny, nz)
+        p.batch = batch; p.nu_mode = mode; p.kl_modes = m; p.kl_w = fake
+        p.nu = fake if mode == B.DN_NU_NODAL else None
+        p.f = f; p.flags = flags
+        return p
+
+    name = lambda p: L.dn_path_name(C.byref(p)).decode()
+    assert name(prob(2, 2048, 2048, 1)) == "strip2d" and name(prob(2, 256, 256, 1)) == "tiled2d"
+    assert name(prob(2, 256, 256, 1, f=fake)) == "strip2d"              # nodal forcing: the strip kernel from 256 nodes on
+    assert name(prob(2, 128, 64, 1, f=fake)) == "generic" and name(prob(2, 1030, 64, 1)) == "generic"
+    for mode in (B.DN_NU_KL_GAUSS, B.DN_NU_NODAL, B.DN_NU_KL_NODAL):
+        assert name(prob(3, 256, 256, 256, mode)) == "strip3d" and name(prob(3, 64, 64, 64, mode, f=fake)) == "strip3d"
+        assert name(prob(3, 8, 2, 2, mode)) == "strip3d" and name(prob(3, 136, 9, 9, mode)) == "strip3d"
+    assert name(prob(3, 260, 16, 16)) == "tiled3d" and name(prob(3, 260, 16, 16, B.DN_NU_KL_NODAL)) == "generic"
+    assert name(prob(3, 512, 16, 16, B.DN_NU_NODAL)) == "tiled3d" and name(prob(3, 516, 16, 16)) == "generic"
+    assert name(prob(3, 64, 64, 64, flags=B.DN_FORCE_GENERIC)) == "generic"
+    # launches per call: tables, line polynomials, fused kernel, seam fix-up, finaliser
+    assert L.dn_launches_per_call(C.byref(prob(3, 256, 256, 256))) == 5
+    assert L.dn_launches_per_call(C.byref(prob(3, 256, 256, 256, B.DN_NU_NODAL))) == 3
+    assert L.dn_launches_per_call(C.byref(prob(2, 2048, 2048, 1))) == 3
+    # the scratch of a 3D problem: seams and the coefficient table, well below one field per sample
+    p = prob(3, 256, 256, 256)
+    assert 0 < L.dn_workspace_bytes(C.byref(p)) < 4 * 256 ** 3 * 4
+    assert L.dn_cg_workspace_bytes(C.byref(p)) > 4 * 4 * 256 ** 3 * 4
+
+
 def test_binding_rejects_host_tensors_and_missing_library(monkeypatch):
     import torch
     from paper_2007_12792_b200 import binding as B
