@@ -116,3 +116,26 @@ def test_strip2d_nodal_forcing(nx, ny, batch, m, mode):
         check(Jg, rg, Jo, ro, f"nodal f, flags={flags}")
         if not (flags & B.DN_NO_MASK):
             assert np.all(rg[..., 0] == 0.0) and np.all(rg[..., -1] == 0.0)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_strip2d_random_shapes(seed):
+    """Seeded random shapes, modes, flags and forcing kinds on the 2D strip kernel."""
+    rng = np.random.default_rng(3000 + seed)
+    f_nodal = rng.random() < 0.5
+    nx = 4 * int(rng.integers(64 if f_nodal else 250, 700))       # without nodal forcing rows below about 1000 nodes run tiled2d
+    ny = int(rng.integers(16, 90))
+    batch, m = int(rng.integers(1, 4)), int(rng.integers(1, 9))
+    mode = KL_MODES[int(rng.integers(0, 3))]
+    flags = int(rng.choice([0, B.DN_NO_MASK, B.DN_IMPOSE_BC_ON_LOAD, B.DN_IMPOSE_BC_ON_LOAD | B.DN_NO_MASK]))
+    inp = inputs.random_inputs(2, nx, ny, 1, batch, m, seed=4000 + seed, f_const=float(rng.choice([0.0, 0.7])))
+    u = inputs.random_field(inp.u.shape, 50 + seed)
+    nu = inputs.random_positive_field(inp.u.shape, 60 + seed) if mode == B.DN_NU_NODAL else None
+    f = inputs.random_field(inp.u.shape, 70 + seed, scale=2.0) if f_nodal else None
+    gJ = rng.uniform(-2, 2, batch).astype(np.float32) if rng.random() < 0.5 else None
+    po, pg = make_problems(inp, mode, nu=nu, f=f, flags=flags, bc=(0.6, -0.2))
+    if B.dn_path_name(pg) != "strip2d":
+        pytest.skip("this width takes the tiled kernel")
+    Jo, _, _, ro = oracle.energy_grad(po, u, gJ=None if gJ is None else gJ.astype(np.float64))
+    Jg, rg = run_gpu(pg, u, gJ=gJ)
+    check(Jg, rg, Jo, ro, f"seed {seed}: {nx}x{ny} b{batch} m{m} mode{mode} flags{flags} f={'nodal' if f_nodal else inp.f_const}")

@@ -108,3 +108,27 @@ def test_strip3d_nodal_forcing_on_cubic_cells():
     Jo, _, _, ro = oracle.energy_grad(po, inp.u)
     Jg, rg = run_gpu(pg, inp.u)
     check(Jg, rg, Jo, ro, "nodal f, cubic cells")
+
+
+@pytest.mark.parametrize("seed", range(36))
+def test_strip3d_random_shapes(seed):
+    """Seeded random shapes, modes, flags and forcing kinds: tiles and chunks with ragged ends, single-row tiles, one-plane
+    chunks, every lane layout, m up to 8 (the coefficient row then needs more pieces than a narrow unit has lanes)."""
+    rng = np.random.default_rng(1000 + seed)
+    nx = int(rng.choice([8, 12, 16, 24, 32, 36, 48, 64, 72, 100, 128, 136, 192, 256]))
+    ny, nz = int(rng.integers(2, 34)), int(rng.integers(2, 34))
+    if nx >= 128:
+        ny, nz = min(ny, 14), min(nz, 14)
+    batch, m = int(rng.integers(1, 6)), int(rng.integers(1, 9))
+    mode = MODES[int(rng.integers(0, 3))]
+    flags = int(rng.choice([0, B.DN_NO_MASK, B.DN_IMPOSE_BC_ON_LOAD, B.DN_IMPOSE_BC_ON_LOAD | B.DN_NO_MASK]))
+    inp = inputs.random_inputs(3, nx, ny, nz, batch, m, seed=2000 + seed, f_const=float(rng.choice([0.0, 0.7])))
+    u = inputs.random_field(inp.u.shape, 50 + seed)
+    nu = inputs.random_positive_field(inp.u.shape, 60 + seed) if mode == B.DN_NU_NODAL else None
+    f = inputs.random_field(inp.u.shape, 70 + seed, scale=2.0) if rng.random() < 0.4 else None
+    gJ = rng.uniform(-2, 2, batch).astype(np.float32) if rng.random() < 0.5 else None
+    po, pg = make_problems(inp, mode, nu=nu, f=f, flags=flags, bc=(0.6, -0.2))
+    assert B.dn_path_name(pg) == "strip3d"
+    Jo, _, _, ro = oracle.energy_grad(po, u, gJ=None if gJ is None else gJ.astype(np.float64))
+    Jg, rg = run_gpu(pg, u, gJ=gJ)
+    check(Jg, rg, Jo, ro, f"seed {seed}: {nx}x{ny}x{nz} b{batch} m{m} mode{mode} flags{flags} f={'nodal' if f is not None else inp.f_const}")
