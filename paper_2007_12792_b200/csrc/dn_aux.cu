@@ -93,6 +93,7 @@ __device__ void rowpoly_entry(const TableArgs& A, long long idx) {
 }
 
 __global__ void tables_kernel(TableArgs A) {
+    dep_wait();                                        // whatever ran before in the stream may still read these tables
     dep_release();
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int m = A.m;
@@ -329,8 +330,7 @@ cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float*
     A.rowpoly = (P.dim == 2) ? rowpoly : nullptr; A.rp_gs = rowpoly_stride; A.rp_nodes = rowpoly_nodes ? 1 : 0;
     if (A.rowpoly) total += 2ll * P.batch * (P.ny - (rowpoly_nodes ? 0 : 1));
     const int threads = 128;
-    tables_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, s>>>(A);
-    return cudaGetLastError();
+    return launch_dependent(tables_kernel, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, s, A);
 }
 
 cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s) {
