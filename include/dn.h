@@ -256,7 +256,7 @@ const char* dn_burgers_path_name(const dn_burgers* problem, const float* u, cons
  * dn_energy_grad call (for launch accounting); 0 if the problem is invalid. */
 int32_t dn_launches_per_call(const dn_problem* problem);
 
-/* Name of the kernel family that dn_energy_grad would use ("strip2d", "strip3d", "tiled2d", "tiled3d", "generic"). */
+/* Name of the kernel family that dn_energy_grad would use ("row2d", "strip2d", "strip3d", "tiled2d", "tiled3d", "generic"). */
 const char* dn_path_name(const dn_problem* problem);
 
 const char* dn_status_string(dn_status status);

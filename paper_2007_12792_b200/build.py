@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdn.so")
-SOURCES = ["dn_api.cu", "dn_aux.cu", "dn_generic.cu", "dn_tiled2d.cu", "dn_strip2d.cu", "dn_tiled3d.cu", "dn_strip3d.cu", "dn_static.cu", "dn_burgers.cu", "dn_cg.cu"]
+SOURCES = ["dn_api.cu", "dn_aux.cu", "dn_generic.cu", "dn_tiled2d.cu", "dn_strip2d.cu", "dn_row2d.cu", "dn_tiled3d.cu", "dn_strip3d.cu", "dn_static.cu", "dn_burgers.cu", "dn_cg.cu"]
 HEADERS = [os.path.join(CSRC, "dn_internal.cuh"), os.path.join(ROOT, "include", "dn.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]

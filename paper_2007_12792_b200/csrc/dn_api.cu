@@ -41,6 +41,7 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 Launch choose_launch(const dn_problem& p, const float* u, const float* r) {
     const bool vec_ok = aligned16(u) && aligned16(r) && (p.nu_mode != DN_NU_NODAL || aligned16(p.nu)) && aligned16(p.f);
     if (!(p.flags & DN_FORCE_GENERIC) && vec_ok) {
+        if (r && row2d_applicable(p)) return row2d_geometry(p);          // narrow 2D rows, constant forcing
         if (r && strip2d_applicable(p)) return strip2d_geometry(p);      // the strip kernels also take nodal forcing
         if (r && strip3d_applicable(p)) return strip3d_geometry(p);
         if (p.f == nullptr) {
@@ -60,6 +61,7 @@ static int max_nblk(const dn_problem& p) {
     int n = generic_blocks_per_sample(nodes_per_sample(p.grid));
     if (tiled2d_applicable(p)) { int t = tiled2d_geometry(p).nblk; if (t > n) n = t; }
     if (strip2d_applicable(p)) { int t = strip2d_geometry(p).nblk; if (t > n) n = t; }
+    if (row2d_applicable(p)) { int t = row2d_geometry(p).nblk; if (t > n) n = t; }
     if (tiled3d_applicable(p)) { int t = tiled3d_geometry(p).nblk; if (t > n) n = t; }
     if (strip3d_applicable(p)) { int t = strip3d_geometry(p).nblk; if (t > n) n = t; }
     return n;
@@ -97,6 +99,7 @@ WsLayout make_layout(const dn_problem& p, const Launch& l, bool tight) {
     }
     w.rowpoly = off;
     if ((tight ? l.path == PATH_STRIP2D : strip2d_applicable(p))) off += align_up(sizeof(float) * strip2d_rowpoly_floats(p) + 16);
+    else if ((tight ? l.path == PATH_ROW2D : row2d_applicable(p))) off += align_up(sizeof(float) * row2d_rowpoly_floats(p) + 16);
     w.zseam = off;
     w.linepoly = off;
     if ((tight ? l.path == PATH_STRIP3D : strip3d_applicable(p))) {
@@ -139,7 +142,7 @@ static cudaError_t tables_into(const dn_problem& p, const Params& P, const WsLay
     float* cn[3] = {reinterpret_cast<float*>(base + w.cn[0]), reinterpret_cast<float*>(base + w.cn[1]),
                     reinterpret_cast<float*>(base + w.cn[2])};
     const cudaError_t e = launch_tables(P, p.kl_w, reinterpret_cast<float*>(base + w.ckl), cg, cn, s,
-                                        (l.path == PATH_STRIP2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
+                                        (l.path == PATH_STRIP2D || l.path == PATH_ROW2D) ? reinterpret_cast<float*>(base + w.rowpoly) : nullptr,
                                         strip2d_rowpoly_stride(p.kl_modes), p.nu_mode == DN_NU_KL_NODAL);
     if (e != cudaSuccess || l.path != PATH_STRIP3D) return e;
     return launch_linepoly3d(P, reinterpret_cast<float*>(base + w.linepoly), s);
@@ -160,9 +163,9 @@ static dn_status plan(const dn_problem* p, const float* u, const float* r, size_
     }
     l = choose_launch(*p, u, r);
     w = make_layout(*p, l, tight);
-    if (tight && l.path == PATH_STRIP2D && ws_bytes < w.total) {
-        // the strip kernel's coefficient table does not fit: the tiled kernel where it can run (rows of at most
-        // 2048 nodes), else the any-size kernel; if that does not fit either the call is refused
+    if (tight && (l.path == PATH_STRIP2D || l.path == PATH_ROW2D) && ws_bytes < w.total) {
+        // the strip / row kernel's coefficient table does not fit: the tiled kernel where it can run (rows of at most
+        // 2048 nodes, constant forcing), else the any-size kernel; if that does not fit either the call is refused
         if (tiled2d_applicable(*p)) {
             l = tiled2d_geometry(*p);
         } else {
@@ -200,6 +203,7 @@ static dn_status run(const dn_problem* p, const float* u, const float* gJ, float
     if (p->nu_mode != DN_NU_NODAL && tables_into(*p, P, w, l, ws, s) != cudaSuccess) return DN_ERR_CUDA;
     if (ev_before && cudaEventRecord(static_cast<cudaEvent_t>(ev_before), s) != cudaSuccess) return DN_ERR_CUDA;
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
+    else if (l.path == PATH_ROW2D) e = launch_row2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
     else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
     else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
     else if (l.path == PATH_STRIP3D) e = launch_strip3d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.linepoly), s);
@@ -225,6 +229,7 @@ dn_status run_operator(const dn_problem* p, const float* u, float* r, void* ws, 
     cudaError_t e = cudaSuccess;
     if (build_tables && p->nu_mode != DN_NU_NODAL && tables_into(*p, P, w, l, ws, s) != cudaSuccess) return DN_ERR_CUDA;
     if (l.path == PATH_STRIP2D) e = launch_strip2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
+    else if (l.path == PATH_ROW2D) e = launch_row2d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.rowpoly), s);
     else if (l.path == PATH_TILED2D) e = launch_tiled2d(P, l, s);
     else if (l.path == PATH_TILED3D) e = launch_tiled3d(P, l, s);
     else if (l.path == PATH_STRIP3D) e = launch_strip3d(P, reinterpret_cast<const float*>(static_cast<char*>(ws) + w.linepoly), s);
@@ -429,6 +434,7 @@ const char* dn_path_name(const dn_problem* p) {
     if (validate(p) != DN_OK) return "invalid";
     // the fused call (the strip kernels also with nodal forcing); the energy-only call of such a problem runs the tiled
     // kernel of its dimension or, with nodal forcing, the any-size kernel
+    if (!(p->flags & DN_FORCE_GENERIC) && row2d_applicable(*p)) return "row2d";
     if (!(p->flags & DN_FORCE_GENERIC) && strip2d_applicable(*p)) return "strip2d";
     if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && tiled2d_applicable(*p)) return "tiled2d";
     if (!(p->flags & DN_FORCE_GENERIC) && strip3d_applicable(*p)) return "strip3d";

@@ -17,7 +17,7 @@ constexpr int kAlign = 256;
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
-enum Path { PATH_GENERIC = 0, PATH_TILED2D = 1, PATH_TILED3D = 2, PATH_STRIP2D = 3, PATH_STRIP3D = 4 };
+enum Path { PATH_GENERIC = 0, PATH_TILED2D = 1, PATH_TILED3D = 2, PATH_STRIP2D = 3, PATH_STRIP3D = 4, PATH_ROW2D = 5 };
 
 // Where things live inside the caller's workspace (byte offsets, all 256-B aligned).
 struct WsLayout {
@@ -28,7 +28,7 @@ struct WsLayout {
     int gstride[3];       // padded row length of cg[a] (multiple of 4)
     size_t cn[3];         // float  [m][nstride[a]] cos(i pi x) at the nodes of axis a
     int nstride[3];
-    size_t rowpoly;       // float  [B][ny-1][GS] polynomial of the KL exponent along every Gauss row (strip 2D kernel)
+    size_t rowpoly;       // float  [B][ny-1][GS] polynomial of the KL exponent along every Gauss row (strip 2D and row 2D kernels)
     size_t zseam;         // float  contributions across the chunk seams of the strip 3D kernel
     size_t linepoly;      // float  [B][nz-1][ny-1][2 GS] the same along the four Gauss lines of every element row (strip 3D kernel)
     int nblk;             // energy partials per sample
@@ -95,6 +95,7 @@ cudaError_t launch_generic(const Params& P, cudaStream_t s);
 cudaError_t launch_tiled2d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_tiled3d(const Params& P, const Launch& l, cudaStream_t s);
 cudaError_t launch_strip2d(const Params& P, const float* rowpoly, cudaStream_t s);
+cudaError_t launch_row2d(const Params& P, const float* rowpoly, cudaStream_t s);   // same table as the strip 2D kernel
 cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s);
 cudaError_t launch_kl_field(const dn_grid& g, int batch, int m, const float* kl_w, float* nu, cudaStream_t s);
 cudaError_t launch_apply_bc(const dn_grid& g, int batch, float b0, float b1, int mode, float* field, cudaStream_t s,
@@ -107,6 +108,9 @@ bool strip2d_applicable(const dn_problem& p);     // fused energy+residual, KL a
 Launch strip2d_geometry(const dn_problem& p);
 size_t strip2d_rowpoly_floats(const dn_problem& p);
 int strip2d_rowpoly_stride(int kl_modes);          // floats per element row of that table
+bool row2d_applicable(const dn_problem& p);       // fused energy+residual, 2D grids whose rows fit one warp (nx <= 256)
+Launch row2d_geometry(const dn_problem& p);
+size_t row2d_rowpoly_floats(const dn_problem& p);
 Launch tiled2d_geometry(const dn_problem& p);
 Launch tiled3d_geometry(const dn_problem& p);
 size_t tiled3d_seam_floats(const dn_problem& p);   // scratch floats the tiled 3D kernel needs for its tile seams
