@@ -50,6 +50,8 @@ NCU_CAPTURES = {
                                            "src": "dn_strip3d.cu", "sha": "8ed5fe52383281c8"},
     "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 556080384, "fp32_ops_per_element": 145.9,
                                              "src": "dn_strip3d.cu", "sha": "8ed5fe52383281c8"},
+    "row2d:cfg1_2d_256^2_b64_m4:kl": {"traffic": 17593600, "fp32_ops_per_element": 51.0,
+                                       "src": "dn_row2d.cu", "sha": "bea68ed88174fe35"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
                                     "src": "dn_burgers.cu", "sha": "baf4524ba7aede8d"},
 }
@@ -636,12 +638,14 @@ def main():
     secondary = None
     if world == 1 and not args.no_secondary and args.config == 2 and args.nu_mode == "kl":
         secondary = []
-        for cfg2, mode2 in ((4, "kl"), (4, "nodal"), (2, "nodal"), (2, "klnodal")):
+        # ... and the three workloads that fit in L2, timed cold (L2 flushed between steps, outside the timed region)
+        for cfg2, mode2 in ((4, "kl"), (4, "nodal"), (2, "nodal"), (2, "klnodal"), (0, "kl"), (1, "kl"), (3, "kl")):
             sub = device_run(cfg2, mode2, max(5, min(K, 20)), 3, ClockSampler(local))
             path2, elements2, roof2, alu2 = roofline_of(sub, sub["step_ms"], sub["main_ms"])
             secondary.append({"workload": sub["wl"].name, "nu_mode": mode2, "kernel_path": path2, "ms_per_step": sub["step_ms"],
                               "value": elements2 / (sub["step_ms"] * 1e-3) / 1e9, "unit": UNIT, "roofline": roof2,
-                              "roofline_alu": alu2, "clocks": sub["clocks"], "checksum_J": float(sub["J"].double().sum())})
+                              "roofline_alu": alu2, "clocks": sub["clocks"], "checksum_J": float(sub["J"].double().sum()),
+                              "l2": "inputs larger than L2" if sub["flush"] is None else "L2 flushed between steps"})
             del sub
             torch.cuda.empty_cache()
 
