@@ -43,7 +43,7 @@ Launch choose_launch(const dn_problem& p, const float* u, const float* r) {
     if (!(p.flags & DN_FORCE_GENERIC) && vec_ok) {
         if (r && row2d_applicable(p)) return row2d_geometry(p);          // narrow 2D rows, constant forcing
         if (r && strip2d_applicable(p)) return strip2d_geometry(p);      // the strip kernels also take nodal forcing
-        if (r && strip3d_applicable(p)) return strip3d_geometry(p);
+        if (strip3d_applicable(p)) return strip3d_geometry(p);           // ... and, without r, run their energy-only variant
         if (p.f == nullptr) {
             if (tiled2d_applicable(p)) return tiled2d_geometry(p);
             if (tiled3d_applicable(p)) return tiled3d_geometry(p);

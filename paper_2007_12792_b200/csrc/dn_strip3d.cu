@@ -202,6 +202,28 @@ __device__ __forceinline__ void s3_element(const float (&Nx)[4], const float (&N
     r[0] = r000; r[1] = r100; r[2] = r010; r[3] = r110; r[4] = r001; r[5] = r101; r[6] = r011; r[7] = dXYZ;
 }
 
+// The element's diffusion energy, twice over and in the same units: sum over the 12 Gauss lines of N D^2 (the
+// derivatives as in s3_element; the residual it returns is the gradient of half this sum).
+__device__ __forceinline__ float s3_energy(const float (&Nx)[4], const float (&Ny)[4], const float (&Nz)[4],
+                                           const float e0, const float s0, const float w0,
+                                           const float txy, const float txz, const float tyz, const float txyz,
+                                           const bool iso, const float kx, const float ky, const float kz) {
+    const float a = DN_GA, bq = DN_GB;
+    const float Axa = fmaf(a, txy, e0), Axb = fmaf(bq, txy, e0);
+    const float Bxa = fmaf(a, txyz, txz), Bxb = fmaf(bq, txyz, txz);
+    const float Dx_aa = fmaf(a, Bxa, Axa), Dx_ab = fmaf(bq, Bxa, Axa), Dx_ba = fmaf(a, Bxb, Axb), Dx_bb = fmaf(bq, Bxb, Axb);
+    const float Aya = fmaf(a, txy, s0), Ayb = fmaf(bq, txy, s0);
+    const float Bya = fmaf(a, txyz, tyz), Byb = fmaf(bq, txyz, tyz);
+    const float Dy_aa = fmaf(a, Bya, Aya), Dy_ab = fmaf(bq, Bya, Aya), Dy_ba = fmaf(a, Byb, Ayb), Dy_bb = fmaf(bq, Byb, Ayb);
+    const float Aza = fmaf(a, txz, w0), Azb = fmaf(bq, txz, w0);
+    const float Dz_aa = fmaf(a, Bya, Aza), Dz_ab = fmaf(bq, Bya, Aza), Dz_ba = fmaf(a, Byb, Azb), Dz_bb = fmaf(bq, Byb, Azb);
+    float ex = (Nx[0] * Dx_aa) * Dx_aa, ey = (Ny[0] * Dy_aa) * Dy_aa, ez = (Nz[0] * Dz_aa) * Dz_aa;
+    ex = fmaf(Nx[1] * Dx_ab, Dx_ab, ex); ey = fmaf(Ny[1] * Dy_ab, Dy_ab, ey); ez = fmaf(Nz[1] * Dz_ab, Dz_ab, ez);
+    ex = fmaf(Nx[2] * Dx_ba, Dx_ba, ex); ey = fmaf(Ny[2] * Dy_ba, Dy_ba, ey); ez = fmaf(Nz[2] * Dz_ba, Dz_ba, ez);
+    ex = fmaf(Nx[3] * Dx_bb, Dx_bb, ex); ey = fmaf(Ny[3] * Dy_bb, Dy_bb, ey); ez = fmaf(Nz[3] * Dz_bb, Dz_bb, ez);
+    return iso ? (ex + ey) + ez : fmaf(kx, ex, fmaf(ky, ey, kz * ez));
+}
+
 // MODE 0: KL at the Gauss points; 1 (KN): KL at the nodes, then Q1 interpolation; 2 (ND): stored nodal field.
 // In the nodal modes a slot of the ring holds the nu row next to the u row: copied from the field (ND), or computed
 // from the polynomial of that node line when the row is first used (KN: the table then holds one polynomial per node
@@ -209,7 +231,9 @@ __device__ __forceinline__ void s3_element(const float (&Nx)[4], const float (&N
 // NF: nodal forcing.  The f row sits in the slot as well; the load is taken element by element (mass matrix applied
 // to the corner values of f) and joins the corner contributions before they are gathered, so it needs no other
 // treatment at the boundary of the domain, a tile or a chunk than the stiffness part.
-template <int NX, int M, int MODE, bool NF, int MINB>
+// EO: energy only.  The same march over the same units, but every element adds its own energy (s3_energy) and
+// nothing is gathered, parked or stored: no residual, no seams.
+template <int NX, int M, int MODE, bool NF, int MINB, bool EO>
 __global__ void __launch_bounds__(S3_WARPS * 32, MINB)
 strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G) {
     extern __shared__ __align__(16) float smem[];
@@ -257,8 +281,8 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const unsigned RSB = (unsigned)RS * 4u, RINGB = (unsigned)C * RSB;
     // PREF (wide rows): the parked sums of a node row come back through shared memory, copied one step ahead of their
     // use; narrow rows load them directly (the copy cost more than it hid there: 83 against 77 us on 64^3 x 32)
-    constexpr bool PREF = (NX == 8);
-    float* ring = smem + (KG ? 4 * NX * LW : 0) + (size_t)(warp * SUBS + sub) * (C * RS + (PREF ? NX * LW : 0));
+    constexpr bool PREF = (NX == 8) && !EO;             // (the energy-only variant keeps the layout and leaves the row unused)
+    float* ring = smem + (KG ? 4 * NX * LW : 0) + (size_t)(warp * SUBS + sub) * (C * RS + (NX == 8 ? NX * LW : 0));
     // behind the ring: one row of parked sums (each lane its own pieces)
     float* cbuf = ring + (size_t)C * RS + 4 * lx;
     const unsigned cbuf_s = (unsigned)__cvta_generic_to_shared(cbuf);
@@ -436,7 +460,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     const unsigned TB = (unsigned)T * RSB;
     for (int kk = 0; kk + 1 < nplanes; ++kk) {
         const int k = kbeg + kk;                        // element plane k lies between node planes k and k + 1: plane k is
-        const bool hascarry = (kk > 0) && act;          // finished now, with the partial sums parked one step before;
+        const bool hascarry = !EO && (kk > 0) && act;   // finished now, with the partial sums parked one step before;
         const bool last = (k + 1 == ke);                // the sums of plane k + 1 are parked (plane ke: finished after the march)
         const float wzlo = (k == 0) ? 0.5f : 1.f;
         const float nllo = -gs * fw * wzlo;
@@ -534,6 +558,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                 const float slo = uB[c] - uA[c], sup = uD[c] - uC[c], w0 = uC[c] - uA[c];
                 const float txy = eB - eA, txyu = eD - eC, txz = eC - eA, tyz = sup - slo, txyz = txyu - txy;
                 float Nx[4], Ny[4], Nz[4], r[8];
+                (void)r;
                 if constexpr (KG) {
                     float nu[8];
                     const ulonglong2 cc = *reinterpret_cast<const ulonglong2*>(cpl + c * LW);
@@ -543,6 +568,20 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                     s3_bilerp(nA[c] + nA[c + 1], nB[c] + nB[c + 1], nC[c] + nC[c + 1], nD[c] + nD[c + 1], Nx);   // (q, s)
                     s3_bilerp(yA[c], yA[c + 1], yC[c], yC[c + 1], Ny);                                           // (p, s)
                     s3_bilerp(zA[c], zA[c + 1], zB[c], zB[c + 1], Nz);                                           // (p, q)
+                }
+                if constexpr (EO) {
+                    const float e = s3_energy(Nx, Ny, Nz, eA, slo, w0, txy, txz, tyz, txyz, iso, kx, ky, kz);
+                    enlo += (c == NX - 1) ? e * g3 : e;
+                    if constexpr (NF) {
+                        const float fc[8] = {fA[c], fA[c + 1], fB[c], fB[c + 1], fC[c], fC[c + 1], fD[c], fD[c + 1]};
+                        const float uc[8] = {uA[c], uA[c + 1], uB[c], uB[c + 1], uC[c], uC[c + 1], uD[c], uD[c + 1]};
+                        float m[8], ef = 0.f;
+                        s3_mass(fc, m);
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) ef = fmaf(uc[t], m[t], ef);
+                        elnf += (c == NX - 1) ? ef * g3 : ef;
+                    }
+                    continue;
                 }
                 s3_element(Nx, Ny, Nz, eA, slo, w0, txy, txz, tyz, txyz, iso, kx, ky, kz, r);
                 if constexpr (NF) {
@@ -565,14 +604,14 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                     q000 = r[0]; q010 = r[2]; q001 = r[4]; q011 = r[6];
                 }
             }
-            node(0, fmaf(a100, lm, q000), fmaf(a110, lm, q010), fmaf(a101, lm, q001), fmaf(a111, lm, q011));
+            if constexpr (!EO) node(0, fmaf(a100, lm, q000), fmaf(a110, lm, q010), fmaf(a101, lm, q001), fmaf(a111, lm, q011));
             if (hasf) {
                 float a = wx0 * uA[0];
 #pragma unroll
                 for (int c = 1; c < NX - 1; ++c) a += uA[c];
                 ello = fmaf(wy, fmaf(wxL, uA[NX - 1], a), ello);
             }
-            if (act) { st4(rlo, olo); st4(rup, oup); }
+            if constexpr (!EO) { if (act) { st4(rlo, olo); st4(rup, oup); } }
             rlo += nx; rup += nx;
             oA = oB; ++n;
         }
@@ -597,13 +636,15 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                     ld4(plo, cin);
                 }
             }
+            if constexpr (!EO) {
 #pragma unroll
-            for (int c = 0; c < NX; ++c) {
-                const float raw = pendL1[c] + cin[c];
-                enlo = fmaf(uA[c], raw, enlo);
-                const float s = (c == 0) ? sc0 : (c == NX - 1) ? scL : sc;
-                const float l = (c == 0) ? lw0 * nlrow : (c == NX - 1) ? lwL * nlrow : nlrow;
-                olo[c] = fmaf(s, raw, l);
+                for (int c = 0; c < NX; ++c) {
+                    const float raw = pendL1[c] + cin[c];
+                    enlo = fmaf(uA[c], raw, enlo);
+                    const float s = (c == 0) ? sc0 : (c == NX - 1) ? scL : sc;
+                    const float l = (c == 0) ? lw0 * nlrow : (c == NX - 1) ? lwL * nlrow : nlrow;
+                    olo[c] = fmaf(s, raw, l);
+                }
             }
             if (hasf) {
                 float a = wx0 * uA[0];
@@ -611,7 +652,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
                 for (int c = 1; c < NX - 1; ++c) a += uA[c];
                 ello = fmaf(wy, fmaf(wxL, uA[NX - 1], a), ello);
             }
-            if (act) { st4(plo, olo); st4(pup, pendU1); }
+            if constexpr (!EO) { if (act) { st4(plo, olo); st4(pup, pendU1); } }
             oA = wrapb(oA + RSB); ++n;
         }
         end += (double)enlo; eld += NF ? (double)elnf : (double)(wzlo * ello);   // per-plane sums go to double
@@ -634,7 +675,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
             float part[NX], uT[NX + 1], o[NX];
 #pragma unroll
             for (int c = 0; c < NX; ++c) part[c] = 0.f;
-            if (act) ld4(p, part);
+            if constexpr (!EO) { if (act) ld4(p, part); }
             ldrow(oA, uT);
 #pragma unroll
             for (int c = 0; c < NX; ++c) {
@@ -647,7 +688,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
 #pragma unroll
             for (int c = 1; c < NX - 1; ++c) a += uT[c];
             eltop = fmaf(wy, fmaf(wxL, uT[NX - 1], a), eltop);
-            if (act) st4(p, o);
+            if constexpr (!EO) { if (act) st4(p, o); }
             ptop += nx;
             oA = wrapb(oA + RSB);
         }
@@ -658,8 +699,9 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     // ---- energy partial of this unit: its lanes summed in a fixed order in double
     // NF: `end` holds sum u (K u - F) in units of kap and `eld` sum u_corner (M_e f_e)_corner, so that
     // the load part is fsabs * eld and the diffusion part half of (kap * end + load part)
+    // (energy only: `end` is sum u K u itself, with or without nodal forcing)
     double l = !act ? 0.0 : NF ? (double)fsabs * eld : hasf ? (double)fw * eld : 0.0;
-    double d = !act ? 0.0 : NF ? 0.5 * ((double)kap * end + l) : 0.5 * (double)kap * end;
+    double d = !act ? 0.0 : (NF && !EO) ? 0.5 * ((double)kap * end + l) : 0.5 * (double)kap * end;
     for (int off = LW >> 1; off > 0; off >>= 1) {
         d += __shfl_down_sync(submask, d, off, LW);
         l += __shfl_down_sync(submask, l, off, LW);
@@ -888,15 +930,21 @@ S3Geo geometry3s(const dn_problem& p) {
     return g;
 }
 
-template <int NX, int M, int MODE, bool NF, int MINB>
-cudaError_t launch_nmf(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+template <int NX, int M, int MODE, bool NF, int MINB, bool EO>
+cudaError_t launch_nmfe(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
     const int subs = 32 / g.LW;
     const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * (g.C * g.RS + (NX == 8 ? NX * g.LW : 0)) + (MODE == 0 ? 4 * NX * g.LW : 0));
     const long long per_block = (long long)S3_WARPS * subs;
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
-    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, NF, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, NF, MINB, EO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(strip3d_kernel<NX, M, MODE, NF, MINB>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
+    return launch_dependent(strip3d_kernel<NX, M, MODE, NF, MINB, EO>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
+}
+
+// no output array: the energy-only variant
+template <int NX, int M, int MODE, bool NF, int MINB>
+cudaError_t launch_nmf(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+    return P.r ? launch_nmfe<NX, M, MODE, NF, MINB, false>(P, linepoly, g, s) : launch_nmfe<NX, M, MODE, NF, MINB, true>(P, linepoly, g, s);
 }
 
 // MINB: blocks per SM without nodal forcing; with it, wide rows run two blocks per SM in every mode (s3_minb)
@@ -1002,7 +1050,7 @@ cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t 
         case 7: e = launch_m3<7>(P, linepoly, g, s); break;
         case 8: e = launch_m3<8>(P, linepoly, g, s); break;
     }
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess || P.r == nullptr) return e;       // energy only: no seams
     const long long nA = (long long)P.batch * (g.ntile - 1) * P.nz * (P.nx / 4);
     const long long nB = (long long)P.batch * (g.nchunk - 1) * P.ny * (P.nx / 4);
     if (nA + nB > 0) {

@@ -9,7 +9,7 @@ import torch
 import oracle
 from paper_2007_12792_b200 import binding as B
 from paper_2007_12792_b200 import inputs
-from parity_util import dev, make_problems, run_gpu, check
+from parity_util import dev, make_problems, run_gpu, check, guarded, guards_intact
 
 pytestmark = pytest.mark.gpu
 
@@ -132,3 +132,41 @@ def test_strip3d_random_shapes(seed):
     Jo, _, _, ro = oracle.energy_grad(po, u, gJ=None if gJ is None else gJ.astype(np.float64))
     Jg, rg = run_gpu(pg, u, gJ=gJ)
     check(Jg, rg, Jo, ro, f"seed {seed}: {nx}x{ny}x{nz} b{batch} m{m} mode{mode} flags{flags} f={'nodal' if f is not None else inp.f_const}")
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("nx,ny,nz,batch,m", [(8, 2, 2, 1, 1), (12, 11, 6, 2, 2), (36, 10, 6, 5, 2), (64, 64, 17, 3, 2), (128, 13, 12, 1, 8),
+                                              (136, 6, 7, 2, 2), (256, 17, 5, 1, 3), (256, 40, 30, 2, 6), (16, 8, 300, 1, 1)])
+def test_strip3d_energy_only(nx, ny, nz, batch, m, mode):
+    """dn_energy runs the same march without the gather (every element adds its own energy): against the oracle's J, with
+    constant and with nodal forcing, cubic and stretched cells, boundary values imposed on load."""
+    inp = inputs.random_inputs(3, nx, ny, nz, batch, m, seed=31 + nx + ny + nz, f_const=0.6)
+    u = inputs.random_field(inp.u.shape, 12)
+    nu = inputs.random_positive_field(inp.u.shape, 5) if mode == B.DN_NU_NODAL else None
+    f = inputs.random_field(inp.u.shape, 9, scale=3.0)
+    for ff, flags in ((None, 0), (None, B.DN_IMPOSE_BC_ON_LOAD), (f, 0), (f, B.DN_IMPOSE_BC_ON_LOAD)):
+        po, pg = make_problems(inp, mode, nu=nu, f=ff, flags=flags, bc=(0.8, -0.3))
+        assert B.dn_path_name(pg) == "strip3d"
+        Jo, _, _, _ = oracle.energy_grad(po, u)
+        ws_n = max(B.dn_workspace_bytes(pg), 256)
+        ws_whole, ws = guarded(ws_n)
+        J_whole, J_bytes = guarded(4 * batch)
+        J = J_bytes.view(torch.float32)
+        B.dn_energy(pg, dev(u), J, ws)
+        torch.cuda.synchronize()
+        assert guards_intact(ws_whole, ws_n) and guards_intact(J_whole, 4 * batch)
+        rel = np.abs(J.cpu().numpy().astype(np.float64) - Jo) / np.abs(Jo)
+        assert np.all(rel <= 1e-5), f"{nx}x{ny}x{nz} mode {mode} f={'nodal' if ff is not None else 'const'} flags={flags}: {rel.max():.2e}"
+
+
+def test_strip3d_energy_only_on_cubic_cells_matches_the_fused_call():
+    inp = inputs.random_inputs(3, 48, 48, 48, 3, 2, seed=77, f_const=1.0)
+    for mode in MODES:
+        nu = inputs.random_positive_field(inp.u.shape, 5) if mode == B.DN_NU_NODAL else None
+        po, pg = make_problems(inp, mode, nu=nu)
+        Jo, _, _, _ = oracle.energy_grad(po, inp.u)
+        Jg, _ = run_gpu(pg, inp.u)
+        J = torch.empty(3, device="cuda")
+        B.dn_energy(pg, dev(inp.u), J, B.new_workspace(pg))
+        Je = J.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(Je - Jo) <= 1e-5 * np.abs(Jo)) and np.all(np.abs(Je - Jg) <= 2e-6 * np.abs(Jo))
