@@ -76,7 +76,8 @@ __host__ __device__ constexpr int s2_gs(int m) { return (2 * (m + 1) + 3) / 4 * 
 // NF: nodal forcing.  The f row rides in the ring next to the u row; the load vector is the consistent mass matrix
 // applied to f, a 3 x 3 stencil that separates into a smoothing along x (neighbours by shuffle) and one along y (the row
 // below carried, the row above arriving), with the one-sided weights on the boundary nodes.
-template <int M, int BPS, int MODE, bool NF>
+// EO: energy only.  The same march, but every element adds its own energy and nothing is gathered or stored.
+template <int M, int BPS, int MODE, bool NF, bool EO>
 __global__ void __launch_bounds__(S2_WARPS * 32, BPS)
 strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, const int nchunk, const int nstrip) {
     extern __shared__ __align__(16) float smem[];
@@ -324,6 +325,7 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         if (lane == 31) hir = has_halo ? halo : 0.f;
 
         float Q0 = 0.f, SY0 = 0.f, R0 = 0.f, Qp = 0.f, Tp = 0.f, rout[NE];
+        float es = 0.f;                                 // EO: sum over this lane's elements of N D^2 (= u K u of the element row)
 #pragma unroll
         for (int k = 0; k < NE; ++k) {
             const float uh = c[k];
@@ -355,6 +357,11 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
                 Na = naa + nba; Nb = nab + nbb; Ma = naa + nab; Mb = nba + nbb;
             }
             const float Gxa = Na * Dxa, Gxb = Nb * Dxb, Gya = Ma * Dya, Gyb = Mb * Dyb;
+            if constexpr (EO) {
+                const float e = fmaf(kx, fmaf(Gxa, Dxa, Gxb * Dxb), ky * fmaf(Gya, Dya, Gyb * Dyb));
+                es += (k == NE - 1) ? g3 * e : e;       // the lane's last element may lie beyond the grid
+                continue;
+            }
             const float SXu = Gxa + Gxb, SYu = Gya + Gyb;
             float T = kxa * Gxa;
             T = fmaf(kxb, Gxb, T); T = fmaf(kya, Gya, T); T = fmaf(kyb, Gyb, T);
@@ -371,11 +378,13 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             }
             Qp = Q; Tp = T;
         }
-        // contributions of the element left of this lane's first node
-        const float ql = __shfl_up_sync(0xffffffffu, Qp, 1);
-        const float tl = __shfl_up_sync(0xffffffffu, Tp, 1);
-        rout[0] = fmaf(-ky, SY0, fmaf(ql, lm, -Q0)) + U[0];
-        U[0] = fmaf(tl, lm, R0);
+        if constexpr (!EO) {
+            // contributions of the element left of this lane's first node
+            const float ql = __shfl_up_sync(0xffffffffu, Qp, 1);
+            const float tl = __shfl_up_sync(0xffffffffu, Tp, 1);
+            rout[0] = fmaf(-ky, SY0, fmaf(ql, lm, -Q0)) + U[0];
+            U[0] = fmaf(tl, lm, R0);
+        }
         float gf_up[NE];                                // NF: smoothed f of node row j + 1
         if constexpr (NF) {
             const float4 q = *reinterpret_cast<const float4*>(slot + FOFF + NE * lane);
@@ -387,8 +396,14 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
         }
         if (j >= n0) {                                  // uniform: this unit owns node row j
             // rout is (K u) of node row j: Euler's identity gives the diffusion energy
+            if constexpr (EO) {
+                en += es;                               // element row j belongs to the chunk that owns node row j
 #pragma unroll
-            for (int k = 0; k < NE; ++k) en = fmaf(a[k], rout[k], en);
+                for (int k = 0; k < NE; ++k) rout[k] = 0.f;
+            } else {
+#pragma unroll
+                for (int k = 0; k < NE; ++k) en = fmaf(a[k], rout[k], en);
+            }
             float4 o;
             if constexpr (NF) {
                 // load of node row j: the y-smoothing of the three smoothed rows (row 0 has no row below)
@@ -409,7 +424,7 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             } else {
                 o.x = gsf * rout[0]; o.y = gs * rout[1]; o.z = gs * rout[2]; o.w = gsl * rout[3];
             }
-            if (owner) *reinterpret_cast<float4*>(rrow) = o;
+            if constexpr (!EO) { if (owner) *reinterpret_cast<float4*>(rrow) = o; }
         }
         rrow += nx;
         if constexpr (NF) {
@@ -439,8 +454,10 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
 
     // ---- the top node row of the grid has no element row above it (lo holds it, U what it received)
     if (n1 == ny) {
+        if constexpr (!EO) {
 #pragma unroll
-        for (int k = 0; k < NE; ++k) en = fmaf(lo[k], U[k], en);
+            for (int k = 0; k < NE; ++k) en = fmaf(lo[k], U[k], en);
+        }
         float4 o;
         if constexpr (NF) {
             float F[NE];
@@ -455,7 +472,7 @@ strip2d_kernel(const Params P, const float* __restrict__ rowpoly, const int R, c
             o.x = fmaf(gsf, U[0], 0.5f * nlf); o.y = fmaf(gs, U[1], 0.5f * nl);
             o.z = fmaf(gs, U[2], 0.5f * nl); o.w = fmaf(gsl, U[3], 0.5f * nll);
         }
-        if (owner) *reinterpret_cast<float4*>(rb + (size_t)(ny - 1) * nx) = o;
+        if constexpr (!EO) { if (owner) *reinterpret_cast<float4*>(rb + (size_t)(ny - 1) * nx) = o; }
     }
 
     // ---- energy partial of this unit: owning lanes summed in a fixed order in double
@@ -504,15 +521,21 @@ GeoS geometry_s(const dn_problem& p) {
     return g;
 }
 
-template <int M, int MODE, bool NF>
-cudaError_t launch_mkf(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
+template <int M, int MODE, bool NF, bool EO>
+cudaError_t launch_mkfe(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
     const size_t smem = sizeof(float) * S2_WARPS * S2_DEPTH0 * S2_SLOT0;
     const long long units = (long long)P.batch * g.nchunk * g.nstrip;
     const unsigned blocks = (unsigned)((units + S2_WARPS - 1) / S2_WARPS);
-    const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2, MODE, NF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip2d_kernel<M, 2, MODE, NF, EO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(strip2d_kernel<M, 2, MODE, NF>, dim3(blocks), dim3(S2_WARPS * 32), smem, s, P, rowpoly, g.R,
+    return launch_dependent(strip2d_kernel<M, 2, MODE, NF, EO>, dim3(blocks), dim3(S2_WARPS * 32), smem, s, P, rowpoly, g.R,
                             g.nchunk, g.nstrip);
+}
+
+// no output array: the energy-only variant
+template <int M, int MODE, bool NF>
+cudaError_t launch_mkf(const Params& P, const float* rowpoly, const GeoS& g, cudaStream_t s) {
+    return P.r ? launch_mkfe<M, MODE, NF, false>(P, rowpoly, g, s) : launch_mkfe<M, MODE, NF, true>(P, rowpoly, g, s);
 }
 
 template <int M, int MODE>

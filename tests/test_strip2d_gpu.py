@@ -7,7 +7,7 @@ import torch
 import oracle
 from paper_2007_12792_b200 import binding as B
 from paper_2007_12792_b200 import inputs
-from parity_util import dev, make_problems, run_gpu, check
+from parity_util import dev, make_problems, run_gpu, check, guarded, guards_intact
 
 pytestmark = pytest.mark.gpu
 
@@ -139,3 +139,28 @@ def test_strip2d_random_shapes(seed):
     Jo, _, _, ro = oracle.energy_grad(po, u, gJ=None if gJ is None else gJ.astype(np.float64))
     Jg, rg = run_gpu(pg, u, gJ=gJ)
     check(Jg, rg, Jo, ro, f"seed {seed}: {nx}x{ny} b{batch} m{m} mode{mode} flags{flags} f={'nodal' if f_nodal else inp.f_const}")
+
+
+@pytest.mark.parametrize("mode", KL_MODES)
+@pytest.mark.parametrize("nx,ny,batch,m", [(1024, 40, 2, 4), (1116, 33, 2, 6), (1120, 16, 2, 2), (1124, 21, 1, 3), (2052, 37, 1, 7),
+                                           (4096, 19, 2, 6), (1024, 300, 5, 2), (256, 64, 3, 4)])
+def test_strip2d_energy_only(nx, ny, batch, m, mode):
+    """dn_energy on wide rows runs the same march without the gather (every element adds its own energy): against the
+    oracle's J, with constant and with nodal forcing, boundary values imposed on load.  Rows of 256 nodes take this
+    kernel with nodal forcing only."""
+    inp = inputs.random_inputs(2, nx, ny, 1, batch, m, seed=19 + nx + ny, f_const=0.6)
+    u = inputs.random_field(inp.u.shape, 12)
+    nu = inputs.random_positive_field(inp.u.shape, 5) if mode == B.DN_NU_NODAL else None
+    f = inputs.random_field(inp.u.shape, 9, scale=3.0)
+    for ff, flags in ((None, 0), (None, B.DN_IMPOSE_BC_ON_LOAD), (f, 0), (f, B.DN_IMPOSE_BC_ON_LOAD)):
+        po, pg = make_problems(inp, mode, nu=nu, f=ff, flags=flags, bc=(0.8, -0.3))
+        Jo, _, _, _ = oracle.energy_grad(po, u)
+        ws_n = max(B.dn_workspace_bytes(pg), 256)
+        ws_whole, ws = guarded(ws_n)
+        J_whole, J_bytes = guarded(4 * batch)
+        J = J_bytes.view(torch.float32)
+        B.dn_energy(pg, dev(u), J, ws)
+        torch.cuda.synchronize()
+        assert guards_intact(ws_whole, ws_n) and guards_intact(J_whole, 4 * batch)
+        rel = np.abs(J.cpu().numpy().astype(np.float64) - Jo) / np.abs(Jo)
+        assert np.all(rel <= 1e-5), f"{nx}x{ny} mode {mode} f={'nodal' if ff is not None else 'const'} flags={flags}: {rel.max():.2e}"

@@ -12,11 +12,11 @@ from paper_2007_12792_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 
-def _run_pair(inp, mode, nu=None, flags=0):
+def _run_pair(inp, mode, nu=None, flags=0, f=None):
     w = torch.from_numpy(inp.kl_w).cuda()
     u = torch.from_numpy(inp.u).cuda()
     p = B.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=mode, nu=nu,
-                  kl_modes=inp.kl_modes, kl_w=w, f_const=inp.f_const, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1, flags=flags)
+                  kl_modes=inp.kl_modes, kl_w=w, f_const=inp.f_const, f=f, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1, flags=flags)
     r_ref = torch.empty_like(u); J_ref = torch.empty(inp.batch, device="cuda")
     B.dn_energy_grad(p, u, None, J_ref, r_ref, B.new_workspace(p))
     r = torch.full_like(u, float("nan")); J = torch.full((inp.batch,), float("nan"), device="cuda")
@@ -44,6 +44,17 @@ def test_static_scratch_matches_workspace_entry_point_on_consecutive_calls():
             B.dn_kl_field(inp.dim, inp.nx, inp.ny, inp.nz, inp.batch, inp.kl_modes, torch.from_numpy(inp.kl_w).cuda(), nu)
         J_ref, r_ref, J, r = _run_pair(inp, mode, nu)
         assert np.isfinite(J).all() and np.isfinite(r).all()
+        assert np.all(np.abs(J - J_ref) <= 1e-5 * np.abs(J_ref))
+        assert np.abs(r - r_ref).max() <= 1e-5 * np.abs(r_ref).max()
+
+
+def test_static_scratch_with_nodal_forcing_when_the_strip_table_does_not_fit():
+    """Nodal forcing on a tall grid: the strip kernel's coefficient table (8 x 2100 rows of 64 bytes) exceeds the array,
+    and the kernels that take over must still apply the nodal forcing (the any-size kernel does; the tiled ones cannot)."""
+    for dim, shape in ((2, (256, 2100, 1)), (3, (64, 64, 70))):
+        inp = inputs.random_inputs(dim, *shape, 8, 6 if dim == 2 else 3, seed=21)
+        f = torch.from_numpy(inputs.random_field(inp.u.shape, 5, scale=2.0)).cuda()
+        J_ref, r_ref, J, r = _run_pair(inp, B.DN_NU_KL_GAUSS, f=f)
         assert np.all(np.abs(J - J_ref) <= 1e-5 * np.abs(J_ref))
         assert np.abs(r - r_ref).max() <= 1e-5 * np.abs(r_ref).max()
 
