@@ -113,8 +113,8 @@ dn_status dn_kl_field(const dn_grid* grid, int32_t batch, int32_t kl_modes, cons
                       float* nu_out, void* stream);
 
 /* Energy only (Eq. (pde_loss) in its variational form): J[b], b < B.  u: [B][nz][ny][nx].
- * The same number as the J output of dn_energy_grad up to rounding (the tiled kernels sum element
- * energies here and take J from the residual there). */
+ * The same number as the J output of dn_energy_grad up to rounding (every kernel family sums element
+ * energies here and takes J from the residual there).  Nothing but J and the workspace is written. */
 dn_status dn_energy(const dn_problem* problem, const float* u, float* J, void* workspace,
                     size_t workspace_bytes, void* stream);
 

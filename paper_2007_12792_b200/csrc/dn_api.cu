@@ -442,8 +442,8 @@ int32_t dn_launches_per_call(const dn_problem* p) {
 
 const char* dn_path_name(const dn_problem* p) {
     if (validate(p) != DN_OK) return "invalid";
-    // the fused call (the strip kernels also with nodal forcing); the energy-only call of such a problem runs the tiled
-    // kernel of its dimension or, with nodal forcing, the any-size kernel
+    // the fused call (the strip kernels also with nodal forcing).  The energy-only call runs the same family in 3D; in
+    // 2D the tiled kernel where it can run (constant forcing, rows of at most 2048 nodes), else the strip kernel
     if (!(p->flags & DN_FORCE_GENERIC) && row2d_applicable(*p)) return "row2d";
     if (!(p->flags & DN_FORCE_GENERIC) && strip2d_applicable(*p)) return "strip2d";
     if (!(p->flags & DN_FORCE_GENERIC) && p->f == nullptr && tiled2d_applicable(*p)) return "tiled2d";
