@@ -554,8 +554,9 @@ cudaError_t launch_m(const Params& P, const float* rowpoly, const GeoS& g, cudaS
 // row takes 3 strips of 128).  The tiled kernel is about 1.16 times slower per element in this mode: the strip
 // kernel takes over where its lanes are at most 15 % more than the row, and wherever the tiled kernel cannot run.
 bool strip2d_applicable(const dn_problem& p) {
+    // with nodal forcing also narrow rows (one strip, part of its lanes idle): the other choice is the any-size kernel
     if (!(p.grid.dim == 2 && p.grid.nx % 4 == 0 &&
-          p.grid.nx >= 2 * S2_COLS && p.grid.ny >= 16))
+          p.grid.nx >= (p.f ? 8 : 2 * S2_COLS) && p.grid.ny >= 16))
         return false;
     const long long lanes = (long long)((p.grid.nx - S2_COLS + S2_STRIDE - 1) / S2_STRIDE + 1) * S2_COLS;
     return !tiled2d_applicable(p) || 100 * lanes <= 115ll * p.grid.nx || p.f != nullptr;   // nodal forcing: the only fast kernel

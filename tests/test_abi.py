@@ -134,12 +134,13 @@ def test_kernel_family_and_launch_count_by_shape(L):
 
     name = lambda p: L.dn_path_name(C.byref(p)).decode()
     assert name(prob(2, 2048, 2048, 1)) == "strip2d" and name(prob(2, 256, 256, 1)) == "row2d"
-    assert name(prob(2, 256, 256, 1, f=fake)) == "strip2d"              # nodal forcing: the strip kernel from 256 nodes on
+    assert name(prob(2, 256, 256, 1, f=fake)) == "strip2d"              # nodal forcing: the strip kernel at every width
     assert name(prob(2, 260, 64, 1)) == "tiled2d" and name(prob(2, 132, 64, 1)) == "tiled2d"   # rows the row kernel's lanes do not tile
     for mode in (B.DN_NU_KL_GAUSS, B.DN_NU_NODAL, B.DN_NU_KL_NODAL):
         assert name(prob(2, 8, 2, 1, mode)) == "row2d" and name(prob(2, 128, 4000, 1, mode)) == "row2d"
     assert name(prob(2, 256, 256, 1, B.DN_NU_KL_NODAL)) == "row2d" and name(prob(2, 256, 256, 1, B.DN_NU_NODAL)) == "tiled2d"
-    assert name(prob(2, 128, 64, 1, f=fake)) == "generic" and name(prob(2, 1030, 64, 1)) == "generic"
+    assert name(prob(2, 128, 64, 1, f=fake)) == "strip2d" and name(prob(2, 128, 8, 1, f=fake)) == "generic"   # ... on grids of 16 rows or more
+    assert name(prob(2, 1030, 64, 1)) == "generic"
     for mode in (B.DN_NU_KL_GAUSS, B.DN_NU_NODAL, B.DN_NU_KL_NODAL):
         assert name(prob(3, 256, 256, 256, mode)) == "strip3d" and name(prob(3, 64, 64, 64, mode, f=fake)) == "strip3d"
         assert name(prob(3, 8, 2, 2, mode)) == "strip3d" and name(prob(3, 136, 9, 9, mode)) == "strip3d"

@@ -99,7 +99,9 @@ def test_strip2d_determinism_and_stale_workspace():
 
 @pytest.mark.parametrize("mode", KL_MODES)
 @pytest.mark.parametrize("nx,ny,batch,m", [(1024, 40, 2, 4), (1120, 16, 2, 2), (1124, 21, 1, 3), (2052, 37, 1, 7), (1024, 300, 5, 2),
-                                           (256, 64, 3, 4), (380, 33, 2, 2)])     # with nodal forcing also rows from 256 nodes on
+                                           (256, 64, 3, 4), (380, 33, 2, 2),      # with nodal forcing also narrow rows
+                                           (8, 16, 2, 1), (12, 40, 3, 2), (64, 64, 5, 3), (100, 17, 2, 4), (128, 33, 1, 8), (132, 20, 2, 2),
+                                           (252, 50, 2, 5)])
 def test_strip2d_nodal_forcing(nx, ny, batch, m, mode):
     """Nodal forcing on the strip kernel: the load vector is the consistent mass matrix applied to f (the f row rides in the
     ring with the u row).  All flag combinations, because the Dirichlet columns take the one-sided mass weights."""
@@ -123,7 +125,7 @@ def test_strip2d_random_shapes(seed):
     """Seeded random shapes, modes, flags and forcing kinds on the 2D strip kernel."""
     rng = np.random.default_rng(3000 + seed)
     f_nodal = rng.random() < 0.5
-    nx = 4 * int(rng.integers(64 if f_nodal else 250, 700))       # without nodal forcing rows below about 1000 nodes run tiled2d
+    nx = 4 * int(rng.integers(2 if f_nodal else 250, 700))        # without nodal forcing rows below about 1000 nodes run tiled2d
     ny = int(rng.integers(16, 90))
     batch, m = int(rng.integers(1, 4)), int(rng.integers(1, 9))
     mode = KL_MODES[int(rng.integers(0, 3))]
