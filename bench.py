@@ -38,18 +38,18 @@ FP32_PEAK_LANE_OPS = 148 * 128 * 1.965e9     # SMs x FP32 lanes x max SM clock: 
 # (FADD + FMUL + FFMA + 2 FFMA2).  Each entry names the kernel source it was taken from and the first 16
 # hex digits of its sha256: once that file changes the entry no longer applies and null is reported.
 NCU_CAPTURES = {
-    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 500348160, "fp32_ops_per_element": 57.7,
-                                          "src": "dn_strip2d.cu", "sha": "20e9f8b91a7ab7a5"},
-    "strip2d:cfg2_2d_2048^2_b16_m6:klnodal": {"traffic": 500662784, "fp32_ops_per_element": 44.0,
-                                               "src": "dn_strip2d.cu", "sha": "20e9f8b91a7ab7a5"},
-    "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 789951488, "fp32_ops_per_element": 35.9,
-                                             "src": "dn_strip2d.cu", "sha": "20e9f8b91a7ab7a5"},
-    "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 610791424, "fp32_ops_per_element": 133.8,
-                                        "src": "dn_strip3d.cu", "sha": "8ed5fe52383281c8"},
-    "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 835259904, "fp32_ops_per_element": 142.2,
-                                           "src": "dn_strip3d.cu", "sha": "8ed5fe52383281c8"},
-    "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 556080384, "fp32_ops_per_element": 145.9,
-                                             "src": "dn_strip3d.cu", "sha": "8ed5fe52383281c8"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 501096959, "fp32_ops_per_element": 57.7,
+                                          "src": "dn_strip2d.cu", "sha": "0210a3b72121a90a"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:klnodal": {"traffic": 501012223, "fp32_ops_per_element": 44.0,
+                                               "src": "dn_strip2d.cu", "sha": "0210a3b72121a90a"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 789712383, "fp32_ops_per_element": 35.9,
+                                             "src": "dn_strip2d.cu", "sha": "0210a3b72121a90a"},
+    "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 602841343, "fp32_ops_per_element": 133.8,
+                                        "src": "dn_strip3d.cu", "sha": "a201206c3945b323"},
+    "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 836410368, "fp32_ops_per_element": 142.2,
+                                           "src": "dn_strip3d.cu", "sha": "a201206c3945b323"},
+    "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 557269504, "fp32_ops_per_element": 145.9,
+                                             "src": "dn_strip3d.cu", "sha": "a201206c3945b323"},
     "row2d:cfg1_2d_256^2_b64_m4:kl": {"traffic": 17593600, "fp32_ops_per_element": 51.0,
                                        "src": "dn_row2d.cu", "sha": "bea68ed88174fe35"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
