@@ -24,10 +24,13 @@
  *    those with ix == 0 or ix == nx-1.
  *  - Every pointer is a DEVICE pointer unless its name ends in _host; structs are read
  *    on the host.  The caller owns every buffer.  The library allocates no memory,
- *    keeps no state between calls and never synchronises.  Two exceptions: the *_host entry
- *    points return after their last copy has finished (also when they fail half-way), and
- *    dn_energy_grad_static remembers, per device, the address of its built-in scratch array
- *    (looked up on the first call on that device; it goes stale if the device is reset).
+ *    keeps no state between calls that could change a result, and never synchronises.
+ *    What it does keep: the *_host entry points return after their last copy has finished
+ *    (also when they fail half-way); dn_energy_grad_static remembers, per device, the
+ *    address of its built-in scratch array (looked up on the first call on that device; it
+ *    goes stale if the device is reset); and every host thread remembers the launch geometry
+ *    of the last problem shape it saw per kernel family (a pure function of the shape, the
+ *    mode and the SM count, searched once instead of on every call).
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
  *    enqueued on it in order; outputs are valid once that work has finished.
  *  - Return value: DN_OK or an error code; nothing is thrown, nothing aborts.  When

@@ -1,6 +1,7 @@
 // Internal declarations shared by the CUDA translation units of libdn.
 #pragma once
 
+#include <cstring>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -16,6 +17,22 @@ namespace dn {
 constexpr int kAlign = 256;
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+// A launch geometry is a pure function of the problem's shape and mode and of the SM count of the current device.  Each
+// kernel family remembers the last one it searched for, per host thread, so that a training loop pays the search once.
+struct GeoKey { int v[10]; };
+inline GeoKey geo_key(const dn_problem& p, int sms) {
+    return GeoKey{{p.grid.dim, p.grid.nx, p.grid.ny, (p.grid.dim == 3) ? p.grid.nz : 1, p.batch, (int)p.nu_mode, p.kl_modes,
+                   p.f != nullptr ? 1 : 0, sms, 1}};
+}
+template <class G, class F>
+G memo_geometry(const dn_problem& p, int sms, F search) {
+    thread_local GeoKey last{};                        // all zero: equal to no real key (the last entry of one is 1)
+    thread_local G geo{};
+    const GeoKey k = geo_key(p, sms);
+    if (memcmp(k.v, last.v, sizeof k.v) != 0) { geo = search(); last = k; }
+    return geo;
+}
 
 enum Path { PATH_GENERIC = 0, PATH_TILED2D = 1, PATH_TILED3D = 2, PATH_STRIP2D = 3, PATH_STRIP3D = 4, PATH_ROW2D = 5 };
 

@@ -420,7 +420,7 @@ int r2_sm_count() {
 int r2_nxl(int nx) { return (nx > 128) ? 8 : 4; }       // nodes per lane
 int r2_minb(int nxl) { return (nxl == 8) ? 3 : 4; }     // resident blocks of 4 warps per SM the kernel is compiled for
 
-R2Geo geometry_r(const dn_problem& p) {
+R2Geo geometry_r_search(const dn_problem& p) {
     R2Geo g{};
     const int nx = p.grid.nx, ny = p.grid.ny;
     const int NX = r2_nxl(nx);
@@ -444,6 +444,10 @@ R2Geo geometry_r(const dn_problem& p) {
     g.nchunk = (ny + g.R - 1) / g.R;
     g.units = (long long)p.batch * g.nchunk;
     return g;
+}
+
+R2Geo geometry_r(const dn_problem& p) {
+    return memo_geometry<R2Geo>(p, r2_sm_count(), [&]() { return geometry_r_search(p); });
 }
 
 template <int NX, int M, int MODE, int MINB>

@@ -500,7 +500,7 @@ int s2_sm_count() {
     return n;
 }
 
-GeoS geometry_s(const dn_problem& p) {
+GeoS geometry_s_search(const dn_problem& p) {
     GeoS g{};
     const int nx = p.grid.nx, ny = p.grid.ny;
     g.nstrip = (nx <= S2_COLS) ? 1 : (nx - S2_COLS + S2_STRIDE - 1) / S2_STRIDE + 1;
@@ -519,6 +519,10 @@ GeoS geometry_s(const dn_problem& p) {
     g.R = bestR;
     g.nchunk = (ny + g.R - 1) / g.R;
     return g;
+}
+
+GeoS geometry_s(const dn_problem& p) {
+    return memo_geometry<GeoS>(p, s2_sm_count(), [&]() { return geometry_s_search(p); });
 }
 
 template <int M, int MODE, bool NF, bool EO>

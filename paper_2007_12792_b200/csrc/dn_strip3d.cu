@@ -892,7 +892,7 @@ int s3_slot_floats(int nxl, int lw, int mode, int m, bool nf) {
     return rows * urow + (mode == DN_NU_KL_GAUSS ? 2 * s3_gs(m) : mode == DN_NU_KL_NODAL ? s3_gs(m) : 0);
 }
 
-S3Geo geometry3s(const dn_problem& p) {
+S3Geo geometry3s_search(const dn_problem& p) {
     S3Geo g{};
     const int nx = p.grid.nx, ny = p.grid.ny, nz = p.grid.nz;
     const int NX = s3_nxl(nx), minb = s3_minb(NX, p.nu_mode, p.f != nullptr);
@@ -928,6 +928,10 @@ S3Geo geometry3s(const dn_problem& p) {
     }
     g.C = g.Ry + 2 + S3_D;
     return g;
+}
+
+S3Geo geometry3s(const dn_problem& p) {
+    return memo_geometry<S3Geo>(p, s3_sm_count(), [&]() { return geometry3s_search(p); });
 }
 
 template <int NX, int M, int MODE, bool NF, int MINB, bool EO>

@@ -616,7 +616,7 @@ int sm_count() {
     return n;
 }
 
-Geo2 geometry(const dn_problem& p) {
+Geo2 geometry_search(const dn_problem& p) {
     Geo2 g{};
     const int nx = p.grid.nx, ny = p.grid.ny;
     g.K = (nx > 128) ? 2 : 1;
@@ -644,6 +644,10 @@ Geo2 geometry(const dn_problem& p) {
     g.smem = sizeof(float) * ((size_t)g.WY * (g.R + 2) * g.GS + (size_t)g.WY * 2 * T2_MAX_WARPS * 2 +
                               (m ? 0 : (size_t)g.WY * T2_STAGES * 2 * ring_row));      // the ring serves the nodal variant
     return g;
+}
+
+Geo2 geometry(const dn_problem& p) {
+    return memo_geometry<Geo2>(p, sm_count(), [&]() { return geometry_search(p); });
 }
 
 template <int K, int M, bool FULL, bool KN>

@@ -575,7 +575,7 @@ int sm_count3() {
     return n;
 }
 
-Geo3 geometry3(const dn_problem& p) {
+Geo3 geometry3_search(const dn_problem& p) {
     Geo3 best{};
     const int nx = p.grid.nx, ny = p.grid.ny, nz = p.grid.nz;
     const int WX = (nx + 127) / 128;
@@ -618,6 +618,10 @@ Geo3 geometry3(const dn_problem& p) {
         }
     }
     return best;
+}
+
+Geo3 geometry3(const dn_problem& p) {
+    return memo_geometry<Geo3>(p, sm_count3(), [&]() { return geometry3_search(p); });
 }
 
 template <int M, bool FULL, bool NARROW>

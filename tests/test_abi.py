@@ -167,3 +167,34 @@ def test_binding_rejects_host_tensors_and_missing_library(monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libdn.so")
     with pytest.raises(RuntimeError):
         B.lib()
+
+
+def test_remembered_launch_geometry_does_not_leak_between_shapes(L):
+    """Each kernel family keeps the launch geometry of the last shape it saw; alternating shapes, modes and forcing kinds
+    must give what a first call gives (sizes differ between them, so a stale geometry would show)."""
+    from paper_2007_12792_b200 import binding as B
+    import threading
+    fake = 0x100000
+
+    def prob(dim, nx, ny, nz, batch, m, mode=B.DN_NU_KL_GAUSS, f=None):
+        p = B.DnProblem()
+        p.grid = B.DnGrid(dim, nx, ny, nz)
+        p.batch = batch; p.nu_mode = mode; p.kl_modes = m; p.kl_w = fake
+        p.nu = fake if mode == B.DN_NU_NODAL else None
+        p.f = f
+        return p
+
+    probs = [prob(3, 256, 256, 256, 4, 3), prob(3, 64, 64, 64, 32, 2), prob(3, 256, 256, 256, 4, 3, B.DN_NU_NODAL),
+             prob(3, 256, 256, 256, 4, 3, f=fake), prob(3, 256, 256, 256, 5, 3), prob(2, 2048, 2048, 1, 16, 6),
+             prob(2, 2048, 2044, 1, 16, 6), prob(2, 256, 256, 1, 64, 4), prob(2, 256, 250, 1, 64, 4), prob(2, 64, 64, 1, 8, 2)]
+    sizes = lambda: [(L.dn_workspace_bytes(C.byref(p)), L.dn_cg_workspace_bytes(C.byref(p)), L.dn_launches_per_call(C.byref(p)))
+                     for p in probs]
+    first = sizes()
+    assert len(set(s[0] for s in first)) == len(first)          # every shape has its own scratch size
+    assert sizes() == first and list(reversed([
+        (L.dn_workspace_bytes(C.byref(p)), L.dn_cg_workspace_bytes(C.byref(p)), L.dn_launches_per_call(C.byref(p)))
+        for p in reversed(probs)])) == first
+    out = {}
+    ts = [threading.Thread(target=lambda i=i: out.__setitem__(i, sizes())) for i in range(4)]   # per-thread memory
+    [t.start() for t in ts]; [t.join() for t in ts]
+    assert all(out[i] == first for i in range(4))
