@@ -1,6 +1,7 @@
-"""Parity at the full benchmark sizes (2D 2048^2 x 16 and 3D 256^3 x 4), in the launch configuration the
-benchmark times: every node of the residual and every sample's energy against the oracle's full pass, in
-all three diffusivity modes, plus properties that hold at any size."""
+"""Parity at the full benchmark sizes (2D 2048^2 x 16 and 3D 256^3 x 4, and the two mid-size workloads 2D 256^2 x 64 and
+3D 64^3 x 32), in the launch configuration the benchmark times: every node of the residual and every sample's energy
+against the oracle's full pass, in all three diffusivity modes, plus properties that hold at any size; and the
+energy-only call on the same inputs."""
 import numpy as np
 import pytest
 import torch
@@ -12,11 +13,11 @@ from parity_util import dev, J_RTOL, R_RTOL, guarded, guards_intact
 
 pytestmark = pytest.mark.gpu
 
-PATHS = {2: ("strip2d",), 4: ("strip3d",)}
+PATHS = {1: ("row2d", "tiled2d"), 2: ("strip2d",), 3: ("strip3d",), 4: ("strip3d",)}   # cfg1 with a stored field: tiled2d
 
 
 @pytest.mark.parametrize("mode", [B.DN_NU_KL_GAUSS, B.DN_NU_NODAL, B.DN_NU_KL_NODAL])
-@pytest.mark.parametrize("cfg", [2, 4])
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4])
 def test_fullsize_every_node(cfg, mode):
     inp = inputs.make_inputs(cfg)
     ud = dev(inp.u)
@@ -39,6 +40,9 @@ def test_fullsize_every_node(cfg, mode):
     torch.cuda.synchronize()
     assert guards_intact(r_whole, 4 * n) and guards_intact(ws_whole, ws_n)
     Jg = J.cpu().numpy().astype(np.float64)
+    Je = torch.full((inp.batch,), float("nan"), device="cuda")
+    B.dn_energy(pg, ud, Je, ws)                                     # the energy-only call: same inputs, same workspace
+    Je = Je.cpu().numpy().astype(np.float64)
     nu_h = nu_d.cpu().numpy() if nu_d is not None else None        # the oracle reads the same float32 field
     po = oracle.Problem(dim=inp.dim, nx=inp.nx, ny=inp.ny, nz=inp.nz, batch=inp.batch, nu_mode=mode, nu=nu_h,
                         kl_modes=inp.kl_modes, kl_w=inp.kl_w, f_const=inp.f_const, bc_x0=inp.bc_x0, bc_x1=inp.bc_x1)
@@ -46,6 +50,7 @@ def test_fullsize_every_node(cfg, mode):
     Jo, _, _, ro = oracle.energy_grad(po, inp.u)
     rel = np.abs(Jg - Jo) / np.abs(Jo)
     assert np.all(rel <= J_RTOL), f"J rel err {rel} J*={Jo}"
+    assert np.all(np.abs(Je - Jo) <= J_RTOL * np.abs(Jo)), f"dn_energy: J rel err {np.abs(Je - Jo) / np.abs(Jo)}"
     scale = np.abs(ro).max()
     worst = 0.0
     for b in range(inp.batch):                                      # sample by sample: bounded host memory
