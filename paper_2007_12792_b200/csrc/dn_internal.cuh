@@ -22,7 +22,8 @@ inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a
 // kernel family remembers the last one it searched for, per host thread, so that a training loop pays the search once.
 struct GeoKey { int v[10]; };
 inline GeoKey geo_key(const dn_problem& p, int sms) {
-    return GeoKey{{p.grid.dim, p.grid.nx, p.grid.ny, (p.grid.dim == 3) ? p.grid.nz : 1, p.batch, (int)p.nu_mode, p.kl_modes,
+    return GeoKey{{p.grid.dim, p.grid.nx, p.grid.ny, (p.grid.dim == 3) ? p.grid.nz : 1, p.batch, (int)p.nu_mode,
+                   (p.nu_mode == DN_NU_NODAL) ? 0 : p.kl_modes,     // not read with a stored field
                    p.f != nullptr ? 1 : 0, sms, 1}};
 }
 template <class G, class F>

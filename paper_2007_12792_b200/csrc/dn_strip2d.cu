@@ -586,7 +586,7 @@ int strip2d_rowpoly_stride(int kl_modes) { return s2_gs(kl_modes); }
 cudaError_t launch_strip2d(const Params& P, const float* rowpoly, cudaStream_t s) {
     dn_problem p{};
     p.grid.dim = 2; p.grid.nx = P.nx; p.grid.ny = P.ny; p.grid.nz = 1; p.batch = P.batch;
-    p.nu_mode = P.nu_mode; p.kl_modes = P.m;
+    p.nu_mode = P.nu_mode; p.kl_modes = P.m; p.f = P.f;
     const GeoS g = geometry_s(p);
     if (P.nu_mode == DN_NU_NODAL) return launch_mk<1, 2>(P, rowpoly, g, s);
     switch (P.m) {
