@@ -38,12 +38,12 @@ FP32_PEAK_LANE_OPS = 148 * 128 * 1.965e9     # SMs x FP32 lanes x max SM clock: 
 # (FADD + FMUL + FFMA + 2 FFMA2).  Each entry names the kernel source it was taken from and the first 16
 # hex digits of its sha256: once that file changes the entry no longer applies and null is reported.
 NCU_CAPTURES = {
-    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 501096959, "fp32_ops_per_element": 57.7,
-                                          "src": "dn_strip2d.cu", "sha": "0210a3b72121a90a"},
-    "strip2d:cfg2_2d_2048^2_b16_m6:klnodal": {"traffic": 501012223, "fp32_ops_per_element": 44.0,
-                                               "src": "dn_strip2d.cu", "sha": "0210a3b72121a90a"},
-    "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 789712383, "fp32_ops_per_element": 35.9,
-                                             "src": "dn_strip2d.cu", "sha": "0210a3b72121a90a"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:kl": {"traffic": 500101632, "fp32_ops_per_element": 57.7,
+                                          "src": "dn_strip2d.cu", "sha": "5ba6034b044c172f"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:klnodal": {"traffic": 500000000, "fp32_ops_per_element": 44.0,
+                                               "src": "dn_strip2d.cu", "sha": "5ba6034b044c172f"},
+    "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 790611967, "fp32_ops_per_element": 35.9,
+                                             "src": "dn_strip2d.cu", "sha": "5ba6034b044c172f"},
     "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 602841343, "fp32_ops_per_element": 133.8,
                                         "src": "dn_strip3d.cu", "sha": "a201206c3945b323"},
     "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 836410368, "fp32_ops_per_element": 142.2,
