@@ -233,7 +233,9 @@ __device__ __forceinline__ float s3_energy(const float (&Nx)[4], const float (&N
 // treatment at the boundary of the domain, a tile or a chunk than the stiffness part.
 // EO: energy only.  The same march over the same units, but every element adds its own energy (s3_energy) and
 // nothing is gathered, parked or stored: no residual, no seams.
-template <int NX, int M, int MODE, bool NF, int MINB, bool EO>
+// LWC: lanes per unit at compile time (8 nodes per lane: 32, or 16 on rows of 65 to 128 nodes), or 0: taken from G
+// (a lane count known to the compiler is worth 3 to 9 % on 256-wide rows).
+template <int NX, int M, int MODE, bool NF, int MINB, bool EO, int LWC>
 __global__ void __launch_bounds__(S3_WARPS * 32, MINB)
 strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G) {
     extern __shared__ __align__(16) float smem[];
@@ -244,8 +246,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
     constexpr int CF = KG ? 2 * GS : KN ? GS : 0;       // coefficient floats per slot (KG: Gauss rows q = a, b of an element row)
     constexpr int CFQ = CF / 4;                         // ... in 16-byte pieces
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // 8 nodes per lane are used on rows of more than 128 nodes only: then a unit is a whole warp
-    const int LW = (NX == 8) ? 32 : G.LW, lwsh = (NX == 8) ? 5 : G.lwsh, SUBS = 32 >> lwsh;
+    const int LW = LWC ? LWC : G.LW, lwsh = (LWC == 32) ? 5 : (LWC == 16) ? 4 : G.lwsh, SUBS = 32 >> lwsh;
     const int sub = lane >> lwsh, lx = lane & (LW - 1);
     const unsigned submask = (LW == 32) ? 0xffffffffu : (((1u << LW) - 1u) << (sub * LW));
     const int nx = P.nx, ny = P.ny, nz = P.nz;
@@ -882,7 +883,13 @@ int s3_sm_count() {
 constexpr size_t S3_SMEM_SM = 233472;              // shared memory of an SM; a block also reserves 1 KiB
 constexpr size_t S3_SMEM_BLOCK = 232448;           // most a block can ask for
 
-int s3_nxl(int nx) { return (nx > 128) ? 8 : 4; }  // nodes per lane (8 on narrow rows was slower: 89 against 79 us on 64^3 x 32)
+// Nodes per lane: 8 on rows of more than 128 nodes; also on rows of 65 to 128 nodes (two units per warp) with KL at the
+// Gauss points and constant forcing, where it is 8 to 9 % faster than 4 (128^3 x 16: 263 against 290 us; with KL at the
+// nodes or a stored field it is not: 314 against 306, 288 against 284 us); on narrower rows 4 (64^3 x 32: 79 against 89 us).
+int s3_nxl(int nx, int mode, bool nf) {
+    if (nx > 128) return 8;
+    return (nx > 64 && nx % 8 == 0 && mode == DN_NU_KL_GAUSS && !nf) ? 8 : 4;
+}
 // resident blocks of 4 warps per SM the kernel is compiled for: the nodal modes keep two rows per slot and trade
 // warps for taller tiles on wide rows
 int s3_minb(int nxl, int mode, bool nf) { return (nxl == 8) ? ((mode == DN_NU_KL_GAUSS && !nf) ? 3 : 2) : 4; }
@@ -895,7 +902,7 @@ int s3_slot_floats(int nxl, int lw, int mode, int m, bool nf) {
 S3Geo geometry3s_search(const dn_problem& p) {
     S3Geo g{};
     const int nx = p.grid.nx, ny = p.grid.ny, nz = p.grid.nz;
-    const int NX = s3_nxl(nx), minb = s3_minb(NX, p.nu_mode, p.f != nullptr);
+    const int NX = s3_nxl(nx, p.nu_mode, p.f != nullptr), minb = s3_minb(NX, p.nu_mode, p.f != nullptr);
     g.LW = 8; g.lwsh = 3;
     while (g.LW * NX < nx) { g.LW *= 2; ++g.lwsh; }
     const int subs = 32 / g.LW;
@@ -934,21 +941,22 @@ S3Geo geometry3s(const dn_problem& p) {
     return memo_geometry<S3Geo>(p, s3_sm_count(), [&]() { return geometry3s_search(p); });
 }
 
-template <int NX, int M, int MODE, bool NF, int MINB, bool EO>
+template <int NX, int M, int MODE, bool NF, int MINB, bool EO, int LWC>
 cudaError_t launch_nmfe(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
     const int subs = 32 / g.LW;
     const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * (g.C * g.RS + (NX == 8 ? NX * g.LW : 0)) + (MODE == 0 ? 4 * NX * g.LW : 0));
     const long long per_block = (long long)S3_WARPS * subs;
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
-    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, NF, MINB, EO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, NF, MINB, EO, LWC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(strip3d_kernel<NX, M, MODE, NF, MINB, EO>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
+    return launch_dependent(strip3d_kernel<NX, M, MODE, NF, MINB, EO, LWC>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
 }
 
 // no output array: the energy-only variant
-template <int NX, int M, int MODE, bool NF, int MINB>
+template <int NX, int M, int MODE, bool NF, int MINB, int LWC = (NX == 8 ? 32 : 0)>
 cudaError_t launch_nmf(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
-    return P.r ? launch_nmfe<NX, M, MODE, NF, MINB, false>(P, linepoly, g, s) : launch_nmfe<NX, M, MODE, NF, MINB, true>(P, linepoly, g, s);
+    return P.r ? launch_nmfe<NX, M, MODE, NF, MINB, false, LWC>(P, linepoly, g, s)
+               : launch_nmfe<NX, M, MODE, NF, MINB, true, LWC>(P, linepoly, g, s);
 }
 
 // MINB: blocks per SM without nodal forcing; with it, wide rows run two blocks per SM in every mode (s3_minb)
@@ -960,9 +968,10 @@ cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cu
 
 template <int M>
 cudaError_t launch_m3(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
-    const bool wide = (s3_nxl(P.nx) == 8);
+    const bool wide = (s3_nxl(P.nx, P.nu_mode, P.f != nullptr) == 8);
     if (P.nu_mode == DN_NU_KL_NODAL)
         return wide ? launch_nm<8, M, 1, 2>(P, linepoly, g, s) : launch_nm<4, M, 1, 4>(P, linepoly, g, s);
+    if (wide && P.nx <= 128) return launch_nmf<8, M, 0, false, 3, 16>(P, linepoly, g, s);      // two units per warp
     return wide ? launch_nm<8, M, 0, 3>(P, linepoly, g, s) : launch_nm<4, M, 0, 4>(P, linepoly, g, s);
 }
 
@@ -1043,7 +1052,7 @@ cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t 
     const S3Geo g = geometry3s(s3_problem_of(P));
     cudaError_t e = cudaErrorInvalidValue;
     if (P.nu_mode == DN_NU_NODAL) {
-        e = (s3_nxl(P.nx) == 8) ? launch_nm<8, 1, 2, 2>(P, linepoly, g, s) : launch_nm<4, 1, 2, 4>(P, linepoly, g, s);
+        e = (s3_nxl(P.nx, P.nu_mode, P.f != nullptr) == 8) ? launch_nm<8, 1, 2, 2>(P, linepoly, g, s) : launch_nm<4, 1, 2, 4>(P, linepoly, g, s);
     } else switch (P.m) {
         case 1: e = launch_m3<1>(P, linepoly, g, s); break;
         case 2: e = launch_m3<2>(P, linepoly, g, s); break;

@@ -16,7 +16,9 @@ pytestmark = pytest.mark.gpu
 # (nx, ny, nz, batch, m)
 SIZES = [(8, 2, 2, 1, 1), (12, 11, 6, 2, 2), (32, 9, 7, 3, 3), (28, 45, 5, 1, 2), (36, 10, 6, 5, 2), (64, 20, 3, 1, 2),
          (60, 37, 6, 2, 3), (64, 64, 17, 3, 2), (100, 7, 9, 2, 4), (128, 13, 12, 1, 8), (132, 9, 5, 1, 3), (136, 6, 7, 2, 2),
-         (200, 5, 4, 1, 5), (256, 17, 5, 1, 3), (256, 40, 30, 2, 6), (64, 150, 40, 9, 2), (16, 8, 300, 1, 1)]
+         (200, 5, 4, 1, 5), (256, 17, 5, 1, 3), (256, 40, 30, 2, 6), (64, 150, 40, 9, 2), (16, 8, 300, 1, 1),
+         # rows of 65 to 128 nodes that are a multiple of 8: 8 nodes per lane and two units per warp (KL at the Gauss points)
+         (72, 9, 7, 3, 2), (96, 20, 5, 2, 3), (120, 6, 6, 1, 4), (128, 40, 9, 5, 2), (88, 3, 30, 7, 1)]
 
 
 MODES = [B.DN_NU_KL_GAUSS, B.DN_NU_KL_NODAL, B.DN_NU_NODAL]   # KL at the Gauss points / at the nodes (in the kernel), stored nodal field
