@@ -44,12 +44,12 @@ NCU_CAPTURES = {
                                                "src": "dn_strip2d.cu", "sha": "5ba6034b044c172f"},
     "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 790611967, "fp32_ops_per_element": 35.9,
                                              "src": "dn_strip2d.cu", "sha": "5ba6034b044c172f"},
-    "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 602841343, "fp32_ops_per_element": 133.8,
-                                        "src": "dn_strip3d.cu", "sha": "a201206c3945b323"},
-    "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 836410368, "fp32_ops_per_element": 142.2,
-                                           "src": "dn_strip3d.cu", "sha": "a201206c3945b323"},
-    "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 557269504, "fp32_ops_per_element": 145.9,
-                                             "src": "dn_strip3d.cu", "sha": "a201206c3945b323"},
+    "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 611784192, "fp32_ops_per_element": 133.8,
+                                        "src": "dn_strip3d.cu", "sha": "c63cbb0fac0e796f"},
+    "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 835513600, "fp32_ops_per_element": 142.2,
+                                           "src": "dn_strip3d.cu", "sha": "c63cbb0fac0e796f"},
+    "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 556568064, "fp32_ops_per_element": 145.9,
+                                             "src": "dn_strip3d.cu", "sha": "c63cbb0fac0e796f"},
     "row2d:cfg1_2d_256^2_b64_m4:kl": {"traffic": 17593600, "fp32_ops_per_element": 51.0,
                                        "src": "dn_row2d.cu", "sha": "bea68ed88174fe35"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
