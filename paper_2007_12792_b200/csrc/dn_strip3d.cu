@@ -233,8 +233,8 @@ __device__ __forceinline__ float s3_energy(const float (&Nx)[4], const float (&N
 // treatment at the boundary of the domain, a tile or a chunk than the stiffness part.
 // EO: energy only.  The same march over the same units, but every element adds its own energy (s3_energy) and
 // nothing is gathered, parked or stored: no residual, no seams.
-// LWC: lanes per unit at compile time (8 nodes per lane: 32, or 16 on rows of 65 to 128 nodes), or 0: taken from G
-// (a lane count known to the compiler is worth 3 to 9 % on 256-wide rows).
+// LWC: lanes per unit at compile time (32 or 16), or 0: taken from G (8 lanes, and every layout with nodal forcing).
+// A lane count known to the compiler is worth 3 to 9 % on 256-wide rows and 3 to 4 % on 64-wide ones.
 template <int NX, int M, int MODE, bool NF, int MINB, bool EO, int LWC>
 __global__ void __launch_bounds__(S3_WARPS * 32, MINB)
 strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G) {
@@ -963,6 +963,10 @@ cudaError_t launch_nmf(const Params& P, const float* linepoly, const S3Geo& g, c
 template <int NX, int M, int MODE, int MINB>
 cudaError_t launch_nm(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
     if (P.f) return launch_nmf<NX, M, MODE, true, (NX == 8 ? 2 : 4)>(P, linepoly, g, s);
+    if constexpr (NX == 4) {                            // 16 or 32 lanes per unit known to the compiler: 3 to 4 % (64^3 x 32: 78.8 -> 76.2 us)
+        if (g.LW == 16) return launch_nmf<NX, M, MODE, false, MINB, 16>(P, linepoly, g, s);
+        if (g.LW == 32) return launch_nmf<NX, M, MODE, false, MINB, 32>(P, linepoly, g, s);
+    }
     return launch_nmf<NX, M, MODE, false, MINB>(P, linepoly, g, s);
 }
 
