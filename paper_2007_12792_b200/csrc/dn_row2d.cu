@@ -70,7 +70,8 @@ struct R2Geo {
 };
 
 // MODE 0: KL at the Gauss points; 1 (KN): KL at the nodes, then Q1 interpolation; 2 (ND): stored nodal field
-template <int NX, int M, int MODE, int MINB>
+// LWC: lanes per unit at compile time (16 or 32), or 0: taken from G (8 lanes)
+template <int NX, int M, int MODE, int MINB, int LWC>
 __global__ void __launch_bounds__(R2_WARPS * 32, MINB)
 row2d_kernel(const Params P, const float* __restrict__ rowpoly, const R2Geo G) {
     extern __shared__ __align__(16) float smem[];
@@ -81,7 +82,7 @@ row2d_kernel(const Params P, const float* __restrict__ rowpoly, const R2Geo G) {
     constexpr int R2_DEPTH = r2_depth(MODE);
     constexpr int CFQ = ND ? 0 : GS / 4;                // 16-byte pieces of a coefficient row
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int LW = G.LW, lwsh = G.lwsh, SUBS = 32 >> lwsh;
+    const int LW = LWC ? LWC : G.LW, lwsh = (LWC == 32) ? 5 : (LWC == 16) ? 4 : G.lwsh, SUBS = 32 >> lwsh;
     const int sub = lane >> lwsh, lx = lane & (LW - 1);
     const unsigned submask = (LW == 32) ? 0xffffffffu : (((1u << LW) - 1u) << (sub * LW));
     const int nx = P.nx, ny = P.ny;
@@ -450,15 +451,22 @@ R2Geo geometry_r(const dn_problem& p) {
     return memo_geometry<R2Geo>(p, r2_sm_count(), [&]() { return geometry_r_search(p); });
 }
 
-template <int NX, int M, int MODE, int MINB>
-cudaError_t launch_r(const Params& P, const float* rowpoly, const R2Geo& g, cudaStream_t s) {
+template <int NX, int M, int MODE, int MINB, int LWC>
+cudaError_t launch_rl(const Params& P, const float* rowpoly, const R2Geo& g, cudaStream_t s) {
     const int subs = 32 / g.LW;
     const size_t smem = sizeof(float) * ((size_t)R2_WARPS * subs * r2_depth(MODE) * g.RS + (MODE == 0 ? 4 * NX * g.LW : 0));
     const long long per_block = (long long)R2_WARPS * subs;
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
-    const cudaError_t e = cudaFuncSetAttribute(row2d_kernel<NX, M, MODE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(row2d_kernel<NX, M, MODE, MINB, LWC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(row2d_kernel<NX, M, MODE, MINB>, dim3(blocks), dim3(R2_WARPS * 32), smem, s, P, rowpoly, g);
+    return launch_dependent(row2d_kernel<NX, M, MODE, MINB, LWC>, dim3(blocks), dim3(R2_WARPS * 32), smem, s, P, rowpoly, g);
+}
+
+template <int NX, int M, int MODE, int MINB>
+cudaError_t launch_r(const Params& P, const float* rowpoly, const R2Geo& g, cudaStream_t s) {
+    if (g.LW == 32) return launch_rl<NX, M, MODE, MINB, 32>(P, rowpoly, g, s);
+    if (g.LW == 16) return launch_rl<NX, M, MODE, MINB, 16>(P, rowpoly, g, s);
+    return launch_rl<NX, M, MODE, MINB, 0>(P, rowpoly, g, s);
 }
 
 template <int M>
