@@ -235,7 +235,9 @@ __device__ __forceinline__ float s3_energy(const float (&Nx)[4], const float (&N
 // nothing is gathered, parked or stored: no residual, no seams.
 // LWC: lanes per unit at compile time (32 or 16), or 0: taken from G (8 lanes, and every layout with nodal forcing).
 // A lane count known to the compiler is worth 3 to 9 % on 256-wide rows and 3 to 4 % on 64-wide ones.
-template <int NX, int M, int MODE, bool NF, int MINB, bool EO, int LWC>
+// ISO: the cells are known to be cubes when the kernel is compiled (the scaling of the sums of nu by kx, ky, kz and the
+// branch around it go: 2 % on 256^3 x 4); false: decided from the spacings at run time.
+template <int NX, int M, int MODE, bool NF, int MINB, bool EO, int LWC, bool ISO>
 __global__ void __launch_bounds__(S3_WARPS * 32, MINB)
 strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G) {
     extern __shared__ __align__(16) float smem[];
@@ -325,7 +327,7 @@ strip3d_kernel(const Params P, const float* __restrict__ linepoly, const S3Geo G
         if (P.bc0_b) bc0 = __ldg(P.bc0_b + b);
         if (P.bc1_b) bc1 = __ldg(P.bc1_b + b);
     }
-    const bool iso = (P.hx == P.hy) && (P.hy == P.hz);
+    const bool iso = ISO ? true : ((P.hx == P.hy) && (P.hy == P.hz));
     const float W8 = 0.125f * P.hx * P.hy * P.hz;
     const float kx = W8 / (P.hx * P.hx), ky = W8 / (P.hy * P.hy), kz = W8 / (P.hz * P.hz);
     const float kap = iso ? kx : 1.f;                   // isotropic cells: one scale applied at the end
@@ -941,15 +943,24 @@ S3Geo geometry3s(const dn_problem& p) {
     return memo_geometry<S3Geo>(p, s3_sm_count(), [&]() { return geometry3s_search(p); });
 }
 
-template <int NX, int M, int MODE, bool NF, int MINB, bool EO, int LWC>
-cudaError_t launch_nmfe(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+template <int NX, int M, int MODE, bool NF, int MINB, bool EO, int LWC, bool ISO>
+cudaError_t launch_nmfei(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
     const int subs = 32 / g.LW;
     const size_t smem = sizeof(float) * ((size_t)S3_WARPS * subs * (g.C * g.RS + (NX == 8 ? NX * g.LW : 0)) + (MODE == 0 ? 4 * NX * g.LW : 0));
     const long long per_block = (long long)S3_WARPS * subs;
     const unsigned blocks = (unsigned)((g.units + per_block - 1) / per_block);
-    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, NF, MINB, EO, LWC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = cudaFuncSetAttribute(strip3d_kernel<NX, M, MODE, NF, MINB, EO, LWC, ISO>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(strip3d_kernel<NX, M, MODE, NF, MINB, EO, LWC>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
+    return launch_dependent(strip3d_kernel<NX, M, MODE, NF, MINB, EO, LWC, ISO>, dim3(blocks), dim3(S3_WARPS * 32), smem, s, P, linepoly, g);
+}
+
+// cubic cells on wide rows with constant forcing: the variant compiled for them
+template <int NX, int M, int MODE, bool NF, int MINB, bool EO, int LWC>
+cudaError_t launch_nmfe(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+    if constexpr (NX == 8 && LWC == 32 && !NF) {
+        if (P.hx == P.hy && P.hy == P.hz) return launch_nmfei<NX, M, MODE, NF, MINB, EO, LWC, true>(P, linepoly, g, s);
+    }
+    return launch_nmfei<NX, M, MODE, NF, MINB, EO, LWC, false>(P, linepoly, g, s);
 }
 
 // no output array: the energy-only variant
