@@ -12,7 +12,12 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdn.so")
-SOURCES = ["dn_api.cu", "dn_aux.cu", "dn_generic.cu", "dn_tiled2d.cu", "dn_strip2d.cu", "dn_row2d.cu", "dn_tiled3d.cu", "dn_strip3d.cu", "dn_static.cu", "dn_burgers.cu", "dn_cg.cu"]
+# (source, object name, extra flags): the 3D strip kernel is compiled in two parts (its template instantiations for
+# m <= 4 and for m >= 5), which run side by side
+SOURCES = [(f, f.replace(".cu", ".o"), []) for f in
+           ["dn_api.cu", "dn_aux.cu", "dn_generic.cu", "dn_tiled2d.cu", "dn_strip2d.cu", "dn_row2d.cu", "dn_tiled3d.cu",
+            "dn_strip3d.cu", "dn_static.cu", "dn_burgers.cu", "dn_cg.cu"]]
+SOURCES.append(("dn_strip3d.cu", "dn_strip3d_hi.o", ["-DDN_S3_PART=1"]))
 HEADERS = [os.path.join(CSRC, "dn_internal.cuh"), os.path.join(ROOT, "include", "dn.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
@@ -31,13 +36,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(objdir, exist_ok=True)
     objs = []
     procs = []
-    for src in SOURCES:
+    for src, objname, extra in SOURCES:
         path = os.path.join(CSRC, src)
-        obj = os.path.join(objdir, src.replace(".cu", ".o"))
+        obj = os.path.join(objdir, objname)
         objs.append(obj)
         if force or _stale(obj, [path] + HEADERS):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", path, "-o", obj]
-            procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", path, "-o", obj]
+            procs.append((objname, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     failed = False
     for src, p in procs:
         out, _ = p.communicate()

@@ -93,6 +93,15 @@ template <int N> __device__ __forceinline__ void s3_wait() { asm volatile("cp.as
 // i = 0..M, padded to a multiple of 4.
 __host__ __device__ constexpr int s3_gs(int m) { return (2 * (m + 1) + 3) / 4 * 4; }
 
+}  // namespace
+
+// The file is compiled twice to halve the build time: DN_S3_PART 0 (the default) holds everything and the kernels for
+// m <= 4 and for the stored field; part 1 holds only the kernels for m = 5..8 and hands them out through
+// launch_strip3d_hi.
+#ifndef DN_S3_PART
+#define DN_S3_PART 0
+#endif
+
 struct S3Geo {
     int Ry, Z;            // element rows per tile, element planes per chunk
     int ntile, nchunk;
@@ -100,6 +109,9 @@ struct S3Geo {
     int C, RS;            // ring slots (rows) per unit, floats per slot
     long long units;
 };
+cudaError_t launch_strip3d_hi(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s);
+
+namespace {
 
 // nu at the 8 Gauss points of one element, index [p][q][s] -> n[4 p + 2 q + s]: four packed Horner chains
 // (column p, row q), each over the planes s = a, b.
@@ -999,6 +1011,18 @@ dn_problem s3_problem_of(const Params& P) {
 
 }  // namespace
 
+#if DN_S3_PART == 1
+cudaError_t launch_strip3d_hi(const Params& P, const float* linepoly, const S3Geo& g, cudaStream_t s) {
+    switch (P.m) {
+        case 5: return launch_m3<5>(P, linepoly, g, s);
+        case 6: return launch_m3<6>(P, linepoly, g, s);
+        case 7: return launch_m3<7>(P, linepoly, g, s);
+        case 8: return launch_m3<8>(P, linepoly, g, s);
+    }
+    return cudaErrorInvalidValue;
+}
+#else
+
 // Rows of at most 128 nodes take 4 nodes per lane, rows of at most 256 nodes 8 (then nx must be a multiple of 8,
 // so that only the last element of the last lane falls outside the grid).
 bool strip3d_applicable(const dn_problem& p) {
@@ -1073,10 +1097,7 @@ cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t 
         case 2: e = launch_m3<2>(P, linepoly, g, s); break;
         case 3: e = launch_m3<3>(P, linepoly, g, s); break;
         case 4: e = launch_m3<4>(P, linepoly, g, s); break;
-        case 5: e = launch_m3<5>(P, linepoly, g, s); break;
-        case 6: e = launch_m3<6>(P, linepoly, g, s); break;
-        case 7: e = launch_m3<7>(P, linepoly, g, s); break;
-        case 8: e = launch_m3<8>(P, linepoly, g, s); break;
+        default: e = launch_strip3d_hi(P, linepoly, g, s); break;      // m = 5..8: compiled in the second part
     }
     if (e != cudaSuccess || P.r == nullptr) return e;       // energy only: no seams
     const long long nA = (long long)P.batch * (g.ntile - 1) * P.nz * (P.nx / 4);
@@ -1088,5 +1109,6 @@ cudaError_t launch_strip3d(const Params& P, const float* linepoly, cudaStream_t 
     }
     return cudaSuccess;
 }
+#endif  // DN_S3_PART
 
 }  // namespace dn
