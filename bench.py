@@ -44,12 +44,12 @@ NCU_CAPTURES = {
                                                "src": "dn_strip2d.cu", "sha": "5ba6034b044c172f"},
     "strip2d:cfg2_2d_2048^2_b16_m6:nodal": {"traffic": 790611967, "fp32_ops_per_element": 35.9,
                                              "src": "dn_strip2d.cu", "sha": "5ba6034b044c172f"},
-    "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 611229440, "fp32_ops_per_element": 133.8,
-                                        "src": "dn_strip3d.cu", "sha": "af3df288f589c63b"},
-    "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 835668736, "fp32_ops_per_element": 142.2,
-                                           "src": "dn_strip3d.cu", "sha": "af3df288f589c63b"},
-    "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 557353728, "fp32_ops_per_element": 145.9,
-                                             "src": "dn_strip3d.cu", "sha": "af3df288f589c63b"},
+    "strip3d:cfg4_3d_256^3_b4_m3:kl": {"traffic": 609947136, "fp32_ops_per_element": 133.8,
+                                        "src": "dn_strip3d.cu", "sha": "f6a30d05f0f96c9e"},
+    "strip3d:cfg4_3d_256^3_b4_m3:nodal": {"traffic": 837124096, "fp32_ops_per_element": 142.2,
+                                           "src": "dn_strip3d.cu", "sha": "f6a30d05f0f96c9e"},
+    "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 557637888, "fp32_ops_per_element": 145.9,
+                                             "src": "dn_strip3d.cu", "sha": "f6a30d05f0f96c9e"},
     "row2d:cfg1_2d_256^2_b64_m4:kl": {"traffic": 17594624, "fp32_ops_per_element": 51.0,
                                        "src": "dn_row2d.cu", "sha": "cc267857ef1ac237"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
