@@ -33,10 +33,10 @@ struct TableArgs {
 // g_i = sum_j ckl[i][j] cos(j pi y_q) are the coefficients in the Chebyshev basis (cos(i pi x) = T_i(c)), converted
 // to monomials in double.  The scaled weights and the cosines are rounded to float first, exactly as the tables
 // hold them, so every kernel family sees the same numbers.  Entry 2k + q of the row; the two Gauss rows of an
-// element row interleave so that they can be evaluated together with two-wide FMAs.  Loops run to the compiled
-// maximum with zero coefficients beyond m, which keeps the small arrays in registers.
+// element row interleave so that they can be evaluated together with two-wide FMAs.  MX >= m is the compiled loop
+// bound (the kernel is instantiated for every m; compile-time bounds keep the small arrays in registers).
+template <int MX>
 __device__ void rowpoly_entry(const TableArgs& A, long long idx) {
-    constexpr int MX = DN_MAX_KL_MODES;
     const int m = A.m, ny = A.n[1];
     const int q = (int)(idx & 1);
     const int rows = A.rp_nodes ? ny : ny - 1;
@@ -88,10 +88,11 @@ __device__ void rowpoly_entry(const TableArgs& A, long long idx) {
     }
     float* dst = A.rowpoly + row * A.rp_gs + q;
 #pragma unroll
-    for (int k = 0; k <= MX; ++k)
-        if (2 * k + q < A.rp_gs) dst[2 * k] = (k <= m) ? (float)acc[k] : 0.f;
+    for (int k = 0; k <= MX; ++k) dst[2 * k] = (float)acc[k];
+    for (int k = MX + 1; 2 * k + q < A.rp_gs; ++k) dst[2 * k] = 0.f;      // the padding of the row
 }
 
+template <int MX>
 __global__ void tables_kernel(TableArgs A) {
     dep_wait();                                        // whatever ran before in the stream may still read these tables
     dep_release();
@@ -137,7 +138,7 @@ __global__ void tables_kernel(TableArgs A) {
         }
         idx -= cnt;
     }
-    if (A.rowpoly && idx < 2ll * A.batch * (A.n[1] - (A.rp_nodes ? 0 : 1))) rowpoly_entry(A, idx);
+    if (A.rowpoly && idx < 2ll * A.batch * (A.n[1] - (A.rp_nodes ? 0 : 1))) rowpoly_entry<MX>(A, idx);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -330,7 +331,17 @@ cudaError_t launch_tables(const Params& P, const float* kl_w, float* ckl, float*
     A.rowpoly = (P.dim == 2) ? rowpoly : nullptr; A.rp_gs = rowpoly_stride; A.rp_nodes = rowpoly_nodes ? 1 : 0;
     if (A.rowpoly) total += 2ll * P.batch * (P.ny - (rowpoly_nodes ? 0 : 1));
     const int threads = 128;
-    return launch_dependent(tables_kernel, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, s, A);
+    const dim3 grid((unsigned)((total + threads - 1) / threads));
+    switch (A.rowpoly ? P.m : DN_MAX_KL_MODES) {       // the loop bound matters to the row polynomials only
+        case 1: return launch_dependent(tables_kernel<1>, grid, dim3(threads), 0, s, A);
+        case 2: return launch_dependent(tables_kernel<2>, grid, dim3(threads), 0, s, A);
+        case 3: return launch_dependent(tables_kernel<3>, grid, dim3(threads), 0, s, A);
+        case 4: return launch_dependent(tables_kernel<4>, grid, dim3(threads), 0, s, A);
+        case 5: return launch_dependent(tables_kernel<5>, grid, dim3(threads), 0, s, A);
+        case 6: return launch_dependent(tables_kernel<6>, grid, dim3(threads), 0, s, A);
+        case 7: return launch_dependent(tables_kernel<7>, grid, dim3(threads), 0, s, A);
+    }
+    return launch_dependent(tables_kernel<DN_MAX_KL_MODES>, grid, dim3(threads), 0, s, A);
 }
 
 cudaError_t launch_finalize(const double* partials, int nblk, int batch, float* J, cudaStream_t s) {
