@@ -50,6 +50,8 @@ NCU_CAPTURES = {
                                            "src": "dn_strip3d.cu", "sha": "f6a30d05f0f96c9e"},
     "strip3d:cfg4_3d_256^3_b4_m3:klnodal": {"traffic": 557637888, "fp32_ops_per_element": 145.9,
                                              "src": "dn_strip3d.cu", "sha": "f6a30d05f0f96c9e"},
+    "strip3d:cfg3_3d_64^3_b32_m2:kl": {"traffic": 49059584, "fp32_ops_per_element": 129.6,
+                                        "src": "dn_strip3d.cu", "sha": "f6a30d05f0f96c9e"},
     "row2d:cfg1_2d_256^2_b64_m4:kl": {"traffic": 17594624, "fp32_ops_per_element": 51.0,
                                        "src": "dn_row2d.cu", "sha": "cc267857ef1ac237"},
     "march:burgers_1024x1024_b64": {"traffic": 499482880, "fp32_ops_per_element": 26.3,
